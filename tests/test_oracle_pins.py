@@ -367,7 +367,7 @@ def test_plane_encode_equals_slice_by_slice_and_handles_ragged_tail():
     # don't-care outputs are the raw network outputs
     raw = np.concatenate([orc.xor_network(M, seed_bits(int(v), 8)) for v in wc])[:mn]
     flips = np.zeros(mn, np.uint8)
-    starts = np.concatenate([[0], np.cumsum(np_)])
+    starts = np.concatenate([[0], np.cumsum(np_.astype(np.int64))]).astype(np.int64)
     for s in range(8):
         for k in range(starts[s], starts[s + 1]):
             flips[s * 80 + dp[k]] ^= 1
@@ -445,5 +445,6 @@ def test_matmul_general_case_against_numpy():
     Y = orc.matmul(planes, mask, alpha, X)
     assert Y.shape == (batch, m)
     assert np.allclose(Y, X @ W.T, rtol=1e-13, atol=1e-13)
-    # a transposed or unmasked product differs
-    assert not np.allclose(Y, X @ (W / np.maximum(mask, 1)).T) or mask.all()
+    # dropping the mask changes the result (the mask really is applied)
+    W_unmasked = ((planes.astype(np.float64) * 2 - 1) * alpha.astype(np.float64).T[:, :, None]).sum(axis=0)
+    assert not np.allclose(Y, X @ W_unmasked.T)
