@@ -1,0 +1,194 @@
+/*
+ * sqnn.h -- C interface of the B200 (sm_100a) library that decodes XOR-gate-network
+ * encrypted weight bit-planes and multiplies the decoded sparse quantized weights with
+ * activations ("Structured Compression by Weight Encryption for Unstructured Pruning and
+ * Quantization", Kwon et al.).
+ *
+ * Notation (the paper's): a layer has m x n weights, pruned by a mask and quantized to n_q
+ * binary-code bit-planes W^q_i (Section 3.1).  Each plane is flattened row-major (flat
+ * position p = r*n + c) and cut into l = ceil(mn / n_out) slices of n_out positions
+ * (Section 3.1; l in Section 3.2).  A slice w^q is stored as its encrypted seed w^c of n_in
+ * bits; the fixed network M (n_out x n_in over GF(2)) expands it: w~ = M . w^c.  Care bits
+ * the network could not produce are listed as n_patch (count, same width for every slice of
+ * a plane) and d_patch (positions inside the slice) and are flipped after the expansion
+ * (Section 3.2).  Positions past mn in the last slice are don't-cares.
+ *
+ * General rules
+ *  - Plain C.  Every function returns an int status (SQNN_OK = 0, negative = error) unless
+ *    noted; nothing aborts, throws or prints.
+ *  - "host" pointers are ordinary process memory, "device" pointers are CUDA global memory
+ *    of the current device.  All pointers are borrowed for the call; device pointers must
+ *    stay valid until the work queued on the stream has run.
+ *  - Device entry points only queue work on the given CUDA stream (a cudaStream_t passed as
+ *    void*, NULL = the legacy default stream) and do not synchronise.  They allocate no
+ *    device memory and create no streams.
+ *  - Host buffers the library returns (blob, unpacked arrays) are released with sqnn_free.
+ *  - d_status (device, one uint32, may be NULL) receives a sticky non-zero code when a
+ *    kernel had to skip a malformed patch entry (position >= n_out, or a patch index past
+ *    the end of the d_patch section); the caller zeroes it.  Kernels never trap.
+ */
+#ifndef SQNN_H_
+#define SQNN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SQNN_MAX_PLANES   8      /* n_q <= 8                                            */
+#define SQNN_MAX_N_OUT    256    /* n_out <= 256: a d_patch position fits one byte      */
+#define SQNN_MAX_N_IN     32     /* n_in <= 32: a seed fits one uint32                  */
+#define SQNN_BLOCK_SLICES 128    /* one d_patch offset is stored per 128 slices         */
+#define SQNN_PAD_SLICES   1024   /* streams are zero-padded to a multiple of 1024 slices*/
+#define SQNN_MAX_BATCH    1024
+
+enum {
+    SQNN_OK            =  0,
+    SQNN_E_INVALID_ARG = -1,   /* NULL where data is required, size / range out of bounds */
+    SQNN_E_BAD_BLOB    = -2,   /* blob fails validation                                   */
+    SQNN_E_UNSUPPORTED = -3,   /* valid request the library has no path for               */
+    SQNN_E_NOMEM       = -4,   /* host allocation failed                                  */
+    SQNN_E_CUDA        = -5,   /* a CUDA runtime call failed (launch configuration, ...)  */
+    SQNN_E_TIMEOUT     = -6,   /* a bounded device-side wait gave up (status word only)   */
+    SQNN_E_WORKSPACE   = -7    /* workspace missing or smaller than sqnn_workspace_bytes  */
+};
+
+/* encode flags */
+#define SQNN_ENCODE_ALG1        0u   /* Algorithm 1 (patch searching), the default           */
+#define SQNN_ENCODE_EXHAUSTIVE  1u   /* all 2^n_in seeds, fewest patches (Section 5.2); n_in <= 20 */
+
+/* activation element types of sqnn_decode_matmul */
+#define SQNN_X_F32   0
+#define SQNN_X_BF16  1
+
+/* The XOR-gate network M (Section 3.1): rows[j] bit t = M[j][t], j < n_out, t < n_in. host */
+typedef struct sqnn_xornet {
+    uint32_t n_out, n_in;
+    const uint32_t *rows;
+} sqnn_xornet;
+
+/* Quantized, pruned layer as packed bits (host).  Bit p of a vector = (word[p >> 6] >> (p & 63)) & 1.
+ * planes: n_q consecutive vectors of ceil(mn / 64) words, bit 1 <-> +1.  mask: 1 = care (unpruned). */
+typedef struct sqnn_planes {
+    uint64_t m, n;
+    uint32_t n_q;
+    const uint64_t *planes;
+    const uint64_t *mask;
+} sqnn_planes;
+
+/* Size accounting.  bpw_eq1 = sum over planes of 1 / r with r from Eq. 1 taken literally
+ * (ceil(lg max p) bits per n_patch, ceil(lg n_out) bits per d_patch entry).  bpw_actual counts
+ * the bytes of the blob sections as stored (padding and the per-128-slice offsets included,
+ * header and the network excluded), per weight.  The pruning mask (1 bit / weight, kept
+ * outside the blob) is not part of either. */
+typedef struct sqnn_stats {
+    uint64_t slices;                          /* l per plane                              */
+    uint64_t patches[SQNN_MAX_PLANES];        /* sum of n_patch per plane                 */
+    uint32_t max_patch[SQNN_MAX_PLANES];      /* max n_patch per plane                    */
+    uint64_t bits_wc, bits_npatch, bits_dpatch, bits_index;   /* stored sizes, all planes */
+    double   bpw_eq1, bpw_actual;
+} sqnn_stats;
+
+/* Parsed blob header.  Offsets are bytes from the start of the blob, each a multiple of 16.
+ * Per plane i: the w^c stream (slice s occupies bits [s*n_in, (s+1)*n_in), least significant
+ * bit first inside little-endian 32-bit words); the n_patch stream (w_np[i] bits per slice,
+ * same packing; absent when w_np[i] = 0); the offsets (uint32 per block of 128 slices: number
+ * of d_patch entries before the block, plus one closing entry = n_dp[i]); the d_patch entries
+ * (one byte each, slice order, ascending inside a slice).  Streams cover slices_padded slices
+ * (padding slices have seed 0 and no patch) and every section ends with >= 16 zero bytes. */
+typedef struct sqnn_desc {
+    uint64_t m, n, slices, slices_padded;
+    uint32_t n_q, n_out, n_in, block_slices;
+    uint32_t w_np[SQNN_MAX_PLANES];
+    uint32_t w_dp;                            /* bits per stored d_patch entry (8)        */
+    uint32_t reserved;
+    uint64_t off_xornet;                      /* n_out uint32 rows                        */
+    uint64_t off_wc[SQNN_MAX_PLANES], off_np[SQNN_MAX_PLANES];
+    uint64_t off_idx[SQNN_MAX_PLANES], off_dp[SQNN_MAX_PLANES];
+    uint64_t n_dp[SQNN_MAX_PLANES];
+    uint64_t total_bytes;
+} sqnn_desc;
+
+/* Encryption of every slice of every plane (Section 3.1, Algorithm 1 of Section 3.3; with
+ * SQNN_ENCODE_EXHAUSTIVE the search of Section 5.2) and packing into one blob.  Host only.
+ * Readings fixed here: care positions are tried in ascending order; the kept system is solved
+ * with all free variables 0 (pivot columns of the reduced row-echelon form, lowest column
+ * first), a slice without care bits gets seed 0; d_patch lists the care positions whose
+ * expanded bit is wrong.  *blob is allocated by the library (sqnn_free).  stats may be NULL.
+ * Errors: INVALID_ARG (NULL, n_out/n_in/n_q out of range, m*n = 0), NOMEM. */
+int sqnn_encode_host(const sqnn_xornet *net, const sqnn_planes *layer, uint32_t flags,
+                     void **blob, size_t *blob_bytes, sqnn_stats *stats);
+
+/* Packs logical per-plane arrays (the three parts of the format, Section 3.2) into a blob:
+ * wc[i][s] seed of slice s (bit t = w^c[t]), np[i][s] = n_patch, dp[i] = all d_patch entries of
+ * plane i in slice order.  Arrays are host, length l, l and sum(np[i]).  Errors: INVALID_ARG
+ * (also for a seed >= 2^n_in or a position >= n_out), NOMEM. */
+int sqnn_pack_host(const sqnn_xornet *net, uint64_t m, uint64_t n, uint32_t n_q,
+                   const uint32_t *const *wc, const uint16_t *const *np, const uint16_t *const *dp,
+                   void **blob, size_t *blob_bytes);
+
+/* Inverse of sqnn_pack_host for one plane.  wc / np get l entries, dp gets *n_dp entries; each
+ * array is allocated by the library (sqnn_free).  Validates the blob first (BAD_BLOB). */
+int sqnn_unpack_host(const void *blob, size_t blob_bytes, uint32_t plane,
+                     uint32_t **wc, uint16_t **np, uint16_t **dp, uint64_t *n_dp);
+
+/* Validates a host blob and fills *desc: magic / version, section bounds and alignment, field
+ * widths, offsets non-decreasing and consistent with the n_patch stream, sum(n_patch) = n_dp,
+ * every d_patch entry < n_out, padding slices empty.  BAD_BLOB on any violation. */
+int sqnn_describe_host(const void *blob, size_t blob_bytes, sqnn_desc *desc);
+
+/* Size accounting of a host blob (Eq. 1, Section 3.2, and stored bytes). */
+int sqnn_stats_host(const void *blob, size_t blob_bytes, sqnn_stats *stats);
+
+/* Releases memory returned by the functions above.  NULL is allowed. */
+void sqnn_free(void *p);
+
+typedef enum sqnn_out_mode {
+    SQNN_OUT_BITS = 0,   /* decoded planes as packed bits: n_q vectors of ceil(mn/64) uint64 words,
+                            bit layout as sqnn_planes.planes; bits past mn in the last word are 0.
+                            All positions are written, don't-care positions included.            */
+    SQNN_OUT_BF16 = 1,   /* dense m x n bf16 (row-major): 0 where mask = 0, else the fp32 sum
+                            (+-alpha[r][0]) + (+-alpha[r][1]) + ... in plane order, rounded to
+                            bf16 nearest-even; bit 1 <-> +alpha.  Needs d_mask and d_alpha.       */
+    SQNN_OUT_SINK = 2    /* one uint64: XOR of all words of the BITS output (measures the pure
+                            compressed-stream rate; nothing but 8 bytes is written).             */
+} sqnn_out_mode;
+
+/* Decryption of a whole layer on the device (Section 3.1: w~ = M . w^c; Section 3.2: flip the
+ * d_patch positions).  desc: host, from sqnn_describe_host.  d_blob: device copy of the same
+ * blob, 16-byte aligned.  d_mask: device, ceil(mn/64) uint64 (BF16 mode only, else may be NULL).
+ * d_alpha: device, m x n_q floats row-major (BF16 mode only).  d_out: device, out_bytes bytes:
+ * BITS n_q*ceil(mn/64)*8, BF16 mn*2, SINK 8; 16-byte aligned.  Errors: INVALID_ARG (NULL,
+ * misaligned, out_bytes too small), UNSUPPORTED, CUDA. */
+int sqnn_decode(const sqnn_desc *desc, const void *d_blob, const uint64_t *d_mask,
+                const float *d_alpha, sqnn_out_mode mode, void *d_out, size_t out_bytes,
+                uint32_t *d_status, void *cuda_stream);
+
+/* Decryption fused with the product the layer exists for: Y[b][r] = sum_c W[r][c] * X[b][c],
+ * W[r][c] = mask[r][c] * sum_i alpha[r][i] * (2 b_i[r][c] - 1) with b_i the decoded planes
+ * (Sections 3.1, 3.2; the sparse quantized product of Section 1).  The decoded weights never
+ * reach global memory.  d_x: device, batch rows of n elements (x_dtype SQNN_X_F32 or
+ * SQNN_X_BF16), row stride ldx elements.  d_y: device fp32, batch rows of m, row stride ldy;
+ * fully overwritten.  batch <= 15 runs the fp32-accumulate GEMV kernel (weights exact);
+ * batch >= 16 runs the tcgen05 kernel (weights rounded to bf16, activations must be BF16,
+ * fp32 accumulation in tensor memory).  d_workspace: device scratch of at least
+ * sqnn_workspace_bytes(desc, batch) bytes, 256-byte aligned, contents undefined before and
+ * after (may be NULL when that size is 0).  Errors: INVALID_ARG, UNSUPPORTED (F32 activations
+ * with batch >= 16, batch > SQNN_MAX_BATCH), WORKSPACE, CUDA. */
+int sqnn_decode_matmul(const sqnn_desc *desc, const void *d_blob, const uint64_t *d_mask,
+                       const float *d_alpha, const void *d_x, int x_dtype, uint32_t batch,
+                       int64_t ldx, float *d_y, int64_t ldy, void *d_workspace,
+                       size_t workspace_bytes, uint32_t *d_status, void *cuda_stream);
+
+/* Scratch bytes sqnn_decode_matmul needs for this layer and batch (0 if none). */
+size_t sqnn_workspace_bytes(const sqnn_desc *desc, uint32_t batch);
+
+/* Human-readable name of a status code; never NULL. */
+const char *sqnn_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SQNN_H_ */

@@ -1,0 +1,474 @@
+// Host side of the library: encryption of slices (Algorithm 1 / exhaustive search), the
+// packed blob format, its validation and size accounting.  No CUDA in this file.
+#include "sqnn.h"
+#include "sqnn_blob.h"
+
+#include <algorithm>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+namespace {
+
+inline int popc64(uint64_t v) { return __builtin_popcountll(v); }
+inline int ctz32(uint32_t v) { return __builtin_ctz(v); }
+
+// `count` (<= 64) bits of a packed vector starting at flat position p; positions >= limit read 0.
+inline uint64_t window(const uint64_t *words, uint64_t p, uint32_t count, uint64_t limit)
+{
+    if (p >= limit) return 0;
+    if (p + count > limit) count = (uint32_t)(limit - p);
+    const uint64_t w = p >> 6;
+    const uint32_t sh = (uint32_t)(p & 63);
+    uint64_t v = words[w] >> sh;
+    if (sh && sh + count > 64) v |= words[w + 1] << (64 - sh);
+    if (count < 64) v &= ((uint64_t)1 << count) - 1;
+    return v;
+}
+
+inline uint32_t ceil_lg_u64(uint64_t v)   // smallest e with 2^e >= v (0 for v <= 1)
+{
+    uint32_t e = 0;
+    while (((uint64_t)1 << e) < v) ++e;
+    return e;
+}
+
+struct SliceBits {            // wanted bits and care flags of one slice, n_out <= 256
+    uint64_t want[4];
+    uint64_t care[4];
+};
+
+inline void load_slice(const uint64_t *plane, const uint64_t *mask, uint64_t mn, uint32_t n_out,
+                       uint64_t s, SliceBits &sb)
+{
+    const uint64_t p0 = s * (uint64_t)n_out;
+    for (uint32_t k = 0; k < 4; ++k) {
+        const uint32_t lo = k * 64;
+        if (lo >= n_out) { sb.want[k] = sb.care[k] = 0; continue; }
+        const uint32_t cnt = std::min<uint32_t>(64, n_out - lo);
+        sb.care[k] = window(mask, p0 + lo, cnt, mn);
+        sb.want[k] = window(plane, p0 + lo, cnt, mn);
+    }
+}
+
+// w~ = M . w^c over GF(2): bit j = parity(rows[j] AND seed)
+inline void expand(const uint32_t *rows, uint32_t n_out, uint32_t seed, uint64_t out[4])
+{
+    out[0] = out[1] = out[2] = out[3] = 0;
+    for (uint32_t j = 0; j < n_out; ++j)
+        out[j >> 6] |= (uint64_t)(__builtin_popcount(rows[j] & seed) & 1) << (j & 63);
+}
+
+// Algorithm 1 on one slice.  The augmented matrix is kept in reduced row-echelon form while
+// care rows are appended in ascending position: a new row is first reduced against the pivots;
+// if it reduces to 0 = 1 it is the unsolvable case and is dropped (it will show up as a patch),
+// if it reduces to 0 = 0 it is redundant, otherwise its lowest set column becomes a new pivot
+// and is eliminated from the older rows.  Free variables are 0, so a pivot variable equals the
+// right-hand side of its row.
+inline uint32_t encode_alg1(const uint32_t *rows, uint32_t n_out, const SliceBits &sb)
+{
+    uint32_t prow[SQNN_MAX_N_IN], pcol[SQNN_MAX_N_IN];
+    uint8_t prhs[SQNN_MAX_N_IN];
+    uint32_t npiv = 0;
+    for (uint32_t k = 0; k * 64 < n_out; ++k) {
+        uint64_t c = sb.care[k];
+        while (c) {
+            const uint32_t j = k * 64 + (uint32_t)__builtin_ctzll(c);
+            c &= c - 1;
+            uint32_t a = rows[j];
+            uint8_t b = (uint8_t)((sb.want[k] >> (j & 63)) & 1);
+            for (uint32_t q = 0; q < npiv; ++q)
+                if ((a >> pcol[q]) & 1) { a ^= prow[q]; b ^= prhs[q]; }
+            if (a == 0) continue;                 // redundant or contradictory: nothing to keep
+            const uint32_t col = (uint32_t)ctz32(a);
+            for (uint32_t q = 0; q < npiv; ++q)
+                if ((prow[q] >> col) & 1) { prow[q] ^= a; prhs[q] ^= b; }
+            prow[npiv] = a; prhs[npiv] = b; pcol[npiv] = col;
+            ++npiv;
+        }
+    }
+    uint32_t seed = 0;
+    for (uint32_t q = 0; q < npiv; ++q)
+        if (prhs[q]) seed |= 1u << pcol[q];
+    return seed;
+}
+
+// All 2^n_in outputs of the network, 4 words each.
+void build_outputs(const uint32_t *rows, uint32_t n_out, uint32_t n_in, std::vector<uint64_t> &tab)
+{
+    const uint64_t cnt = (uint64_t)1 << n_in;
+    tab.assign(cnt * 4, 0);
+    for (uint64_t v = 0; v < cnt; ++v) expand(rows, n_out, (uint32_t)v, &tab[v * 4]);
+}
+
+inline uint32_t encode_exhaustive(const std::vector<uint64_t> &tab, uint32_t n_in, const SliceBits &sb)
+{
+    const uint64_t cnt = (uint64_t)1 << n_in;
+    uint32_t best = 0;
+    int best_wrong = 1 << 30;
+    for (uint64_t v = 0; v < cnt; ++v) {
+        const uint64_t *o = &tab[v * 4];
+        int wrong = 0;
+        for (int k = 0; k < 4; ++k) wrong += popc64((o[k] ^ sb.want[k]) & sb.care[k]);
+        if (wrong < best_wrong) { best_wrong = wrong; best = (uint32_t)v; }
+    }
+    return best;
+}
+
+struct PlaneArrays {
+    std::vector<uint32_t> wc;
+    std::vector<uint16_t> np;
+    std::vector<uint8_t> dp;
+};
+
+uint64_t round_up(uint64_t v, uint64_t a) { return (v + a - 1) / a * a; }
+
+// Packs bit fields of `width` bits (value i at bits [i*width, (i+1)*width)) into uint32 words.
+// Groups of 32 values fill whole words, so groups can be written independently.
+template <typename T>
+void pack_fields(const T *vals, uint64_t count, uint32_t width, uint32_t *dst)
+{
+    if (width == 0) return;
+    const int64_t groups = (int64_t)((count + 31) / 32);
+#pragma omp parallel for schedule(static)
+    for (int64_t g = 0; g < groups; ++g) {
+        uint32_t *w = dst + (uint64_t)g * width;
+        uint64_t acc = 0;
+        uint32_t have = 0, wi = 0;
+        const uint64_t lo = (uint64_t)g * 32, hi = std::min<uint64_t>(count, lo + 32);
+        for (uint64_t i = lo; i < hi; ++i) {
+            acc |= (uint64_t)vals[i] << have;
+            have += width;
+            while (have >= 32) { w[wi++] = (uint32_t)acc; acc >>= 32; have -= 32; }
+        }
+        if (have) w[wi] = (uint32_t)acc;
+    }
+}
+
+inline uint32_t read_field(const uint32_t *src, uint64_t index, uint32_t width)
+{
+    if (width == 0) return 0;
+    const uint64_t bit = index * width;
+    const uint64_t w = bit >> 5;
+    const uint32_t sh = (uint32_t)(bit & 31);
+    uint64_t v = (uint64_t)src[w] | ((uint64_t)src[w + 1] << 32);   // sections end with slack
+    return (uint32_t)((v >> sh) & (((uint64_t)1 << width) - 1));
+}
+
+int build_blob(const sqnn_xornet *net, uint64_t m, uint64_t n, uint32_t n_q,
+               const uint32_t *const *wc, const uint16_t *const *np, const uint8_t *const *dp8,
+               const uint16_t *const *dp16, void **blob, size_t *blob_bytes)
+{
+    const uint64_t mn = m * n;
+    const uint32_t n_out = net->n_out, n_in = net->n_in;
+    const uint64_t l = (mn + n_out - 1) / n_out;
+    const uint64_t lp = round_up(l, SQNN_PAD_SLICES);
+    sqnn_desc d;
+    std::memset(&d, 0, sizeof d);
+    d.m = m; d.n = n; d.slices = l; d.slices_padded = lp;
+    d.n_q = n_q; d.n_out = n_out; d.n_in = n_in; d.block_slices = SQNN_BLOCK_SLICES;
+    d.w_dp = 8;
+    uint64_t off = SQNN_BLOB_HEADER_BYTES;
+    d.off_xornet = off;
+    off += round_up((uint64_t)n_out * 4, 16) + 16;
+    std::vector<uint64_t> ndp(n_q, 0);
+    for (uint32_t i = 0; i < n_q; ++i) {
+        uint32_t maxp = 0;
+        uint64_t sum = 0;
+        for (uint64_t s = 0; s < l; ++s) {
+            if (np[i][s] > n_out) return SQNN_E_INVALID_ARG;
+            maxp = std::max<uint32_t>(maxp, np[i][s]);
+            sum += np[i][s];
+        }
+        ndp[i] = sum;
+        d.n_dp[i] = sum;
+        d.w_np[i] = ceil_lg_u64((uint64_t)maxp + 1);
+        d.off_wc[i] = off;  off += round_up(lp * n_in / 8, 16) + 16;
+        d.off_np[i] = off;  if (d.w_np[i]) off += round_up(lp * d.w_np[i] / 8, 16) + 16;
+        d.off_idx[i] = off; off += round_up((lp / SQNN_BLOCK_SLICES + 1) * 4, 16) + 16;
+        d.off_dp[i] = off;  off += round_up(sum, 16) + 16;
+    }
+    d.total_bytes = off;
+    uint8_t *b = (uint8_t *)std::calloc(off, 1);
+    if (!b) return SQNN_E_NOMEM;
+    sqnn_blob_header *h = (sqnn_blob_header *)b;
+    std::memcpy(h->magic, SQNN_BLOB_MAGIC, 8);
+    h->version = SQNN_BLOB_VERSION;
+    h->header_bytes = SQNN_BLOB_HEADER_BYTES;
+    h->desc = d;
+    std::memcpy(b + d.off_xornet, net->rows, (size_t)n_out * 4);
+    const uint32_t seed_limit_bits = n_in;
+    for (uint32_t i = 0; i < n_q; ++i) {
+        if (seed_limit_bits < 32)
+            for (uint64_t s = 0; s < l; ++s)
+                if (wc[i][s] >> seed_limit_bits) { std::free(b); return SQNN_E_INVALID_ARG; }
+        pack_fields(wc[i], l, n_in, (uint32_t *)(b + d.off_wc[i]));
+        pack_fields(np[i], l, d.w_np[i], (uint32_t *)(b + d.off_np[i]));
+        uint32_t *idx = (uint32_t *)(b + d.off_idx[i]);
+        uint8_t *dst = b + d.off_dp[i];
+        uint64_t run = 0;
+        const uint64_t blocks = lp / SQNN_BLOCK_SLICES;
+        for (uint64_t blk = 0; blk <= blocks; ++blk) {
+            idx[blk] = (uint32_t)run;
+            if (blk == blocks) break;
+            const uint64_t lo = blk * SQNN_BLOCK_SLICES, hi = std::min<uint64_t>(l, lo + SQNN_BLOCK_SLICES);
+            for (uint64_t s = lo; s < hi; ++s) run += np[i][s];
+        }
+        if (run != ndp[i] || ndp[i] > 0xffffffffull) { std::free(b); return SQNN_E_INVALID_ARG; }
+        for (uint64_t k = 0; k < ndp[i]; ++k) {
+            const uint32_t pos = dp8 ? dp8[i][k] : dp16[i][k];
+            if (pos >= n_out) { std::free(b); return SQNN_E_INVALID_ARG; }
+            dst[k] = (uint8_t)pos;
+        }
+    }
+    *blob = b;
+    *blob_bytes = off;
+    return SQNN_OK;
+}
+
+bool net_ok(const sqnn_xornet *net)
+{
+    return net && net->rows && net->n_out >= 1 && net->n_out <= SQNN_MAX_N_OUT &&
+           net->n_in >= 1 && net->n_in <= SQNN_MAX_N_IN;
+}
+
+}  // namespace
+
+extern "C" {
+
+void sqnn_free(void *p) { std::free(p); }
+
+const char *sqnn_status_string(int status)
+{
+    switch (status) {
+        case SQNN_OK: return "ok";
+        case SQNN_E_INVALID_ARG: return "invalid argument";
+        case SQNN_E_BAD_BLOB: return "malformed blob";
+        case SQNN_E_UNSUPPORTED: return "unsupported";
+        case SQNN_E_NOMEM: return "out of host memory";
+        case SQNN_E_CUDA: return "CUDA runtime error";
+        case SQNN_E_TIMEOUT: return "device-side wait timed out";
+        case SQNN_E_WORKSPACE: return "workspace missing or too small";
+        default: return "unknown status";
+    }
+}
+
+int sqnn_encode_host(const sqnn_xornet *net, const sqnn_planes *layer, uint32_t flags,
+                     void **blob, size_t *blob_bytes, sqnn_stats *stats)
+{
+    if (!net_ok(net) || !layer || !blob || !blob_bytes) return SQNN_E_INVALID_ARG;
+    if (!layer->planes || !layer->mask || layer->n_q < 1 || layer->n_q > SQNN_MAX_PLANES)
+        return SQNN_E_INVALID_ARG;
+    if (layer->m == 0 || layer->n == 0 || layer->m > ((uint64_t)1 << 40) / layer->n)
+        return SQNN_E_INVALID_ARG;
+    const bool exhaustive = (flags & SQNN_ENCODE_EXHAUSTIVE) != 0;
+    if (exhaustive && net->n_in > 20) return SQNN_E_INVALID_ARG;
+    try {
+        const uint64_t mn = layer->m * layer->n;
+        const uint32_t n_out = net->n_out, n_in = net->n_in, n_q = layer->n_q;
+        const uint64_t l = (mn + n_out - 1) / n_out;
+        const uint64_t words = (mn + 63) / 64;
+        std::vector<uint64_t> tab;
+        if (exhaustive) build_outputs(net->rows, n_out, n_in, tab);
+        std::vector<PlaneArrays> pa(n_q);
+        for (uint32_t i = 0; i < n_q; ++i) {
+            const uint64_t *plane = layer->planes + (uint64_t)i * words;
+            pa[i].wc.assign(l, 0);
+            pa[i].np.assign(l, 0);
+            // pass 1: seed and patch count of every slice (slices are independent)
+#pragma omp parallel for schedule(dynamic, 4096)
+            for (int64_t s = 0; s < (int64_t)l; ++s) {
+                SliceBits sb;
+                load_slice(plane, layer->mask, mn, n_out, (uint64_t)s, sb);
+                const uint32_t seed = exhaustive ? encode_exhaustive(tab, n_in, sb)
+                                                 : encode_alg1(net->rows, n_out, sb);
+                uint64_t out[4];
+                expand(net->rows, n_out, seed, out);
+                int wrong = 0;
+                for (int k = 0; k < 4; ++k) wrong += popc64((out[k] ^ sb.want[k]) & sb.care[k]);
+                pa[i].wc[s] = seed;
+                pa[i].np[s] = (uint16_t)wrong;
+            }
+            // pass 2: positions of the wrong care bits, written at the running offset
+            std::vector<uint64_t> start(l + 1, 0);
+            for (uint64_t s = 0; s < l; ++s) start[s + 1] = start[s] + pa[i].np[s];
+            pa[i].dp.assign(start[l] + 1, 0);
+#pragma omp parallel for schedule(dynamic, 4096)
+            for (int64_t s = 0; s < (int64_t)l; ++s) {
+                if (!pa[i].np[s]) continue;
+                SliceBits sb;
+                load_slice(plane, layer->mask, mn, n_out, (uint64_t)s, sb);
+                uint64_t out[4];
+                expand(net->rows, n_out, pa[i].wc[s], out);
+                uint64_t at = start[s];
+                for (uint32_t k = 0; k * 64 < n_out; ++k) {
+                    uint64_t bad = (out[k] ^ sb.want[k]) & sb.care[k];
+                    while (bad) {
+                        pa[i].dp[at++] = (uint8_t)(k * 64 + (uint32_t)__builtin_ctzll(bad));
+                        bad &= bad - 1;
+                    }
+                }
+            }
+        }
+        std::vector<const uint32_t *> wcp(n_q);
+        std::vector<const uint16_t *> npp(n_q);
+        std::vector<const uint8_t *> dpp(n_q);
+        for (uint32_t i = 0; i < n_q; ++i) { wcp[i] = pa[i].wc.data(); npp[i] = pa[i].np.data(); dpp[i] = pa[i].dp.data(); }
+        int rc = build_blob(net, layer->m, layer->n, n_q, wcp.data(), npp.data(), dpp.data(), nullptr, blob, blob_bytes);
+        if (rc != SQNN_OK) return rc;
+        if (stats) {
+            rc = sqnn_stats_host(*blob, *blob_bytes, stats);
+            if (rc != SQNN_OK) { std::free(*blob); *blob = nullptr; return rc; }
+        }
+        return SQNN_OK;
+    } catch (const std::bad_alloc &) {
+        return SQNN_E_NOMEM;
+    }
+}
+
+int sqnn_pack_host(const sqnn_xornet *net, uint64_t m, uint64_t n, uint32_t n_q,
+                   const uint32_t *const *wc, const uint16_t *const *np, const uint16_t *const *dp,
+                   void **blob, size_t *blob_bytes)
+{
+    if (!net_ok(net) || !wc || !np || !dp || !blob || !blob_bytes) return SQNN_E_INVALID_ARG;
+    if (n_q < 1 || n_q > SQNN_MAX_PLANES || m == 0 || n == 0 || m > ((uint64_t)1 << 40) / n)
+        return SQNN_E_INVALID_ARG;
+    for (uint32_t i = 0; i < n_q; ++i)
+        if (!wc[i] || !np[i] || !dp[i]) return SQNN_E_INVALID_ARG;
+    try {
+        return build_blob(net, m, n, n_q, wc, np, nullptr, dp, blob, blob_bytes);
+    } catch (const std::bad_alloc &) {
+        return SQNN_E_NOMEM;
+    }
+}
+
+int sqnn_describe_host(const void *blob, size_t blob_bytes, sqnn_desc *desc)
+{
+    if (!blob || !desc) return SQNN_E_INVALID_ARG;
+    if (blob_bytes < SQNN_BLOB_HEADER_BYTES) return SQNN_E_BAD_BLOB;
+    const uint8_t *b = (const uint8_t *)blob;
+    sqnn_blob_header h;
+    std::memcpy(&h, b, sizeof h);
+    if (std::memcmp(h.magic, SQNN_BLOB_MAGIC, 8) != 0 || h.version != SQNN_BLOB_VERSION ||
+        h.header_bytes != SQNN_BLOB_HEADER_BYTES)
+        return SQNN_E_BAD_BLOB;
+    const sqnn_desc &d = h.desc;
+    if (d.n_out < 1 || d.n_out > SQNN_MAX_N_OUT || d.n_in < 1 || d.n_in > SQNN_MAX_N_IN ||
+        d.n_q < 1 || d.n_q > SQNN_MAX_PLANES || d.block_slices != SQNN_BLOCK_SLICES || d.w_dp != 8)
+        return SQNN_E_BAD_BLOB;
+    if (d.m == 0 || d.n == 0 || d.m > ((uint64_t)1 << 40) / d.n) return SQNN_E_BAD_BLOB;
+    const uint64_t mn = d.m * d.n;
+    const uint64_t l = (mn + d.n_out - 1) / d.n_out;
+    if (d.slices != l || d.slices_padded != round_up(l, SQNN_PAD_SLICES)) return SQNN_E_BAD_BLOB;
+    if (d.total_bytes != blob_bytes) return SQNN_E_BAD_BLOB;
+    const uint64_t lp = d.slices_padded;
+    auto section_ok = [&](uint64_t off, uint64_t payload) {
+        return (off % 16 == 0) && off >= SQNN_BLOB_HEADER_BYTES && payload <= blob_bytes &&
+               off <= blob_bytes - payload && blob_bytes - off - payload >= 16;
+    };
+    if (!section_ok(d.off_xornet, (uint64_t)d.n_out * 4)) return SQNN_E_BAD_BLOB;
+    const uint32_t *rows = (const uint32_t *)(b + d.off_xornet);
+    if (d.n_in < 32)
+        for (uint32_t j = 0; j < d.n_out; ++j)
+            if (rows[j] >> d.n_in) return SQNN_E_BAD_BLOB;
+    uint64_t prev_end = d.off_xornet + (uint64_t)d.n_out * 4;
+    for (uint32_t i = 0; i < d.n_q; ++i) {
+        if (d.w_np[i] > 9 || d.n_dp[i] > 0xffffffffull) return SQNN_E_BAD_BLOB;
+        const uint64_t wc_bytes = lp * d.n_in / 8, np_bytes = lp * d.w_np[i] / 8;
+        const uint64_t idx_bytes = (lp / SQNN_BLOCK_SLICES + 1) * 4;
+        if (!section_ok(d.off_wc[i], wc_bytes) || d.off_wc[i] < prev_end) return SQNN_E_BAD_BLOB;
+        prev_end = d.off_wc[i] + wc_bytes;
+        if (d.w_np[i]) {
+            if (!section_ok(d.off_np[i], np_bytes) || d.off_np[i] < prev_end) return SQNN_E_BAD_BLOB;
+            prev_end = d.off_np[i] + np_bytes;
+        }
+        if (!section_ok(d.off_idx[i], idx_bytes) || d.off_idx[i] < prev_end) return SQNN_E_BAD_BLOB;
+        prev_end = d.off_idx[i] + idx_bytes;
+        if (!section_ok(d.off_dp[i], d.n_dp[i]) || d.off_dp[i] < prev_end) return SQNN_E_BAD_BLOB;
+        prev_end = d.off_dp[i] + d.n_dp[i];
+        const uint32_t *wcs = (const uint32_t *)(b + d.off_wc[i]);
+        const uint32_t *nps = (const uint32_t *)(b + d.off_np[i]);
+        const uint32_t *idx = (const uint32_t *)(b + d.off_idx[i]);
+        const uint8_t *dp = b + d.off_dp[i];
+        uint64_t run = 0;
+        const uint64_t blocks = lp / SQNN_BLOCK_SLICES;
+        for (uint64_t blk = 0; blk < blocks; ++blk) {
+            if (idx[blk] != run) return SQNN_E_BAD_BLOB;
+            for (uint64_t s = blk * SQNN_BLOCK_SLICES; s < (blk + 1) * SQNN_BLOCK_SLICES; ++s) {
+                const uint32_t p = read_field(nps, s, d.w_np[i]);
+                if (s >= l && (p != 0 || read_field(wcs, s, d.n_in) != 0)) return SQNN_E_BAD_BLOB;
+                if (p > d.n_out) return SQNN_E_BAD_BLOB;
+                run += p;
+            }
+            if (run > d.n_dp[i]) return SQNN_E_BAD_BLOB;
+        }
+        if (idx[blocks] != run || run != d.n_dp[i]) return SQNN_E_BAD_BLOB;
+        for (uint64_t k = 0; k < d.n_dp[i]; ++k)
+            if (dp[k] >= d.n_out) return SQNN_E_BAD_BLOB;
+    }
+    *desc = d;
+    return SQNN_OK;
+}
+
+int sqnn_unpack_host(const void *blob, size_t blob_bytes, uint32_t plane,
+                     uint32_t **wc, uint16_t **np, uint16_t **dp, uint64_t *n_dp)
+{
+    if (!wc || !np || !dp || !n_dp) return SQNN_E_INVALID_ARG;
+    sqnn_desc d;
+    int rc = sqnn_describe_host(blob, blob_bytes, &d);
+    if (rc != SQNN_OK) return rc;
+    if (plane >= d.n_q) return SQNN_E_INVALID_ARG;
+    const uint8_t *b = (const uint8_t *)blob;
+    const uint64_t l = d.slices;
+    uint32_t *w = (uint32_t *)std::malloc(sizeof(uint32_t) * (l ? l : 1));
+    uint16_t *p = (uint16_t *)std::malloc(sizeof(uint16_t) * (l ? l : 1));
+    uint16_t *q = (uint16_t *)std::malloc(sizeof(uint16_t) * (d.n_dp[plane] ? d.n_dp[plane] : 1));
+    if (!w || !p || !q) { std::free(w); std::free(p); std::free(q); return SQNN_E_NOMEM; }
+    const uint32_t *wcs = (const uint32_t *)(b + d.off_wc[plane]);
+    const uint32_t *nps = (const uint32_t *)(b + d.off_np[plane]);
+    for (uint64_t s = 0; s < l; ++s) {
+        w[s] = read_field(wcs, s, d.n_in);
+        p[s] = (uint16_t)read_field(nps, s, d.w_np[plane]);
+    }
+    for (uint64_t k = 0; k < d.n_dp[plane]; ++k) q[k] = b[d.off_dp[plane] + k];
+    *wc = w; *np = p; *dp = q; *n_dp = d.n_dp[plane];
+    return SQNN_OK;
+}
+
+int sqnn_stats_host(const void *blob, size_t blob_bytes, sqnn_stats *stats)
+{
+    if (!stats) return SQNN_E_INVALID_ARG;
+    sqnn_desc d;
+    int rc = sqnn_describe_host(blob, blob_bytes, &d);
+    if (rc != SQNN_OK) return rc;
+    std::memset(stats, 0, sizeof *stats);
+    const uint8_t *b = (const uint8_t *)blob;
+    const uint64_t mn = d.m * d.n, l = d.slices, lp = d.slices_padded;
+    stats->slices = l;
+    double eq1_bits = 0.0;
+    for (uint32_t i = 0; i < d.n_q; ++i) {
+        const uint32_t *nps = (const uint32_t *)(b + d.off_np[i]);
+        uint32_t maxp = 0;
+        uint64_t sum = 0;
+        for (uint64_t s = 0; s < l; ++s) {
+            const uint32_t p = read_field(nps, s, d.w_np[i]);
+            maxp = std::max(maxp, p);
+            sum += p;
+        }
+        stats->patches[i] = sum;
+        stats->max_patch[i] = maxp;
+        // Eq. 1, literally: n_in/n_out * mn + l * ceil(lg max p) + sum p * ceil(lg n_out)
+        eq1_bits += (double)d.n_in / (double)d.n_out * (double)mn +
+                    (double)l * ceil_lg_u64(maxp) + (double)sum * ceil_lg_u64(d.n_out);
+        stats->bits_wc += (round_up(lp * d.n_in / 8, 16) + 16) * 8;
+        if (d.w_np[i]) stats->bits_npatch += (round_up(lp * d.w_np[i] / 8, 16) + 16) * 8;
+        stats->bits_index += (round_up((lp / SQNN_BLOCK_SLICES + 1) * 4, 16) + 16) * 8;
+        stats->bits_dpatch += (round_up(sum, 16) + 16) * 8;
+    }
+    stats->bpw_eq1 = eq1_bits / (double)mn;
+    stats->bpw_actual = (double)(stats->bits_wc + stats->bits_npatch + stats->bits_index + stats->bits_dpatch) / (double)mn;
+    return SQNN_OK;
+}
+
+}  // extern "C"

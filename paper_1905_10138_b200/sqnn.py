@@ -1,0 +1,228 @@
+"""Thin ctypes binding over ``libsqnn.so`` -- same names as ``include/sqnn.h``.
+
+Argument marshalling only: every step of the decode / product path runs in the library's
+kernels.  Device buffers are torch CUDA tensors (torch is used for device memory and
+streams, nothing else).  There is no CPU fallback: if the library cannot be loaded every
+call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libsqnn.so")
+
+MAX_PLANES = 8
+OUT_BITS, OUT_BF16, OUT_SINK = 0, 1, 2
+X_F32, X_BF16 = 0, 1
+ENCODE_ALG1, ENCODE_EXHAUSTIVE = 0, 1
+OK, E_INVALID_ARG, E_BAD_BLOB, E_UNSUPPORTED, E_NOMEM, E_CUDA, E_TIMEOUT, E_WORKSPACE = 0, -1, -2, -3, -4, -5, -6, -7
+
+
+class SqnnError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        super().__init__(f"{what}: {status_string(status)} ({status})")
+
+
+class XorNet(ctypes.Structure):
+    _fields_ = [("n_out", ctypes.c_uint32), ("n_in", ctypes.c_uint32), ("rows", ctypes.c_void_p)]
+
+
+class Planes(ctypes.Structure):
+    _fields_ = [("m", ctypes.c_uint64), ("n", ctypes.c_uint64), ("n_q", ctypes.c_uint32),
+                ("planes", ctypes.c_void_p), ("mask", ctypes.c_void_p)]
+
+
+class Stats(ctypes.Structure):
+    _fields_ = [("slices", ctypes.c_uint64), ("patches", ctypes.c_uint64 * MAX_PLANES),
+                ("max_patch", ctypes.c_uint32 * MAX_PLANES),
+                ("bits_wc", ctypes.c_uint64), ("bits_npatch", ctypes.c_uint64),
+                ("bits_dpatch", ctypes.c_uint64), ("bits_index", ctypes.c_uint64),
+                ("bpw_eq1", ctypes.c_double), ("bpw_actual", ctypes.c_double)]
+
+    def as_dict(self, n_q: int) -> dict:
+        return {"slices": int(self.slices), "patches": [int(v) for v in self.patches[:n_q]],
+                "max_patch": [int(v) for v in self.max_patch[:n_q]],
+                "bits_wc": int(self.bits_wc), "bits_npatch": int(self.bits_npatch),
+                "bits_dpatch": int(self.bits_dpatch), "bits_index": int(self.bits_index),
+                "bpw_eq1": float(self.bpw_eq1), "bpw_actual": float(self.bpw_actual)}
+
+
+class Desc(ctypes.Structure):
+    _fields_ = [("m", ctypes.c_uint64), ("n", ctypes.c_uint64), ("slices", ctypes.c_uint64),
+                ("slices_padded", ctypes.c_uint64),
+                ("n_q", ctypes.c_uint32), ("n_out", ctypes.c_uint32), ("n_in", ctypes.c_uint32),
+                ("block_slices", ctypes.c_uint32),
+                ("w_np", ctypes.c_uint32 * MAX_PLANES), ("w_dp", ctypes.c_uint32), ("reserved", ctypes.c_uint32),
+                ("off_xornet", ctypes.c_uint64),
+                ("off_wc", ctypes.c_uint64 * MAX_PLANES), ("off_np", ctypes.c_uint64 * MAX_PLANES),
+                ("off_idx", ctypes.c_uint64 * MAX_PLANES), ("off_dp", ctypes.c_uint64 * MAX_PLANES),
+                ("n_dp", ctypes.c_uint64 * MAX_PLANES), ("total_bytes", ctypes.c_uint64)]
+
+
+_lib = None
+
+
+def lib():
+    """The loaded C library.  Raises if it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: build it with "
+                              "`python -m paper_1905_10138_b200.build` (needs nvcc, sm_100a)")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, u32, u64, i64, i32, sz = (ctypes.c_void_p, ctypes.c_uint32, ctypes.c_uint64, ctypes.c_int64,
+                                      ctypes.c_int, ctypes.c_size_t)
+        P = ctypes.POINTER
+        L.sqnn_encode_host.argtypes = [P(XorNet), P(Planes), u32, P(vp), P(sz), P(Stats)]
+        L.sqnn_pack_host.argtypes = [P(XorNet), u64, u64, u32, P(vp), P(vp), P(vp), P(vp), P(sz)]
+        L.sqnn_unpack_host.argtypes = [vp, sz, u32, P(vp), P(vp), P(vp), P(u64)]
+        L.sqnn_describe_host.argtypes = [vp, sz, P(Desc)]
+        L.sqnn_stats_host.argtypes = [vp, sz, P(Stats)]
+        L.sqnn_free.argtypes = [vp]
+        L.sqnn_free.restype = None
+        L.sqnn_decode.argtypes = [P(Desc), vp, vp, vp, i32, vp, sz, vp, vp]
+        L.sqnn_decode_matmul.argtypes = [P(Desc), vp, vp, vp, vp, i32, u32, i64, vp, i64, vp, sz, vp, vp]
+        L.sqnn_workspace_bytes.argtypes = [P(Desc), u32]
+        L.sqnn_workspace_bytes.restype = sz
+        L.sqnn_status_string.argtypes = [i32]
+        L.sqnn_status_string.restype = ctypes.c_char_p
+        for name in ("sqnn_encode_host", "sqnn_pack_host", "sqnn_unpack_host", "sqnn_describe_host",
+                     "sqnn_stats_host", "sqnn_decode", "sqnn_decode_matmul"):
+            getattr(L, name).restype = i32
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().sqnn_status_string(int(status)).decode()
+
+
+def _check(status: int, what: str):
+    if status != OK:
+        raise SqnnError(status, what)
+
+
+def _np_ptr(a: np.ndarray):
+    return ctypes.c_void_p(a.ctypes.data)
+
+
+def _take(ptr: ctypes.c_void_p, nbytes: int) -> np.ndarray:
+    """Copies a library-owned host buffer into a numpy array and frees it."""
+    out = np.empty(nbytes, dtype=np.uint8)
+    if nbytes:
+        ctypes.memmove(out.ctypes.data, ptr.value, nbytes)
+    lib().sqnn_free(ptr)
+    return out
+
+
+def _net(rows: np.ndarray, n_in: int):
+    rows = np.ascontiguousarray(rows, dtype=np.uint32)
+    return XorNet(int(rows.size), int(n_in), rows.ctypes.data), rows
+
+
+def sqnn_encode_host(rows, n_in, m, n, n_q, planes_words, mask_words, flags=ENCODE_ALG1):
+    """rows uint32 [n_out]; planes_words uint64 [n_q * ceil(mn/64)]; mask_words uint64 [ceil(mn/64)].
+    Returns (blob uint8 array, stats dict)."""
+    net, _keep = _net(rows, n_in)
+    planes_words = np.ascontiguousarray(planes_words, dtype=np.uint64)
+    mask_words = np.ascontiguousarray(mask_words, dtype=np.uint64)
+    words = (m * n + 63) // 64
+    if planes_words.size != n_q * words or mask_words.size != words:
+        raise ValueError("packed plane / mask size mismatch")
+    layer = Planes(m, n, n_q, planes_words.ctypes.data, mask_words.ctypes.data)
+    blob, nbytes, st = ctypes.c_void_p(), ctypes.c_size_t(), Stats()
+    _check(lib().sqnn_encode_host(ctypes.byref(net), ctypes.byref(layer), flags, ctypes.byref(blob),
+                                  ctypes.byref(nbytes), ctypes.byref(st)), "sqnn_encode_host")
+    return _take(blob, nbytes.value), st.as_dict(n_q)
+
+
+def sqnn_pack_host(rows, n_in, m, n, wc, np_, dp):
+    """wc / np_ / dp: lists (one entry per plane) of uint32 [l], uint16 [l], uint16 [sum np]."""
+    net, _keep = _net(rows, n_in)
+    n_q = len(wc)
+    wc = [np.ascontiguousarray(a, dtype=np.uint32) for a in wc]
+    np_ = [np.ascontiguousarray(a, dtype=np.uint16) for a in np_]
+    dp = [np.ascontiguousarray(np.concatenate([a, [0]]) if a.size == 0 else a, dtype=np.uint16) for a in dp]
+    arr = ctypes.c_void_p * n_q
+    blob, nbytes = ctypes.c_void_p(), ctypes.c_size_t()
+    _check(lib().sqnn_pack_host(ctypes.byref(net), m, n, n_q,
+                                arr(*[a.ctypes.data for a in wc]), arr(*[a.ctypes.data for a in np_]),
+                                arr(*[a.ctypes.data for a in dp]), ctypes.byref(blob), ctypes.byref(nbytes)),
+           "sqnn_pack_host")
+    return _take(blob, nbytes.value)
+
+
+def sqnn_describe_host(blob: np.ndarray) -> Desc:
+    blob = np.ascontiguousarray(blob, dtype=np.uint8)
+    d = Desc()
+    _check(lib().sqnn_describe_host(_np_ptr(blob), blob.size, ctypes.byref(d)), "sqnn_describe_host")
+    return d
+
+
+def sqnn_stats_host(blob: np.ndarray) -> dict:
+    blob = np.ascontiguousarray(blob, dtype=np.uint8)
+    st = Stats()
+    _check(lib().sqnn_stats_host(_np_ptr(blob), blob.size, ctypes.byref(st)), "sqnn_stats_host")
+    d = sqnn_describe_host(blob)
+    return st.as_dict(d.n_q)
+
+
+def sqnn_unpack_host(blob: np.ndarray, plane: int):
+    """Returns (wc uint32 [l], np uint16 [l], dp uint16 [n_dp]) of one plane."""
+    blob = np.ascontiguousarray(blob, dtype=np.uint8)
+    d = sqnn_describe_host(blob)
+    wc, np_, dp, n_dp = ctypes.c_void_p(), ctypes.c_void_p(), ctypes.c_void_p(), ctypes.c_uint64()
+    _check(lib().sqnn_unpack_host(_np_ptr(blob), blob.size, plane, ctypes.byref(wc), ctypes.byref(np_),
+                                  ctypes.byref(dp), ctypes.byref(n_dp)), "sqnn_unpack_host")
+    l = int(d.slices)
+    return (_take(wc, 4 * l).view(np.uint32), _take(np_, 2 * l).view(np.uint16),
+            _take(dp, 2 * int(n_dp.value)).view(np.uint16))
+
+
+def _dev_ptr(t):
+    return ctypes.c_void_p(t.data_ptr()) if t is not None else None
+
+
+def _stream_ptr(stream):
+    import torch
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def sqnn_decode(desc: Desc, d_blob, d_mask, d_alpha, mode: int, d_out, d_status=None, stream=None):
+    """Queues the decode kernel on ``stream`` (default: torch's current stream).  Tensors are CUDA."""
+    _check(lib().sqnn_decode(ctypes.byref(desc), _dev_ptr(d_blob), _dev_ptr(d_mask), _dev_ptr(d_alpha),
+                             int(mode), _dev_ptr(d_out), d_out.numel() * d_out.element_size(),
+                             _dev_ptr(d_status), _stream_ptr(stream)), "sqnn_decode")
+
+
+def sqnn_workspace_bytes(desc: Desc, batch: int) -> int:
+    return int(lib().sqnn_workspace_bytes(ctypes.byref(desc), int(batch)))
+
+
+def sqnn_decode_matmul(desc: Desc, d_blob, d_mask, d_alpha, d_x, d_y, d_workspace=None, d_status=None,
+                       stream=None):
+    """Y[b, r] = sum_c W[r, c] X[b, c].  d_x: [batch, n] float32 or bfloat16 (row stride free);
+    d_y: [batch, m] float32.  Queues on ``stream``; does not synchronise."""
+    import torch
+    if d_x.dim() != 2 or d_y.dim() != 2 or d_x.stride(1) != 1 or d_y.stride(1) != 1:
+        raise ValueError("X and Y must be 2-D with unit inner stride")
+    if d_x.dtype == torch.float32:
+        xdt = X_F32
+    elif d_x.dtype == torch.bfloat16:
+        xdt = X_BF16
+    else:
+        raise ValueError("X must be float32 or bfloat16")
+    if d_y.dtype != torch.float32:
+        raise ValueError("Y must be float32")
+    batch = d_x.shape[0]
+    ws_bytes = d_workspace.numel() * d_workspace.element_size() if d_workspace is not None else 0
+    _check(lib().sqnn_decode_matmul(ctypes.byref(desc), _dev_ptr(d_blob), _dev_ptr(d_mask), _dev_ptr(d_alpha),
+                                    _dev_ptr(d_x), xdt, batch, d_x.stride(0), _dev_ptr(d_y), d_y.stride(0),
+                                    _dev_ptr(d_workspace), ws_bytes, _dev_ptr(d_status), _stream_ptr(stream)),
+           "sqnn_decode_matmul")

@@ -1,0 +1,110 @@
+"""GPU parity: the CUDA decode kernels against the CPU oracle, bit for bit, through the C ABI."""
+import numpy as np
+import pytest
+
+from oracle import oracle as orc
+from paper_1905_10138_b200 import sqnn
+from paper_1905_10138_b200 import workloads as wl
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+SMALL = [
+    ("cfg1", lambda: wl.make_layer(1)),                                   # 820 slices, ragged last slice
+    ("cfg2-s", lambda: wl.make_layer(2, m=37, n=9216)),                   # 13.3 warp tiles, rows straddle slices
+    ("cfg3-s", lambda: wl.make_layer(3, m=203, n=3000)),                  # 2 planes
+    ("cfg4-s", lambda: wl.make_layer(4, m=41, n=16384)),                  # 3 planes
+    ("sw-40x16-S60", lambda: wl.make_sweep_layer(0, 0, m=61, n=4099)),
+    ("sw-80x16-S60", lambda: wl.make_sweep_layer(0, 1, m=61, n=4099)),
+    ("sw-100x10-S60", lambda: wl.make_sweep_layer(0, 2, m=61, n=4099)),   # ~15 patches per slice
+    ("sw-200x10-S60", lambda: wl.make_sweep_layer(0, 3, m=61, n=4099)),   # ~35 patches per slice
+    ("sw-100x10-S90", lambda: wl.make_sweep_layer(2, 2, m=129, n=4001)),
+    ("sw-200x10-S95", lambda: wl.make_sweep_layer(3, 3, m=129, n=4001)),
+    ("sw-40x16-S95", lambda: wl.make_sweep_layer(3, 0, m=129, n=4001)),   # no patches at all
+]
+
+
+def generic_layer(n_out, n_in, m, n, keep, seed, n_q=1):
+    """A layer with an arbitrary network shape (exercises the run-time-shape kernels)."""
+    rng = np.random.default_rng(seed)
+    planes = rng.integers(0, 2, (n_q, m, n), dtype=np.uint8)
+    mask = (rng.random((m, n)) < keep).astype(np.uint8)
+    alpha = (rng.random((m, n_q)) + 0.5).astype(np.float32)
+    return wl.Layer(name=f"gen-{n_out}x{n_in}", cfg=0, m=m, n=n, n_q=n_q, n_out=n_out, n_in=n_in,
+                    prune_rate=1 - keep, M=wl.xor_network(n_out, n_in, seed + 1), planes=planes, mask=mask,
+                    alpha=alpha, x_dtype="f32", batches=(1,), seed_x=seed + 2)
+
+
+GENERIC = [
+    ("gen-13x5", lambda: generic_layer(13, 5, 57, 1001, 0.3, 11)),
+    ("gen-256x32", lambda: generic_layer(256, 32, 64, 3000, 0.15, 12)),
+    ("gen-33x20", lambda: generic_layer(33, 20, 31, 2049, 0.5, 13, n_q=2)),
+    ("gen-64x7", lambda: generic_layer(64, 7, 16, 4096, 0.2, 14)),
+    ("gen-1x1", lambda: generic_layer(1, 1, 5, 77, 0.5, 15)),
+    ("gen-96x9-q8", lambda: generic_layer(96, 9, 20, 999, 0.1, 16, n_q=8)),
+    ("gen-tiny", lambda: generic_layer(100, 10, 1, 3, 1.0, 17)),
+]
+
+
+@pytest.mark.parametrize("name,make", SMALL + GENERIC, ids=[n for n, _ in SMALL + GENERIC])
+def test_decode_bits_sink_and_bf16_match_oracle_exactly(name, make):
+    layer = make()
+    arrays = H.oracle_encode(layer)
+    ref_bits = H.oracle_decode(layer, arrays)
+    dev = H.DeviceLayer(layer, H.blob_from_oracle(layer, arrays))
+    # packed bits: every position, don't-cares included; bits past mn in the last word are zero
+    got = dev.decode_bits()
+    for i in range(layer.n_q):
+        assert np.array_equal(got[i], wl.pack_bits(ref_bits[i])), (name, i)
+    # checksum sink
+    expect_sink = 0
+    for i in range(layer.n_q):
+        expect_sink ^= int(np.bitwise_xor.reduce(wl.pack_bits(ref_bits[i])))
+    assert dev.decode_sink() == expect_sink
+    # masked, rescaled bf16 weights
+    _, ref_bf16 = orc.reconstruct(ref_bits, layer.mask, layer.alpha, want_f32=False)
+    assert np.array_equal(dev.decode_bf16(), ref_bf16)
+    assert dev.status_value() == 0
+
+
+def test_library_encoded_blob_decodes_to_the_same_bits():
+    layer = wl.make_layer(3, m=203, n=3000)
+    blob, _ = H.blob_from_library(layer)
+    dev = H.DeviceLayer(layer, blob)
+    got = dev.decode_bits()
+    ref = H.oracle_decode(layer, H.oracle_encode(layer))
+    for i in range(layer.n_q):
+        assert np.array_equal(got[i], wl.pack_bits(ref[i]))
+
+
+def test_malformed_device_patch_entries_set_the_status_word_and_do_not_fault():
+    """The host validator rejects such blobs; if a device copy is damaged anyway the kernel
+    skips the entry and reports through the status word."""
+    import torch
+    layer = wl.make_sweep_layer(1, 2, m=40, n=1000)
+    blob, _ = H.blob_from_library(layer)
+    dev = H.DeviceLayer(layer, blob)
+    d = dev.desc
+    assert d.n_dp[0] > 0
+    clean = dev.decode_bits()
+    assert dev.status_value() == 0
+    dev.blob[int(d.off_dp[0])] = 250                     # position >= n_out = 100
+    torch.cuda.synchronize()
+    damaged = dev.decode_bits()
+    assert dev.status_value() == 1
+    diff = np.bitwise_xor(clean, damaged)
+    assert sum(bin(int(w)).count("1") for w in diff.ravel()) == 1      # exactly the skipped flip
+
+
+def test_output_buffer_size_and_alignment_are_checked():
+    import torch
+    layer = wl.make_layer(1, m=16, n=80)
+    blob, _ = H.blob_from_library(layer)
+    dev = H.DeviceLayer(layer, blob)
+    small = torch.zeros(1, dtype=torch.int64, device="cuda")
+    with pytest.raises(sqnn.SqnnError) as e:
+        sqnn.sqnn_decode(dev.desc, dev.blob, None, None, sqnn.OUT_BITS, small)
+    assert e.value.status == sqnn.E_INVALID_ARG
+    with pytest.raises(sqnn.SqnnError):
+        sqnn.sqnn_decode(dev.desc, dev.blob, None, None, sqnn.OUT_BF16,
+                         torch.zeros(16 * 80, dtype=torch.bfloat16, device="cuda"))   # mask / alpha missing

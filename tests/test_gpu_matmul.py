@@ -1,0 +1,68 @@
+"""GPU parity: fused decode + product against the oracle's fp64 product, through the C ABI."""
+import numpy as np
+import pytest
+
+from oracle import oracle as orc
+from paper_1905_10138_b200 import workloads as wl
+from tests import helpers as H
+from tests.test_gpu_decode import generic_layer
+
+pytestmark = pytest.mark.gpu
+
+# Tolerances (max |y - y_ref| / max(|y_ref|, rms(y_ref))):
+#  1e-4: fp32 accumulation of exact weights (GEMV path, batch <= 15)
+#  1e-2: weights rounded to bf16 (tensor-core path, batch >= 16)
+TOL_F32 = 1e-4
+TOL_BF16 = 1e-2
+
+
+def reference(layer, x):
+    """The product depends on care bits only, and those are reproduced exactly (checked by the
+    decode parity tests), so the oracle's product runs on the oracle-decoded planes."""
+    ref_bits = H.oracle_decode(layer, H.oracle_encode(layer))
+    return orc.matmul(ref_bits, layer.mask, layer.alpha, x.astype(np.float64))
+
+
+GEMV = [
+    ("cfg1-b1-f32", lambda: wl.make_layer(1), "f32", 1),
+    ("cfg2-s-b1", lambda: wl.make_layer(2, m=37, n=9216), "bf16", 1),
+    ("cfg3-s-b1", lambda: wl.make_layer(3, m=203, n=3000), "bf16", 1),
+    ("cfg3-s-b8", lambda: wl.make_layer(3, m=203, n=3000), "bf16", 8),
+    ("cfg4-s-b3", lambda: wl.make_layer(4, m=41, n=16384), "bf16", 3),
+    ("cfg4-s-b15-f32", lambda: wl.make_layer(4, m=41, n=16384), "f32", 15),
+    ("gen-13x5-b2", lambda: generic_layer(13, 5, 57, 1001, 0.3, 11), "f32", 2),
+    ("gen-33x20-q2-b5", lambda: generic_layer(33, 20, 31, 2049, 0.5, 13, n_q=2), "bf16", 5),
+    ("gen-narrow-n", lambda: generic_layer(40, 12, 300, 17, 0.4, 21), "f32", 4),        # rows shorter than a word
+    ("gen-empty-rows", lambda: generic_layer(100, 10, 64, 500, 0.0, 22), "f32", 1),     # everything pruned
+]
+
+
+@pytest.mark.parametrize("name,make,xdt,batch", GEMV, ids=[g[0] for g in GEMV])
+def test_fused_gemv_matches_fp64_oracle(name, make, xdt, batch):
+    import torch
+    layer = make()
+    layer.x_dtype = xdt
+    x = layer.activations(batch)
+    ref = reference(layer, x)
+    dev = H.DeviceLayer(layer, H.blob_from_library(layer)[0])
+    y = dev.matmul(x, torch.float32 if xdt == "f32" else torch.bfloat16)
+    assert y.shape == (batch, layer.m)
+    assert H.rel_err(y, ref) <= TOL_F32, H.rel_err(y, ref)
+    assert dev.status_value() == 0
+
+
+def test_gemv_respects_row_strides():
+    import torch
+    from paper_1905_10138_b200 import sqnn
+    layer = wl.make_layer(3, m=50, n=3000)
+    x = layer.activations(3)
+    ref = reference(layer, x)
+    dev = H.DeviceLayer(layer, H.blob_from_library(layer)[0])
+    xbuf = torch.zeros((3, 3000 + 24), dtype=torch.bfloat16, device="cuda")
+    xbuf[:, :3000] = torch.from_numpy(x).cuda().to(torch.bfloat16)
+    ybuf = torch.full((3, 50 + 7), 7.0, dtype=torch.float32, device="cuda")
+    sqnn.sqnn_decode_matmul(dev.desc, dev.blob, dev.mask, dev.alpha, xbuf[:, :3000], ybuf[:, :50], None, dev.status)
+    torch.cuda.synchronize()
+    y = ybuf.cpu().numpy()
+    assert H.rel_err(y[:, :50], ref) <= TOL_F32
+    assert np.all(y[:, 50:] == 7.0)

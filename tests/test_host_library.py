@@ -1,0 +1,186 @@
+"""CPU tests of the C-ABI library's host side: exported symbols, the encoder against the
+oracle's Algorithm 1 (logical arrays must be identical), blob packing / validation, stats."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+from oracle import oracle as orc
+from paper_1905_10138_b200 import sqnn
+from paper_1905_10138_b200 import workloads as wl
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def oracle_arrays(layer):
+    """Per-plane (wc, np, dp) from the oracle's encoder."""
+    care = layer.mask.ravel()
+    return [orc.encode_plane(layer.M, layer.planes[i].ravel(), care) for i in range(layer.n_q)]
+
+
+def library_blob(layer, flags=sqnn.ENCODE_ALG1):
+    planes_words = np.concatenate([wl.pack_bits(layer.planes[i]) for i in range(layer.n_q)])
+    return sqnn.sqnn_encode_host(wl.network_rows(layer.M), layer.n_in, layer.m, layer.n, layer.n_q,
+                                 planes_words, wl.pack_bits(layer.mask), flags)
+
+
+def test_library_exports_every_declared_symbol():
+    text = open(os.path.join(ROOT, "include", "sqnn.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    names = set(re.findall(r"\b(sqnn_[a-z_]+)\s*\(", text))
+    assert {"sqnn_encode_host", "sqnn_decode", "sqnn_decode_matmul"} <= names
+    L = sqnn.lib()
+    for name in sorted(names):
+        assert hasattr(L, name), name
+
+
+def test_struct_layouts_match_the_header_sizes():
+    # sizes computed by hand from include/sqnn.h (natural alignment)
+    assert ctypes.sizeof(sqnn.Desc) == 4 * 8 + 4 * 4 + 8 * 4 + 8 + 8 + 4 * 8 * 8 + 8 * 8 + 8
+    assert ctypes.sizeof(sqnn.Stats) == 8 + 64 + 32 + 32 + 16
+
+
+LAYERS = [
+    ("cfg1", lambda: wl.make_layer(1)),
+    ("cfg2-small", lambda: wl.make_layer(2, m=96, n=1000)),
+    ("cfg3-small", lambda: wl.make_layer(3, m=120, n=300)),
+    ("cfg4-small", lambda: wl.make_layer(4, m=64, n=1030)),
+    ("sweep-heavy", lambda: wl.make_sweep_layer(0, 3, m=64, n=1000)),     # S=0.6, (200,10): many patches
+    ("sweep-80x16", lambda: wl.make_sweep_layer(1, 1, m=50, n=999)),
+    ("sweep-40x16", lambda: wl.make_sweep_layer(3, 0, m=33, n=777)),
+]
+
+
+@pytest.mark.parametrize("name,make", LAYERS, ids=[n for n, _ in LAYERS])
+def test_encoder_matches_oracle_algorithm1_bit_for_bit(name, make):
+    layer = make()
+    blob, stats = library_blob(layer)
+    ref = oracle_arrays(layer)
+    d = sqnn.sqnn_describe_host(blob)
+    assert (d.m, d.n, d.n_q, d.n_out, d.n_in) == (layer.m, layer.n, layer.n_q, layer.n_out, layer.n_in)
+    assert d.slices == (layer.mn + layer.n_out - 1) // layer.n_out
+    eq1_bits = 0.0
+    for i in range(layer.n_q):
+        wc, np_, dp = sqnn.sqnn_unpack_host(blob, i)
+        assert np.array_equal(wc.astype(np.uint64), ref[i][0])
+        assert np.array_equal(np_, ref[i][1])
+        assert np.array_equal(dp, ref[i][2])
+        assert stats["patches"][i] == int(ref[i][1].sum())
+        assert stats["max_patch"][i] == int(ref[i][1].max())
+        e = orc.eq1(layer.mn, layer.n_out, layer.n_in, ref[i][1])
+        eq1_bits += e["bits_wc"] + e["bits_npatch"] + e["bits_dpatch"]
+    assert abs(stats["bpw_eq1"] - eq1_bits / layer.mn) < 1e-12
+    stored = stats["bits_wc"] + stats["bits_npatch"] + stats["bits_dpatch"] + stats["bits_index"]
+    assert abs(stats["bpw_actual"] - stored / layer.mn) < 1e-12
+    # packing the oracle's arrays gives the very same bytes
+    blob2 = sqnn.sqnn_pack_host(wl.network_rows(layer.M), layer.n_in, layer.m, layer.n,
+                                [r[0].astype(np.uint32) for r in ref], [r[1] for r in ref], [r[2] for r in ref])
+    assert np.array_equal(blob, blob2)
+
+
+def test_exhaustive_encoder_matches_oracle_exhaustive():
+    layer = wl.make_layer(1, m=40, n=100)
+    blob, stats = library_blob(layer, sqnn.ENCODE_EXHAUSTIVE)
+    wc, np_, dp = sqnn.sqnn_unpack_host(blob, 0)
+    rwc, rnp, rdp = orc.encode_plane(layer.M, layer.planes[0].ravel(), layer.mask.ravel(), exhaustive=True)
+    assert np.array_equal(wc.astype(np.uint64), rwc) and np.array_equal(np_, rnp) and np.array_equal(dp, rdp)
+    _, stats_a = library_blob(layer)
+    assert stats["patches"][0] <= stats_a["patches"][0]
+
+
+def test_odd_network_shapes_and_tiny_layers():
+    rng = np.random.default_rng(8)
+    for (n_out, n_in, m, n) in [(13, 5, 7, 31), (1, 1, 3, 5), (256, 32, 9, 300), (33, 20, 40, 41), (64, 7, 1, 64)]:
+        M = wl.xor_network(n_out, n_in, n_out * 100 + n_in)
+        bits = rng.integers(0, 2, (m, n), dtype=np.uint8)
+        mask = (rng.random((m, n)) < 0.3).astype(np.uint8)
+        blob, _ = sqnn.sqnn_encode_host(wl.network_rows(M), n_in, m, n, 1, wl.pack_bits(bits), wl.pack_bits(mask))
+        wc, np_, dp = sqnn.sqnn_unpack_host(blob, 0)
+        rwc, rnp, rdp = orc.encode_plane(M, bits.ravel(), mask.ravel())
+        assert np.array_equal(wc.astype(np.uint64), rwc) and np.array_equal(np_, rnp) and np.array_equal(dp, rdp)
+        out = orc.decode_plane(M, m * n, rwc, rnp, rdp)
+        assert np.array_equal(out[mask.ravel() == 1], bits.ravel()[mask.ravel() == 1])
+
+
+def test_blob_layout_invariants():
+    layer = wl.make_layer(3, m=60, n=300)
+    blob, _ = library_blob(layer)
+    d = sqnn.sqnn_describe_host(blob)
+    assert d.total_bytes == blob.size and d.slices_padded % 1024 == 0 and d.block_slices == 128
+    for i in range(d.n_q):
+        for off in (d.off_wc[i], d.off_np[i], d.off_idx[i], d.off_dp[i]):
+            assert off % 16 == 0
+        idx = blob[d.off_idx[i]: d.off_idx[i] + 4 * (d.slices_padded // 128 + 1)].view(np.uint32)
+        _, np_, _ = sqnn.sqnn_unpack_host(blob, i)
+        padded = np.zeros(d.slices_padded, np.int64)
+        padded[: np_.size] = np_
+        expect = np.concatenate([[0], np.cumsum(padded.reshape(-1, 128).sum(axis=1))])
+        assert np.array_equal(idx.astype(np.int64), expect)
+        assert idx[-1] == d.n_dp[i]
+    rows = blob[d.off_xornet: d.off_xornet + 4 * d.n_out].view(np.uint32)
+    assert np.array_equal(rows, wl.network_rows(layer.M))
+
+
+def test_malformed_blobs_are_rejected_on_the_host():
+    layer = wl.make_sweep_layer(1, 2, m=40, n=1000)           # has patches
+    blob, _ = library_blob(layer)
+    d = sqnn.sqnn_describe_host(blob)
+    assert d.n_dp[0] > 0
+
+    def bad(mutate):
+        b = blob.copy()
+        mutate(b)
+        with pytest.raises(sqnn.SqnnError) as e:
+            sqnn.sqnn_describe_host(b)
+        assert e.value.status == sqnn.E_BAD_BLOB
+
+    bad(lambda b: b.__setitem__(0, b[0] ^ 1))                                  # magic
+    bad(lambda b: b.__setitem__(8, 9))                                         # version
+    bad(lambda b: b.__setitem__(int(d.off_dp[0]), 255))                        # position >= n_out
+    bad(lambda b: b.__setitem__(int(d.off_idx[0]) + 4, b[int(d.off_idx[0]) + 4] ^ 1))   # offsets
+    bad(lambda b: b.__setitem__(int(d.off_np[0]), b[int(d.off_np[0])] ^ 1))    # n_patch sum
+    with pytest.raises(sqnn.SqnnError):
+        sqnn.sqnn_describe_host(blob[:-16])                                    # truncated
+    with pytest.raises(sqnn.SqnnError):
+        sqnn.sqnn_describe_host(blob[:100])
+    hdr = blob.copy()
+    hdr[16:24] = np.frombuffer(np.uint64(1 << 50).tobytes(), dtype=np.uint8)   # absurd m
+    with pytest.raises(sqnn.SqnnError):
+        sqnn.sqnn_describe_host(hdr)
+
+
+def test_invalid_arguments_return_codes_not_crashes():
+    M = wl.xor_network(8, 4, 1)
+    rows = wl.network_rows(M)
+    bits = np.zeros(64, np.uint8)
+    with pytest.raises(sqnn.SqnnError) as e:
+        sqnn.sqnn_encode_host(rows, 40, 8, 8, 1, wl.pack_bits(bits), wl.pack_bits(bits))     # n_in > 32
+    assert e.value.status == sqnn.E_INVALID_ARG
+    with pytest.raises(sqnn.SqnnError):
+        sqnn.sqnn_encode_host(rows, 4, 8, 8, 9, np.zeros(9, np.uint64), wl.pack_bits(bits))  # n_q > 8
+    with pytest.raises(sqnn.SqnnError):      # seed does not fit n_in bits
+        sqnn.sqnn_pack_host(rows, 4, 1, 8, [np.array([16], np.uint32)], [np.array([0], np.uint16)],
+                            [np.zeros(0, np.uint16)])
+    with pytest.raises(sqnn.SqnnError):      # patch position >= n_out
+        sqnn.sqnn_pack_host(rows, 4, 1, 8, [np.array([3], np.uint32)], [np.array([1], np.uint16)],
+                            [np.array([8], np.uint16)])
+    assert sqnn.status_string(0) == "ok" and "unknown" in sqnn.status_string(-99)
+
+
+def test_device_entry_points_reject_bad_arguments_without_a_gpu():
+    layer = wl.make_layer(1, m=16, n=80)
+    blob, _ = library_blob(layer)
+    d = sqnn.sqnn_describe_host(blob)
+    L = sqnn.lib()
+    # NULL blob / NULL output are refused before any CUDA call
+    assert L.sqnn_decode(ctypes.byref(d), None, None, None, 0, None, 0, None, None) == sqnn.E_INVALID_ARG
+    assert L.sqnn_decode(ctypes.byref(d), ctypes.c_void_p(16), None, None, 0, None, 0, None, None) == sqnn.E_INVALID_ARG
+    assert L.sqnn_decode(ctypes.byref(d), ctypes.c_void_p(24), None, None, 0, ctypes.c_void_p(16), 1 << 20,
+                         None, None) == sqnn.E_INVALID_ARG                      # misaligned blob
+    assert L.sqnn_decode(ctypes.byref(d), ctypes.c_void_p(32), None, None, 0, ctypes.c_void_p(16), 8,
+                         None, None) == sqnn.E_INVALID_ARG                      # out too small
+    assert L.sqnn_decode_matmul(ctypes.byref(d), ctypes.c_void_p(32), None, None, None, 0, 1, 80, None, 16,
+                                None, 0, None, None) == sqnn.E_INVALID_ARG
+    assert sqnn.sqnn_workspace_bytes(d, 1) == 0
