@@ -78,10 +78,10 @@ SQNN_DEV void flag(uint32_t *status, uint32_t code)
     if (status) atomicMax(status, code);
 }
 
-// Shared-memory words the tables need.
+// Shared-memory words the tables need, rounded so that what follows stays 16-byte aligned.
 inline __host__ __device__ uint32_t table_words(uint32_t n_in, uint32_t nwp, uint32_t nchunks, uint32_t cb)
 {
-    return nchunks * (1u << cb) * nwp + n_in * nwp;
+    return (nchunks * (1u << cb) * nwp + n_in * nwp + 3u) & ~3u;
 }
 
 // Builds the column words of M and the chunk tables.  All threads of the block take part.
