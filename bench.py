@@ -319,7 +319,7 @@ def oracle_step(layer, rows, sub_mask, arrays, x64):
     return orc.matmul(bits, sub_mask, layer.alpha[:rows], x64)
 
 
-def cpu_baseline(layer, rows=1024):
+def cpu_baseline(layer, rows=4096):
     """The oracle as it stands (decode of every slice, then the fp64 product) on the host cores."""
     from oracle import oracle as orc
     rows = min(rows, layer.m)
@@ -327,7 +327,7 @@ def cpu_baseline(layer, rows=1024):
     x64 = layer.activations(1).astype(np.float64)
     oracle_step(layer, rows, sub_mask, arrays, x64)
     t0 = time.perf_counter()
-    reps = 3
+    reps = 10
     for _ in range(reps):
         oracle_step(layer, rows, sub_mask, arrays, x64)
     dt = (time.perf_counter() - t0) / reps
@@ -343,7 +343,7 @@ def run_reference(args):
     from oracle import oracle as orc
     from paper_1905_10138_b200 import workloads as wl
     layer = wl.make_layer(2)
-    rows = 1024
+    rows = 2048
     _, sub_mask, arrays = oracle_sample(layer, rows)
     x64 = layer.activations(1).astype(np.float64)
     for _ in range(args.warmup):

@@ -9,8 +9,11 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libsqnn.so")
-SOURCES = ["sqnn_host.cpp", "sqnn_kernels.cu", "sqnn_mma.cu"]
-HEADERS = ["sqnn_blob.h", "sqnn_decode.cuh", "sqnn_launch.h"]
+SOURCES = ["sqnn_host.cpp", "sqnn_api.cu", "sqnn_mma.cu"]
+SHAPE_SOURCE = "sqnn_shape.cu"
+# (n_out, n_in) with compile-time kernels -- the list in csrc/sqnn_shapes.h -- plus the run-time shape (0, 0)
+SHAPES = [(40, 12), (40, 16), (60, 12), (80, 8), (80, 16), (100, 10), (200, 10), (0, 0)]
+HEADERS = ["sqnn_blob.h", "sqnn_decode.cuh", "sqnn_launch.h", "sqnn_kernels.cuh", "sqnn_shapes.h", SHAPE_SOURCE]
 
 
 def _nvcc() -> str:
@@ -37,14 +40,24 @@ def build(force: bool = False, verbose: bool = False) -> str:
               "-I", INCLUDE, "-I", CSRC, "-Xcompiler", "-fPIC,-fopenmp,-O3"]
     if verbose:
         common += ["-Xptxas", "-v"]
-    procs, objs = [], []
+    jobs = []
     for s in SOURCES:
-        o = os.path.join(objdir, os.path.splitext(s)[0] + ".o")
-        objs.append(o)
-        procs.append(subprocess.Popen([_nvcc(), *common, "-c", os.path.join(CSRC, s), "-o", o]))
-    for p in procs:
-        if p.wait() != 0:
+        jobs.append(([os.path.join(CSRC, s)], os.path.join(objdir, os.path.splitext(s)[0] + ".o")))
+    for no, ni in SHAPES:
+        jobs.append(([f"-DSQNN_NO={no}", f"-DSQNN_NI={ni}", os.path.join(CSRC, SHAPE_SOURCE)],
+                     os.path.join(objdir, f"sqnn_shape_{no}x{ni}.o")))
+    objs = [o for _, o in jobs]
+    width = max(1, min(len(jobs), os.cpu_count() or 4))
+    pending, running = list(jobs), []
+    while pending or running:
+        while pending and len(running) < width:
+            extra, o = pending.pop(0)
+            running.append(subprocess.Popen([_nvcc(), *common, "-c", *extra, "-o", o]))
+        if running[0].wait() != 0:
+            for r in running[1:]:
+                r.wait()
             raise RuntimeError("nvcc failed")
+        running.pop(0)
     subprocess.run([_nvcc(), "-shared", "-o", LIB, *objs, "-Xcompiler", "-fopenmp", "-lgomp"], check=True)
     return LIB
 

@@ -1,0 +1,148 @@
+// C entry points of the device side: argument checks and dispatch on the network shape.
+#include "sqnn.h"
+#include "sqnn_decode.cuh"
+#include "sqnn_launch.h"
+#include "sqnn_shapes.h"
+
+#include <cuda_runtime.h>
+
+namespace sqnn {
+
+template <int N_OUT, int N_IN>
+int decode_shape(const DecodeArgs &A, sqnn_out_mode mode, const uint64_t *d_mask, const float *d_alpha,
+                 uint64_t n, void *d_out, cudaStream_t st);
+template <int N_OUT, int N_IN>
+int gemv_shape(const DecodeArgs &A, const uint64_t *d_mask, const float *d_alpha, const void *d_x, int x_dtype,
+               int64_t ldx, uint32_t batch, float *d_y, int64_t ldy, uint64_t n, cudaStream_t st);
+#define SQNN_DECLARE(NO, NI)                                                                                  \
+    template <> int decode_shape<NO, NI>(const DecodeArgs &, sqnn_out_mode, const uint64_t *, const float *,  \
+                                         uint64_t, void *, cudaStream_t);                                     \
+    template <> int gemv_shape<NO, NI>(const DecodeArgs &, const uint64_t *, const float *, const void *, int, \
+                                       int64_t, uint32_t, float *, int64_t, uint64_t, cudaStream_t);
+SQNN_FOR_SHAPES(SQNN_DECLARE)
+SQNN_DECLARE(0, 0)
+#undef SQNN_DECLARE
+
+int fill_decode_args(const sqnn_desc *d, const void *d_blob, uint32_t *d_status, DecodeArgs *A)
+{
+    if (!d || !d_blob) return SQNN_E_INVALID_ARG;
+    if (((uintptr_t)d_blob & 15) != 0) return SQNN_E_INVALID_ARG;
+    if (d->n_out < 1 || d->n_out > SQNN_MAX_N_OUT || d->n_in < 1 || d->n_in > SQNN_MAX_N_IN ||
+        d->n_q < 1 || d->n_q > SQNN_MAX_PLANES || d->m == 0 || d->n == 0 ||
+        d->block_slices != SQNN_BLOCK_SLICES || d->slices_padded % SQNN_PAD_SLICES != 0)
+        return SQNN_E_INVALID_ARG;
+    const uint8_t *b = (const uint8_t *)d_blob;
+    A->mn = d->m * d->n;
+    A->words64 = (A->mn + 63) / 64;
+    A->n_out = d->n_out; A->n_in = d->n_in; A->n_q = d->n_q;
+    A->G = slices_per_lane(d->n_out);
+    A->W = A->G * d->n_out / 32;
+    A->tiles = d->slices_padded / (32ull * A->G);
+    A->nw = entry_words(d->n_out);
+    A->nwp = entry_words_padded(d->n_out);
+    A->nchunks = table_chunks(d->n_in, A->nwp);
+    A->cb = chunk_bits(d->n_in, A->nwp);
+    A->rows = (const uint32_t *)(b + d->off_xornet);
+    A->status = d_status;
+    for (uint32_t i = 0; i < d->n_q; ++i) {
+        if (d->off_wc[i] % 16 || d->off_np[i] % 16 || d->off_idx[i] % 16 || d->off_dp[i] % 16 ||
+            d->n_dp[i] > 0xffffffffull || d->w_np[i] > 9)
+            return SQNN_E_INVALID_ARG;
+        A->pl[i].wc = (const uint32_t *)(b + d->off_wc[i]);
+        A->pl[i].np = (const uint32_t *)(b + d->off_np[i]);
+        A->pl[i].idx = (const uint32_t *)(b + d->off_idx[i]);
+        A->pl[i].dp = b + d->off_dp[i];
+        A->pl[i].n_dp = (uint32_t)d->n_dp[i];
+        A->pl[i].w_np = d->w_np[i];
+    }
+    for (uint32_t i = d->n_q; i < 8; ++i) A->pl[i] = A->pl[0];
+    return SQNN_OK;
+}
+
+int sm_count()
+{
+    static int cached[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    if (cached[dev] == 0) {
+        int v = 0;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) v = 148;
+        cached[dev] = v;
+    }
+    return cached[dev];
+}
+
+
+static int gemv_dispatch(const DecodeArgs &A, const uint64_t *d_mask, const float *d_alpha, const void *d_x,
+                         int x_dtype, int64_t ldx, uint32_t batch, float *d_y, int64_t ldy, uint64_t m, uint64_t n,
+                         cudaStream_t st)
+{
+    // Y is accumulated with atomics: clear it first.
+    cudaError_t e = (ldy == (int64_t)m)
+        ? cudaMemsetAsync(d_y, 0, (size_t)batch * m * sizeof(float), st)
+        : cudaMemset2DAsync(d_y, (size_t)ldy * sizeof(float), 0, (size_t)m * sizeof(float), batch, st);
+    if (e != cudaSuccess) return SQNN_E_CUDA;
+#define SQNN_GEMV_CASE(NO, NI) \
+    if (A.n_out == NO && A.n_in == NI) return gemv_shape<NO, NI>(A, d_mask, d_alpha, d_x, x_dtype, ldx, batch, d_y, ldy, n, st);
+    SQNN_FOR_SHAPES(SQNN_GEMV_CASE)
+#undef SQNN_GEMV_CASE
+    return gemv_shape<0, 0>(A, d_mask, d_alpha, d_x, x_dtype, ldx, batch, d_y, ldy, n, st);
+}
+
+}  // namespace sqnn
+
+using namespace sqnn;
+
+
+extern "C" int sqnn_decode(const sqnn_desc *desc, const void *d_blob, const uint64_t *d_mask,
+                           const float *d_alpha, sqnn_out_mode mode, void *d_out, size_t out_bytes,
+                           uint32_t *d_status, void *cuda_stream)
+{
+    DecodeArgs A;
+    int rc = fill_decode_args(desc, d_blob, d_status, &A);
+    if (rc != SQNN_OK) return rc;
+    if (!d_out || ((uintptr_t)d_out & 15) != 0) return SQNN_E_INVALID_ARG;
+    size_t need = 0;
+    switch (mode) {
+        case SQNN_OUT_BITS: need = (size_t)A.n_q * A.words64 * 8; break;
+        case SQNN_OUT_BF16: need = (size_t)A.mn * 2; break;
+        case SQNN_OUT_SINK: need = 8; break;
+        default: return SQNN_E_INVALID_ARG;
+    }
+    if (out_bytes < need) return SQNN_E_INVALID_ARG;
+    if (mode == SQNN_OUT_BF16 && (!d_mask || !d_alpha)) return SQNN_E_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+#define SQNN_DECODE_CASE(NO, NI) \
+    if (A.n_out == NO && A.n_in == NI) return decode_shape<NO, NI>(A, mode, d_mask, d_alpha, desc->n, d_out, st);
+    SQNN_FOR_SHAPES(SQNN_DECODE_CASE)
+#undef SQNN_DECODE_CASE
+    return decode_shape<0, 0>(A, mode, d_mask, d_alpha, desc->n, d_out, st);
+}
+
+extern "C" size_t sqnn_workspace_bytes(const sqnn_desc *desc, uint32_t batch)
+{
+    if (!desc || batch < 16) return 0;
+    return mma_workspace_bytes(desc, batch);
+}
+
+extern "C" int sqnn_decode_matmul(const sqnn_desc *desc, const void *d_blob, const uint64_t *d_mask,
+                                  const float *d_alpha, const void *d_x, int x_dtype, uint32_t batch,
+                                  int64_t ldx, float *d_y, int64_t ldy, void *d_workspace,
+                                  size_t workspace_bytes, uint32_t *d_status, void *cuda_stream)
+{
+    DecodeArgs A;
+    int rc = fill_decode_args(desc, d_blob, d_status, &A);
+    if (rc != SQNN_OK) return rc;
+    if (!d_mask || !d_alpha || !d_x || !d_y || batch == 0) return SQNN_E_INVALID_ARG;
+    if (x_dtype != SQNN_X_F32 && x_dtype != SQNN_X_BF16) return SQNN_E_INVALID_ARG;
+    if (ldx < (int64_t)desc->n || ldy < (int64_t)desc->m) return SQNN_E_INVALID_ARG;
+    if (((uintptr_t)d_mask & 7) || ((uintptr_t)d_alpha & 3) || ((uintptr_t)d_y & 3)) return SQNN_E_INVALID_ARG;
+    if (batch > SQNN_MAX_BATCH || desc->n > (1ull << 30)) return SQNN_E_UNSUPPORTED;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (batch <= 15)
+        return gemv_dispatch(A, d_mask, d_alpha, d_x, x_dtype, ldx, batch, d_y, ldy, desc->m, desc->n, st);
+    if (x_dtype != SQNN_X_BF16) return SQNN_E_UNSUPPORTED;
+    const size_t need = mma_workspace_bytes(desc, batch);
+    if (need && (!d_workspace || workspace_bytes < need || ((uintptr_t)d_workspace & 255))) return SQNN_E_WORKSPACE;
+    return mma_dispatch(desc, A, d_mask, d_alpha, d_x, ldx, batch, d_y, ldy, d_workspace, st);
+}

@@ -1,11 +1,12 @@
 // Device-side decryption of one warp tile: seeds -> XOR-gate network (table lookup) ->
 // patch flips, producing a run of consecutive output words in shared memory.
 //
-// Work split.  A lane owns G consecutive slices, G chosen so that G * n_out is a multiple of
-// 32 bits and 32 * G is a multiple of 128 slices; its W = G * n_out / 32 output words are
-// private to it while it expands and patches.  A warp tile is therefore 32 * G consecutive
-// slices = 32 * W consecutive 32-bit words of the flattened plane, starting on a boundary of
-// the per-128-slice d_patch offsets.
+// Work split.  A lane owns G consecutive slices, G a multiple of 4 chosen so that G * n_out is
+// a multiple of 32 bits; its W = G * n_out / 32 output words are private to it while it expands
+// and patches.  A warp tile is therefore 32 * G consecutive slices = 32 * W consecutive 32-bit
+// words of the flattened plane, and it starts on a boundary of the per-128-slice d_patch
+// offsets.  In the packed streams a tile is G * n_in words of seeds and G * w_np words of
+// n_patch counts.
 //
 // The network (Section 3.1, w~ = M . w^c) is evaluated with tables: the seed is cut into
 // chunks of cb bits and table[chunk][value] holds the XOR of the columns of M selected by
@@ -41,9 +42,14 @@ struct DecodeArgs {
 };
 
 __host__ __device__ constexpr uint32_t gcd_u32(uint32_t a, uint32_t b) { return b == 0 ? a : gcd_u32(b, a % b); }
+// Smallest multiple of 4 slices whose bits fill whole words, doubled (up to 8) while the lane
+// would own fewer than 16 words, so that small networks still get tiles worth their overhead.
 __host__ __device__ constexpr uint32_t slices_per_lane(uint32_t n_out)
 {
-    return (32 / gcd_u32(n_out, 32)) < 4 ? 4 : (32 / gcd_u32(n_out, 32));
+    uint32_t g = 32 / gcd_u32(n_out, 32);
+    if (g < 4) g = 4;
+    while (g < 8 && g * n_out / 32 < 16) g *= 2;
+    return g;
 }
 __host__ __device__ constexpr uint32_t entry_words(uint32_t n_out) { return (n_out + 31) / 32; }
 __host__ __device__ constexpr uint32_t entry_words_padded(uint32_t n_out)
@@ -85,28 +91,45 @@ inline __host__ __device__ uint32_t table_words(uint32_t n_in, uint32_t nwp, uin
 }
 
 // Builds the column words of M and the chunk tables.  All threads of the block take part.
+// An entry's value splits as (high << lo_bits) | low: entries with only low or only high bits
+// are XORed together from the columns directly, every other entry is the XOR of those two.
 SQNN_DEV void build_tables(const DecodeArgs &A, uint32_t *tab)
 {
     const uint32_t nwp = A.nwp, n_in = A.n_in, n_out = A.n_out, cb = A.cb;
+    const uint32_t kshift = nwp == 1 ? 0 : nwp == 2 ? 1 : nwp == 4 ? 2 : 3;
     uint32_t *cols = tab + A.nchunks * (1u << cb) * nwp;
     for (uint32_t i = threadIdx.x; i < n_in * nwp; i += blockDim.x) {
-        const uint32_t t = i / nwp, k = i % nwp;
+        const uint32_t t = i >> kshift, k = i & (nwp - 1);
         uint32_t w = 0;
         for (uint32_t j = 32 * k; j < n_out && j < 32 * k + 32; ++j)
             w |= ((__ldg(A.rows + j) >> t) & 1u) << (j - 32 * k);
         cols[i] = w;
     }
     __syncthreads();
-    const uint32_t total = A.nchunks * (1u << cb) * nwp;
-    for (uint32_t i = threadIdx.x; i < total; i += blockDim.x) {
-        const uint32_t k = i % nwp, e = i / nwp;
-        const uint32_t v = e & ((1u << cb) - 1u), ch = e >> cb;
+    const uint32_t lo_bits = cb / 2, hi_bits = cb - lo_bits;
+    const uint32_t n_lo = 1u << lo_bits, n_hi = 1u << hi_bits;
+    const uint32_t direct = (n_lo + n_hi - 1) * nwp;          // per chunk: low-only and high-only entries
+    for (uint32_t i = threadIdx.x; i < A.nchunks * direct; i += blockDim.x) {
+        const uint32_t ch = i / direct, r = i - ch * direct;
+        const uint32_t k = r & (nwp - 1), e = r >> kshift;
+        const uint32_t v = e < n_lo ? e : (e - n_lo + 1) << lo_bits;
         uint32_t x = 0;
         for (uint32_t b = 0; b < cb; ++b) {
             const uint32_t t = ch * cb + b;
-            if (t < n_in && ((v >> b) & 1u)) x ^= cols[t * nwp + k];
+            if (t < n_in && ((v >> b) & 1u)) x ^= cols[(t << kshift) + k];
         }
-        tab[i] = x;
+        tab[((((ch << cb) | v)) << kshift) + k] = x;
+    }
+    __syncthreads();
+    const uint32_t total = A.nchunks * (1u << cb) * nwp;
+    for (uint32_t i = threadIdx.x; i < total; i += blockDim.x) {
+        const uint32_t k = i & (nwp - 1), e = i >> kshift;
+        const uint32_t v = e & ((1u << cb) - 1u);
+        const uint32_t l = v & (n_lo - 1), h = v & ~(n_lo - 1);
+        if (l != 0 && h != 0) {
+            const uint32_t chbase = e - v;
+            tab[i] = tab[((chbase | l) << kshift) + k] ^ tab[((chbase | h) << kshift) + k];
+        }
     }
     __syncthreads();
 }
@@ -130,73 +153,240 @@ SQNN_DEV void load_entry(const uint32_t *tab, uint32_t e, uint32_t (&x)[NWP])
     }
 }
 
-// Expands and patches the lane's G slices of warp tile `tile` of `plane` into
-// region[lane * W .. lane * W + W).  N_OUT / N_IN = 0 selects the run-time shape.
+// d_patch entries a warp stages in shared memory per tile: 128 words, of which up to 3 leading
+// bytes are alignment; entries past that are read from global memory one by one.
+constexpr uint32_t STAGE_WORDS = 128;
+constexpr uint32_t STAGE_BYTES = STAGE_WORDS * 4 - 4;
+
+// Compile-time facts of a network shape.
 template <int N_OUT, int N_IN>
-SQNN_DEV void decode_warp_tile(const DecodeArgs &A, uint32_t plane, uint64_t tile,
-                               uint32_t *region, const uint32_t *tab, uint32_t lane)
+struct Shape {
+    static constexpr uint32_t n_out = N_OUT, n_in = N_IN;
+    static constexpr uint32_t G = slices_per_lane(N_OUT), W = G * N_OUT / 32;
+    static constexpr uint32_t NW = entry_words(N_OUT), NWP = entry_words_padded(N_OUT);
+    static constexpr uint32_t NCH = table_chunks(N_IN, NWP), CB = chunk_bits(N_IN, NWP);
+    static constexpr uint32_t SPAN = G * N_IN, NSW = (SPAN + 31) / 32;
+    static_assert(G <= 8, "compile-time shapes keep at most 8 slices per lane");
+};
+
+// What one lane reads from global memory for one tile of one plane.
+template <int N_OUT, int N_IN>
+struct TileIn {
+    uint32_t raw[Shape<N_OUT, N_IN>::NSW + 1];   // words holding the lane's G seeds
+    uint32_t np0, np1, np2;                      // words holding the lane's G n_patch fields
+    uint32_t base, total;                        // the tile's run of d_patch entries
+};
+
+template <int N_OUT, int N_IN>
+SQNN_DEV void tile_fetch(const PlanePtrs &P, uint64_t tile, uint32_t lane, TileIn<N_OUT, N_IN> &in)
 {
-    const PlanePtrs &P = A.pl[plane];
-    if constexpr (N_OUT != 0) {
-        constexpr uint32_t n_out = N_OUT, n_in = N_IN;
-        constexpr uint32_t G = slices_per_lane(n_out), W = G * n_out / 32;
-        constexpr uint32_t NW = entry_words(n_out), NWP = entry_words_padded(n_out);
-        constexpr uint32_t NCH = table_chunks(n_in, NWP), CB = chunk_bits(n_in, NWP);
-        const uint64_t s0 = (tile * 32 + lane) * G;
-        uint32_t *mine = region + lane * W;
-        uint32_t seeds[G];
+    using S = Shape<N_OUT, N_IN>;
+    const uint32_t *w = P.wc + tile * (S::G * S::n_in) + ((lane * S::SPAN) >> 5);
 #pragma unroll
-        for (uint32_t i = 0; i < G; ++i) seeds[i] = extract_bits(P.wc, (s0 + i) * n_in, n_in);
-        uint64_t acc = 0;
-        uint32_t have = 0, wp = 0;
+    for (uint32_t k = 0; k <= S::NSW; ++k) in.raw[k] = __ldg(w + k);
+    in.base = in.total = in.np0 = in.np1 = in.np2 = 0;
+    if (P.w_np != 0) {
+        const uint32_t *ix = P.idx + tile * (S::G / 4);
+        in.base = __ldg(ix);
+        in.total = __ldg(ix + S::G / 4) - in.base;
+        const uint32_t *q = P.np + tile * (S::G * P.w_np) + ((lane * S::G * P.w_np) >> 5);
+        in.np0 = __ldg(q);
+        in.np1 = __ldg(q + 1);
+        in.np2 = __ldg(q + 2);
+    }
+}
+
+// The tile's staged d_patch words: lane l fetches words l, l + 32, l + 64, l + 96 of the run.
+template <int N_OUT, int N_IN>
+SQNN_DEV void stage_fetch(const DecodeArgs &A, const PlanePtrs &P, TileIn<N_OUT, N_IN> &in, uint32_t lane,
+                          uint32_t (&st)[4])
+{
+    st[0] = st[1] = st[2] = st[3] = 0;
+    if (in.total == 0) return;
+    if (in.base > P.n_dp || in.total > P.n_dp - in.base) {       // offsets point outside the section
+        flag(A.status, 2u);
+        in.total = 0;
+        return;
+    }
+    const uint32_t nbytes = in.total < STAGE_BYTES ? in.total : STAGE_BYTES;
+    const uint32_t nwords = ((in.base & 3u) + nbytes + 3) >> 2;
+    const uint32_t *src = reinterpret_cast<const uint32_t *>(P.dp) + (in.base >> 2);
+#pragma unroll
+    for (uint32_t j = 0; j < 4; ++j)
+        if (lane + 32 * j < nwords) st[j] = __ldg(src + lane + 32 * j);
+}
+
+// Flips the lane's patched positions in its private words `mine` (Section 3.2).  `first` is the
+// index, inside the tile's d_patch run, of the lane's first entry; `win` holds the lane's
+// n_patch fields (G fields of w_np bits, least significant first), `cnt` their sum.
+// The fields are rewritten in unary (n_patch ones, then a zero, per slice) so that one flat
+// loop over the lane's entries recovers each entry's slice without nested loops: the j-th one
+// sits at bit b, and b - j zeros (slices) precede it.
+template <uint32_t G, typename WT>
+SQNN_DEV void apply_patches(const DecodeArgs &A, const PlanePtrs &P, uint32_t n_out, uint32_t *mine,
+                            const uint8_t *stage8, uint32_t base, uint32_t total, uint32_t first,
+                            WT win, uint32_t cnt)
+{
+    const uint32_t w_np = P.w_np;
+    const uint32_t fm = (1u << w_np) - 1u;
+    if (cnt + G <= 8 * sizeof(WT)) {
+        WT unary = 0;
+        uint32_t at = 0;
 #pragma unroll
         for (uint32_t i = 0; i < G; ++i) {
-            uint32_t x[NWP];
-            load_entry<NWP>(tab, seeds[i] & ((1u << CB) - 1u), x);
-#pragma unroll
-            for (uint32_t ch = 1; ch < NCH; ++ch) {
-                uint32_t y[NWP];
-                load_entry<NWP>(tab, (ch << CB) | ((seeds[i] >> (ch * CB)) & ((1u << CB) - 1u)), y);
-#pragma unroll
-                for (uint32_t k = 0; k < NW; ++k) x[k] ^= y[k];
-            }
-#pragma unroll
-            for (uint32_t k = 0; k < NW; ++k) {
-                const uint32_t bits = (k == NW - 1) ? n_out - 32 * k : 32;
-                acc |= (uint64_t)x[k] << have;
-                have += bits;
-                if (have >= 32) { mine[wp++] = (uint32_t)acc; acc >>= 32; have -= 32; }
-            }
+            const uint32_t npi = (uint32_t)(win >> (i * w_np)) & fm;
+            unary |= (((WT)1 << npi) - (WT)1) << at;
+            at += npi + 1;
+        }
+        for (uint32_t j = 0; j < cnt; ++j) {
+            uint32_t b;
+            if constexpr (sizeof(WT) == 4) b = (uint32_t)__ffs((int)unary) - 1u;
+            else b = (uint32_t)__ffsll((long long)unary) - 1u;
+            unary &= unary - (WT)1;
+            const uint32_t e = first + j;
+            if (e >= total) { flag(A.status, 2u); break; }            // counts disagree with the offsets
+            const uint32_t pos = e < STAGE_BYTES ? stage8[e] : P.dp[base + e];
+            if (pos >= n_out) { flag(A.status, 1u); continue; }
+            const uint32_t bit = (b - j) * n_out + pos;
+            mine[bit >> 5] ^= 1u << (bit & 31);
         }
     } else {
-        const uint32_t n_out = A.n_out, n_in = A.n_in, G = A.G, W = A.W;
-        const uint32_t nw = A.nw, nwp = A.nwp, nch = A.nchunks, cb = A.cb;
-        const uint32_t cmask = (1u << cb) - 1u;
-        const uint64_t s0 = (tile * 32 + lane) * G;
-        uint32_t *mine = region + lane * W;
-        uint64_t acc = 0;
-        uint32_t have = 0, wp = 0;
+        uint32_t e = first;
+#pragma unroll 1
         for (uint32_t i = 0; i < G; ++i) {
-            const uint32_t seed = extract_bits(P.wc, (s0 + i) * n_in, n_in);
-            for (uint32_t k = 0; k < nw; ++k) {
-                uint32_t x = 0;
-                for (uint32_t ch = 0; ch < nch; ++ch)
-                    x ^= tab[((ch << cb) | ((seed >> (ch * cb)) & cmask)) * nwp + k];
-                const uint32_t bits = (k == nw - 1) ? n_out - 32 * k : 32;
-                acc |= (uint64_t)x << have;
-                have += bits;
-                if (have >= 32) { mine[wp++] = (uint32_t)acc; acc >>= 32; have -= 32; }
+            const uint32_t npi = (uint32_t)(win >> (i * w_np)) & fm;
+            for (uint32_t k = 0; k < npi; ++k, ++e) {
+                if (e >= total) { flag(A.status, 2u); continue; }
+                const uint32_t pos = e < STAGE_BYTES ? stage8[e] : P.dp[base + e];
+                if (pos >= n_out) { flag(A.status, 1u); continue; }
+                const uint32_t bit = i * n_out + pos;
+                mine[bit >> 5] ^= 1u << (bit & 31);
             }
+        }
+    }
+}
+
+template <uint32_t G, typename WT>
+SQNN_DEV void patch_lane(const DecodeArgs &A, const PlanePtrs &P, uint32_t n_out, uint32_t *mine,
+                         const uint32_t *stage, uint32_t base, uint32_t total, WT win, uint32_t lane)
+{
+    const uint32_t fm = (1u << P.w_np) - 1u;
+    uint32_t cnt = 0;
+#pragma unroll
+    for (uint32_t i = 0; i < G; ++i) cnt += (uint32_t)(win >> (i * P.w_np)) & fm;
+    uint32_t incl = cnt;
+#pragma unroll
+    for (uint32_t d = 1; d < 32; d <<= 1) {
+        const uint32_t v = __shfl_up_sync(0xffffffffu, incl, d);
+        if (lane >= d) incl += v;
+    }
+    if (cnt != 0)
+        apply_patches<G, WT>(A, P, n_out, mine, reinterpret_cast<const uint8_t *>(stage) + (base & 3u),
+                             base, total, incl - cnt, win, cnt);
+}
+
+// Expands and patches the lane's G slices of one tile (already fetched into `in`, staged d_patch
+// words in `st`) into region[lane * W .. lane * W + W).  `stage` is the warp's STAGE_WORDS
+// words of shared scratch.  Ends with the warp synchronised.
+template <int N_OUT, int N_IN>
+SQNN_DEV void tile_decode(const DecodeArgs &A, const PlanePtrs &P, const TileIn<N_OUT, N_IN> &in,
+                          const uint32_t (&st)[4], uint32_t *region, const uint32_t *tab, uint32_t *stage,
+                          uint32_t lane)
+{
+    using S = Shape<N_OUT, N_IN>;
+    constexpr uint32_t G = S::G, W = S::W, NW = S::NW, NWP = S::NWP, NCH = S::NCH, CB = S::CB;
+    constexpr uint32_t n_out = S::n_out, n_in = S::n_in, NSW = S::NSW;
+    uint32_t *mine = region + lane * W;
+
+    // seeds -> table entries
+    const uint32_t sh0 = (lane * S::SPAN) & 31u;
+    uint32_t al[NSW];
+#pragma unroll
+    for (uint32_t k = 0; k < NSW; ++k) al[k] = __funnelshift_r(in.raw[k], in.raw[k + 1], sh0);
+    uint32_t x[G][NWP];
+#pragma unroll
+    for (uint32_t i = 0; i < G; ++i) {
+        constexpr uint32_t smask = n_in >= 32 ? 0xffffffffu : ((1u << n_in) - 1u);
+        const uint32_t o = i * n_in, w = o >> 5, s = o & 31;
+        uint32_t seed;
+        if (s + n_in <= 32) seed = (al[w] >> s) & smask;
+        else seed = __funnelshift_r(al[w], al[w + 1 < NSW ? w + 1 : w], s) & smask;
+        load_entry<NWP>(tab, seed & ((1u << CB) - 1u), x[i]);
+#pragma unroll
+        for (uint32_t ch = 1; ch < NCH; ++ch) {
+            uint32_t y[NWP];
+            load_entry<NWP>(tab, (ch << CB) | ((seed >> (ch * CB)) & ((1u << CB) - 1u)), y);
+#pragma unroll
+            for (uint32_t k = 0; k < NW; ++k) x[i][k] ^= y[k];
+        }
+    }
+    // output word k = bits [32k, 32k + 32) of the concatenated entries (entry bits >= n_out are 0)
+#pragma unroll
+    for (uint32_t k = 0; k < W; ++k) {
+        const uint32_t i0 = (32 * k) / n_out, o = 32 * k - i0 * n_out;
+        const uint32_t lo = x[i0][o >> 5];
+        const uint32_t hi = ((o >> 5) + 1 < NW) ? x[i0][((o >> 5) + 1 < NW) ? (o >> 5) + 1 : 0] : 0u;
+        uint32_t word = (o & 31) ? __funnelshift_r(lo, hi, o & 31) : lo;
+        uint32_t filled = n_out - o;
+#pragma unroll
+        for (uint32_t i = i0 + 1; i < G; ++i) {
+            if (filled < 32) { word |= x[i][0] << filled; filled += n_out; }
+        }
+        mine[k] = word;
+    }
+
+    // patches (warp-uniform branch: `total` is the same in every lane)
+    if (in.total != 0) {
+#pragma unroll
+        for (uint32_t j = 0; j < 4; ++j) stage[lane + 32 * j] = st[j];
+        __syncwarp();
+        const uint32_t nb = lane * G * P.w_np, sh = nb & 31u;
+        if (G * P.w_np <= 32) {
+            const uint32_t win = __funnelshift_r(in.np0, in.np1, sh) &
+                                 (G * P.w_np == 32 ? 0xffffffffu : (1u << (G * P.w_np)) - 1u);
+            patch_lane<G, uint32_t>(A, P, n_out, mine, stage, in.base, in.total, win, lane);
+        } else {
+            uint64_t win = (uint64_t)__funnelshift_r(in.np0, in.np1, sh) |
+                           ((uint64_t)__funnelshift_r(in.np1, in.np2, sh) << 32);
+            if (G * P.w_np < 64) win &= (1ull << (G * P.w_np)) - 1ull;
+            patch_lane<G, uint64_t>(A, P, n_out, mine, stage, in.base, in.total, win, lane);
+        }
+    }
+    __syncwarp();
+}
+
+// Fetch + decode of one tile without overlap (for the kernels that do more work per tile).
+template <int N_OUT, int N_IN>
+SQNN_DEV void decode_warp_tile(const DecodeArgs &A, uint32_t plane, uint64_t tile,
+                               uint32_t *region, const uint32_t *tab, uint32_t *stage, uint32_t lane);
+
+// Run-time shape: plain loops, every read through extract_bits.
+SQNN_DEV void decode_warp_tile_generic(const DecodeArgs &A, uint32_t plane, uint64_t tile,
+                                       uint32_t *region, const uint32_t *tab, uint32_t lane)
+{
+    const PlanePtrs &P = A.pl[plane];
+    const uint32_t n_out = A.n_out, n_in = A.n_in, G = A.G, W = A.W;
+    const uint32_t nw = A.nw, nwp = A.nwp, nch = A.nchunks, cb = A.cb;
+    const uint32_t cmask = (1u << cb) - 1u;
+    const uint64_t s0 = (tile * 32 + lane) * G;
+    uint32_t *mine = region + lane * W;
+    uint64_t acc = 0;
+    uint32_t have = 0, wp = 0;
+    for (uint32_t i = 0; i < G; ++i) {
+        const uint32_t seed = extract_bits(P.wc, (s0 + i) * n_in, n_in);
+        for (uint32_t k = 0; k < nw; ++k) {
+            uint32_t x = 0;
+            for (uint32_t ch = 0; ch < nch; ++ch)
+                x ^= tab[((ch << cb) | ((seed >> (ch * cb)) & cmask)) * nwp + k];
+            const uint32_t bits = (k == nw - 1) ? n_out - 32 * k : 32;
+            acc |= (uint64_t)x << have;
+            have += bits;
+            if (have >= 32) { mine[wp++] = (uint32_t)acc; acc >>= 32; have -= 32; }
         }
     }
     // Patches (Section 3.2): the lane's first entry sits at the block offset of the tile plus
     // the n_patch counts of the lanes before it.
     if (P.w_np != 0) {
-        const uint32_t n_out = N_OUT ? (uint32_t)N_OUT : A.n_out;
-        const uint32_t G = N_OUT ? slices_per_lane(N_OUT ? N_OUT : 1) : A.G;
-        const uint32_t W = N_OUT ? G * n_out / 32 : A.W;
-        const uint64_t s0 = (tile * 32 + lane) * G;
-        uint32_t *mine = region + lane * W;
         uint32_t cnt = 0;
         for (uint32_t i = 0; i < G; ++i) cnt += extract_bits(P.np, (s0 + i) * P.w_np, P.w_np);
         uint32_t incl = cnt;
@@ -205,21 +395,36 @@ SQNN_DEV void decode_warp_tile(const DecodeArgs &A, uint32_t plane, uint64_t til
             const uint32_t o = __shfl_up_sync(0xffffffffu, incl, d);
             if (lane >= d) incl += o;
         }
-        if (__any_sync(0xffffffffu, cnt != 0)) {
+        if (cnt != 0) {
             uint32_t at = __ldg(P.idx + tile * (G / 4)) + incl - cnt;
-            if (cnt != 0) {
-                for (uint32_t i = 0; i < G; ++i) {
-                    const uint32_t npi = extract_bits(P.np, (s0 + i) * P.w_np, P.w_np);
-                    for (uint32_t k = 0; k < npi; ++k, ++at) {
-                        if (at >= P.n_dp) { flag(A.status, 2u); continue; }
-                        const uint32_t pos = P.dp[at];
-                        if (pos >= n_out) { flag(A.status, 1u); continue; }
-                        const uint32_t bit = i * n_out + pos;
-                        mine[bit >> 5] ^= 1u << (bit & 31);
-                    }
+            for (uint32_t i = 0; i < G; ++i) {
+                const uint32_t npi = extract_bits(P.np, (s0 + i) * P.w_np, P.w_np);
+                for (uint32_t k = 0; k < npi; ++k, ++at) {
+                    if (at >= P.n_dp) { flag(A.status, 2u); continue; }
+                    const uint32_t pos = P.dp[at];
+                    if (pos >= n_out) { flag(A.status, 1u); continue; }
+                    const uint32_t bit = i * n_out + pos;
+                    mine[bit >> 5] ^= 1u << (bit & 31);
                 }
             }
         }
+    }
+    __syncwarp();
+}
+
+template <int N_OUT, int N_IN>
+SQNN_DEV void decode_warp_tile(const DecodeArgs &A, uint32_t plane, uint64_t tile,
+                               uint32_t *region, const uint32_t *tab, uint32_t *stage, uint32_t lane)
+{
+    if constexpr (N_OUT != 0) {
+        const PlanePtrs &P = A.pl[plane];
+        TileIn<N_OUT, N_IN> in;
+        uint32_t st[4];
+        tile_fetch<N_OUT, N_IN>(P, tile, lane, in);
+        stage_fetch<N_OUT, N_IN>(A, P, in, lane, st);
+        tile_decode<N_OUT, N_IN>(A, P, in, st, region, tab, stage, lane);
+    } else {
+        decode_warp_tile_generic(A, plane, tile, region, tab, lane);
     }
 }
 

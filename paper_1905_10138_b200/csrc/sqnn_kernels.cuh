@@ -1,0 +1,408 @@
+// Decode kernels (packed bits, bf16 weights, checksum sink) and the fused decode-GEMV kernel,
+// as templates over the network shape, with their launchers.
+#pragma once
+#include "sqnn.h"
+#include "sqnn_decode.cuh"
+#include "sqnn_launch.h"
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+namespace sqnn {
+
+// ------------------------------------------------------------------------------------------
+// shared-memory layout of the warp-tile kernels:
+//   [tables][warp 0: regions, d_patch stage][warp 1: ...]...[activations (GEMV only)]
+// a region is a run of 32 * W words (one warp tile of one plane)
+// ------------------------------------------------------------------------------------------
+SQNN_DEV uint64_t tile_word64(const uint32_t *region, uint32_t q)
+{
+    const uint2 v = *reinterpret_cast<const uint2 *>(region + 2 * q);
+    return (uint64_t)v.x | ((uint64_t)v.y << 32);
+}
+
+SQNN_DEV uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+// Asynchronous copy shared -> global by the bulk-copy engine; 16-byte aligned, size % 16 == 0.
+SQNN_DEV void bulk_store(void *gdst, const void *ssrc, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;\n"
+                 :: "l"(gdst), "r"(smem_addr(ssrc)), "r"(bytes) : "memory");
+    asm volatile("cp.async.bulk.commit_group;\n" ::: "memory");
+}
+template <int PENDING>
+SQNN_DEV void bulk_wait_read()
+{
+    asm volatile("cp.async.bulk.wait_group.read %0;\n" :: "n"(PENDING) : "memory");
+}
+SQNN_DEV void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory"); }
+
+template <int N_OUT>
+SQNN_DEV uint32_t words_per_lane(const DecodeArgs &A)
+{
+    if constexpr (N_OUT != 0) return slices_per_lane(N_OUT) * N_OUT / 32;
+    else return A.W;
+}
+
+// K1: decoded planes as packed bits.  One warp tile = 16 * W consecutive uint64 of one plane,
+// built in one of two shared-memory regions and written out by a bulk copy while the warp
+// already decodes its next tile into the other region; the global loads of the next tile are
+// issued before the current tile is expanded.  SINK = true: XOR of all those words instead of
+// storing them.
+template <int N_OUT, int N_IN, bool SINK>
+__global__ void __launch_bounds__(256, 3)
+k_decode_bits(DecodeArgs A, uint64_t *__restrict__ out)
+{
+    extern __shared__ __align__(16) uint32_t smem[];
+    build_tables(A, smem);
+    const uint32_t W = words_per_lane<N_OUT>(A);
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    const uint32_t per_warp = 2 * 32 * W + STAGE_WORDS;
+    uint32_t *mybase = smem + table_words(A.n_in, A.nwp, A.nchunks, A.cb) + warp * per_warp;
+    uint32_t *stage = mybase + 2 * 32 * W;
+    const uint64_t tail_bits = A.mn & 63;
+    // tiles that hold at least one real word, per plane; (plane, tile) advance without division
+    const uint64_t live = (A.words64 + 16 * W - 1) / (16 * W);
+    const uint64_t stride = (uint64_t)gridDim.x * nwarps;
+    uint64_t tile = (uint64_t)blockIdx.x * nwarps + warp;
+    uint32_t plane = 0;
+    while (plane < A.n_q && tile >= live) { tile -= live; ++plane; }
+    uint64_t sink = 0;
+    uint32_t par = 0;
+    if constexpr (N_OUT != 0) {
+        TileIn<N_OUT, N_IN> cur, nxt;
+        if (plane < A.n_q) tile_fetch<N_OUT, N_IN>(A.pl[plane], tile, lane, cur);
+        while (plane < A.n_q) {
+            uint64_t ntile = tile + stride;
+            uint32_t nplane = plane;
+            while (nplane < A.n_q && ntile >= live) { ntile -= live; ++nplane; }
+            if (nplane < A.n_q) tile_fetch<N_OUT, N_IN>(A.pl[nplane], ntile, lane, nxt);
+            uint32_t st[4];
+            stage_fetch<N_OUT, N_IN>(A, A.pl[plane], cur, lane, st);
+            uint32_t *region = mybase + par * 32 * W;
+            if constexpr (!SINK) {
+                if (lane == 0) bulk_wait_read<1>();      // the copy that last read this region is done
+                __syncwarp();
+            }
+            tile_decode<N_OUT, N_IN>(A, A.pl[plane], cur, st, region, smem, stage, lane);
+            const uint64_t q0 = tile * 16 * W;           // first uint64 of the tile inside the plane
+            uint64_t *dst = out + (uint64_t)plane * A.words64 + q0;
+            const bool whole = q0 + 16 * W < A.words64 || (q0 + 16 * W == A.words64 && tail_bits == 0);
+            if (!SINK && whole && (reinterpret_cast<uintptr_t>(dst) & 15) == 0) {
+                fence_async_smem();
+                __syncwarp();
+                if (lane == 0) bulk_store(dst, region, 128 * W);
+            } else {
+                for (uint32_t q = lane; q < 16 * W; q += 32) {
+                    if (q0 + q >= A.words64) break;
+                    uint64_t v = tile_word64(region, q);
+                    if (q0 + q == A.words64 - 1 && tail_bits) v &= (1ull << tail_bits) - 1ull;
+                    if constexpr (SINK) sink ^= v; else dst[q] = v;
+                }
+                __syncwarp();
+            }
+            par ^= 1;
+            cur = nxt;
+            tile = ntile;
+            plane = nplane;
+        }
+    } else {
+        while (plane < A.n_q) {
+            uint32_t *region = mybase;
+            decode_warp_tile<0, 0>(A, plane, tile, region, smem, stage, lane);
+            const uint64_t q0 = tile * 16 * W;
+            uint64_t *dst = out + (uint64_t)plane * A.words64 + q0;
+            for (uint32_t q = lane; q < 16 * W; q += 32) {
+                if (q0 + q >= A.words64) break;
+                uint64_t v = tile_word64(region, q);
+                if (q0 + q == A.words64 - 1 && tail_bits) v &= (1ull << tail_bits) - 1ull;
+                if constexpr (SINK) sink ^= v; else dst[q] = v;
+            }
+            __syncwarp();
+            tile += stride;
+            while (plane < A.n_q && tile >= live) { tile -= live; ++plane; }
+        }
+    }
+    if constexpr (SINK) {
+#pragma unroll
+        for (uint32_t d = 16; d >= 1; d >>= 1) sink ^= __shfl_xor_sync(0xffffffffu, sink, d);
+        if (lane == 0 && sink) atomicXor(reinterpret_cast<unsigned long long *>(out), (unsigned long long)sink);
+    } else {
+        if (lane == 0) bulk_wait_read<0>();              // shared memory must outlive the copies
+    }
+}
+
+// K2: decoded, masked, rescaled weights as bf16.  Lane j of an iteration writes the 8 weights
+// of byte j of a 32-byte group of the tile's bit run, so a warp stores 512 contiguous bytes.
+template <int N_OUT, int N_IN>
+__global__ void __launch_bounds__(256)
+k_decode_bf16(DecodeArgs A, const uint8_t *__restrict__ mask8, const float *__restrict__ alpha,
+              uint64_t n, __nv_bfloat16 *__restrict__ out)
+{
+    extern __shared__ __align__(16) uint32_t smem[];
+    build_tables(A, smem);
+    const uint32_t W = words_per_lane<N_OUT>(A);
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    const uint32_t n_q = A.n_q;
+    const uint32_t per_warp = n_q * 32 * W + STAGE_WORDS;
+    uint32_t *region = smem + table_words(A.n_in, A.nwp, A.nchunks, A.cb) + warp * per_warp;
+    uint32_t *stage = region + n_q * 32 * W;
+    const uint32_t tile_bytes = 128 * W;                 // bytes of bits per tile and plane
+    for (uint64_t tile = (uint64_t)blockIdx.x * nwarps + warp; tile < A.tiles; tile += (uint64_t)gridDim.x * nwarps) {
+        const uint64_t p_tile = tile * (uint64_t)tile_bytes * 8;
+        if (p_tile >= A.mn) continue;
+        for (uint32_t i = 0; i < n_q; ++i)
+            decode_warp_tile<N_OUT, N_IN>(A, i, tile, region + i * 32 * W, smem, stage, lane);
+        __syncwarp();
+        uint64_t p = p_tile + 8ull * lane;               // first weight of this lane's group
+        uint64_t r = p / n;
+        uint64_t c = p - r * n;
+        for (uint32_t t = lane; t < tile_bytes; t += 32, p += 256, c += 256) {
+            if (p >= A.mn) break;
+            while (c >= n) { c -= n; ++r; }
+            const uint32_t mk = mask8[p >> 3];
+            uint32_t bits[8];
+#pragma unroll
+            for (uint32_t i = 0; i < 8; ++i)
+                bits[i] = i < n_q ? reinterpret_cast<const uint8_t *>(region + i * 32 * W)[t] : 0u;
+            __align__(16) __nv_bfloat16 v[8];
+            uint64_t rr = r, cc = c;
+#pragma unroll
+            for (uint32_t k = 0; k < 8; ++k) {
+                if (cc >= n) { cc -= n; ++rr; }
+                float s = 0.0f;
+                if ((mk >> k) & 1u) {
+#pragma unroll
+                    for (uint32_t i = 0; i < 8; ++i) {
+                        if (i < n_q) {
+                            const float a = __ldg(alpha + rr * n_q + i);
+                            s = __fadd_rn(s, ((bits[i] >> k) & 1u) ? a : -a);
+                        }
+                    }
+                }
+                v[k] = __float2bfloat16_rn(s);
+                ++cc;
+            }
+            if (p + 8 <= A.mn) {
+                *reinterpret_cast<uint4 *>(out + p) = *reinterpret_cast<const uint4 *>(v);
+            } else {
+                for (uint32_t k = 0; k < 8 && p + k < A.mn; ++k) out[p + k] = v[k];
+            }
+        }
+        __syncwarp();
+    }
+}
+
+SQNN_DEV float to_float(float v) { return v; }
+SQNN_DEV float to_float(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+// BT activations of one column, stored contiguously in shared memory.
+template <int BT, typename XT>
+SQNN_DEV void load_x(const XT *p, float (&v)[BT])
+{
+    struct __align__(sizeof(XT) * BT > 16 ? 16 : sizeof(XT) * BT) Pack { XT e[BT]; };
+    const Pack pk = *reinterpret_cast<const Pack *>(p);
+#pragma unroll
+    for (int q = 0; q < BT; ++q) v[q] = to_float(pk.e[q]);
+}
+
+// K3: decryption fused with Y[b][r] = sum_c W[r][c] X[b][c] for small batch, fp32 accumulate.
+// A warp decodes its tile of every plane into shared memory, then walks the row segments the
+// tile covers: lanes take the tile's 32-bit words in turn, visit the set bits of the mask word,
+// rebuild the weight value (+-alpha_1) + (+-alpha_2) + ... and accumulate value * x.  Partial
+// sums of a row segment are reduced over the warp and added to Y with one atomic per (row, b).
+// XS = true: the activations of the current batch chunk sit in shared memory as xs[c][BT].
+template <int N_OUT, int N_IN, int BT, typename XT, bool XS>
+__global__ void __launch_bounds__(256)
+k_decode_gemv(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__restrict__ alpha,
+              const XT *__restrict__ x, int64_t ldx, uint32_t batch, float *__restrict__ y,
+              int64_t ldy, uint32_t n)
+{
+    extern __shared__ __align__(16) uint32_t smem[];
+    build_tables(A, smem);
+    const uint32_t W = words_per_lane<N_OUT>(A);
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    const uint32_t n_q = A.n_q;
+    const uint32_t per_warp = n_q * 32 * W + STAGE_WORDS;
+    uint32_t *warp0 = smem + table_words(A.n_in, A.nwp, A.nchunks, A.cb);
+    uint32_t *region = warp0 + warp * per_warp;
+    uint32_t *stage = region + n_q * 32 * W;
+    XT *xs = reinterpret_cast<XT *>(warp0 + nwarps * per_warp);
+    for (uint32_t bc = 0; bc < batch; bc += BT) {
+        if constexpr (XS) {
+            __syncthreads();
+            for (uint32_t i = threadIdx.x; i < n * BT; i += blockDim.x) {
+                const uint32_t c = i / BT, q = i % BT;
+                xs[i] = bc + q < batch ? x[(int64_t)(bc + q) * ldx + c] : XT(0.0f);
+            }
+            __syncthreads();
+        }
+        for (uint64_t tile = (uint64_t)blockIdx.x * nwarps + warp; tile < A.tiles; tile += (uint64_t)gridDim.x * nwarps) {
+            const uint64_t gw0 = tile * 32 * W;          // first 32-bit word of the tile
+            const uint64_t P0 = gw0 * 32;
+            if (P0 >= A.mn) continue;
+            const uint64_t P1 = (P0 + 1024ull * W < A.mn) ? P0 + 1024ull * W : A.mn;
+            for (uint32_t i = 0; i < n_q; ++i)
+                decode_warp_tile<N_OUT, N_IN>(A, i, tile, region + i * 32 * W, smem, stage, lane);
+            __syncwarp();
+            for (uint64_t r = P0 / n; r * n < P1; ++r) {
+                const uint64_t a = r * n > P0 ? r * n : P0;
+                const uint64_t b = (r + 1) * n < P1 ? (r + 1) * n : P1;
+                float al[8];
+#pragma unroll
+                for (uint32_t i = 0; i < 8; ++i) al[i] = i < n_q ? __ldg(alpha + r * n_q + i) : 0.0f;
+                const uint32_t lw_lo = (uint32_t)((a >> 5) - gw0), lw_hi = (uint32_t)(((b - 1) >> 5) - gw0);
+                const int32_t c_tile = (int32_t)((int64_t)P0 - (int64_t)(r * n));   // column of tile bit 0
+                const uint32_t a_loc = (uint32_t)(a - P0), b_loc = (uint32_t)(b - P0);
+                float acc[BT];
+#pragma unroll
+                for (int q = 0; q < BT; ++q) acc[q] = 0.0f;
+                for (uint32_t lw = lw_lo + lane; lw <= lw_hi; lw += 32) {
+                    uint32_t mk = __ldg(mask32 + gw0 + lw);
+                    const uint32_t lo = lw * 32;
+                    if (lo < a_loc) mk &= 0xffffffffu << (a_loc - lo);
+                    if (lo + 32 > b_loc) mk &= 0xffffffffu >> (lo + 32 - b_loc);
+                    uint32_t wb[8];
+#pragma unroll
+                    for (uint32_t i = 0; i < 8; ++i) wb[i] = i < n_q ? region[i * 32 * W + lw] : 0u;
+                    const int32_t cbase = c_tile + (int32_t)lo;
+                    while (mk) {
+                        const uint32_t k = (uint32_t)__ffs((int)mk) - 1u;
+                        mk &= mk - 1u;
+                        float v = 0.0f;
+#pragma unroll
+                        for (uint32_t i = 0; i < 8; ++i)
+                            if (i < n_q) v += ((wb[i] >> k) & 1u) ? al[i] : -al[i];
+                        const int32_t c = cbase + (int32_t)k;
+                        if constexpr (XS) {
+                            float xv[BT];
+                            load_x<BT, XT>(xs + (uint32_t)c * BT, xv);
+#pragma unroll
+                            for (int q = 0; q < BT; ++q) acc[q] = fmaf(v, xv[q], acc[q]);
+                        } else {
+#pragma unroll
+                            for (int q = 0; q < BT; ++q)
+                                if (bc + q < batch) acc[q] = fmaf(v, to_float(x[(int64_t)(bc + q) * ldx + c]), acc[q]);
+                        }
+                    }
+                }
+#pragma unroll
+                for (int q = 0; q < BT; ++q) {
+                    float s = acc[q];
+#pragma unroll
+                    for (uint32_t d = 16; d >= 1; d >>= 1) s += __shfl_xor_sync(0xffffffffu, s, d);
+                    if (lane == 0 && bc + q < batch) atomicAdd(y + (int64_t)(bc + q) * ldy + r, s);
+                }
+            }
+            __syncwarp();
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// launchers
+// ------------------------------------------------------------------------------------------
+// Picks warps per block so the dynamic shared memory fits; returns 0 if not even one warp fits.
+inline uint32_t pick_warps(const DecodeArgs &A, uint32_t regions, size_t extra, size_t *smem_bytes)
+{
+    const size_t tab = (size_t)table_words(A.n_in, A.nwp, A.nchunks, A.cb) * 4;
+    const size_t per_warp = ((size_t)regions * 32 * A.W + STAGE_WORDS) * 4;
+    const size_t limit = 200 * 1024;
+    if (tab + per_warp + extra > limit) return 0;
+    uint32_t warps = (uint32_t)((limit - tab - extra) / per_warp);
+    if (warps > 8) warps = 8;
+    *smem_bytes = tab + warps * per_warp + extra;
+    return warps;
+}
+
+template <typename K>
+inline int prepare(K kernel, size_t smem)
+{
+    if (smem > 48 * 1024 &&
+        cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return SQNN_E_CUDA;
+    return SQNN_OK;
+}
+
+inline uint32_t grid_for(uint64_t warp_tiles, uint32_t warps, uint32_t blocks_per_sm)
+{
+    uint64_t need = (warp_tiles + warps - 1) / warps;
+    uint64_t cap = (uint64_t)sm_count() * blocks_per_sm;
+    if (need < 1) need = 1;
+    return (uint32_t)(need < cap ? need : cap);
+}
+
+template <int N_OUT, int N_IN>
+inline int launch_decode(const DecodeArgs &A, sqnn_out_mode mode, const uint64_t *d_mask,
+                         const float *d_alpha, uint64_t n, void *d_out, cudaStream_t st)
+{
+    size_t smem = 0;
+    if (mode == SQNN_OUT_BITS || mode == SQNN_OUT_SINK) {
+        const uint32_t warps = pick_warps(A, 2, 0, &smem);
+        if (!warps) return SQNN_E_UNSUPPORTED;
+        const uint64_t live = (A.words64 + 16ull * A.W - 1) / (16ull * A.W);
+        const uint32_t grid = grid_for(live * A.n_q, warps, 3);
+        if (mode == SQNN_OUT_BITS) {
+            auto k = k_decode_bits<N_OUT, N_IN, false>;
+            if (prepare(k, smem)) return SQNN_E_CUDA;
+            k<<<grid, warps * 32, smem, st>>>(A, (uint64_t *)d_out);
+        } else {
+            if (cudaMemsetAsync(d_out, 0, 8, st) != cudaSuccess) return SQNN_E_CUDA;
+            auto k = k_decode_bits<N_OUT, N_IN, true>;
+            if (prepare(k, smem)) return SQNN_E_CUDA;
+            k<<<grid, warps * 32, smem, st>>>(A, (uint64_t *)d_out);
+        }
+    } else {
+        const uint32_t warps = pick_warps(A, A.n_q, 0, &smem);
+        if (!warps) return SQNN_E_UNSUPPORTED;
+        const uint32_t grid = grid_for(A.tiles, warps, 4);
+        auto k = k_decode_bf16<N_OUT, N_IN>;
+        if (prepare(k, smem)) return SQNN_E_CUDA;
+        k<<<grid, warps * 32, smem, st>>>(A, (const uint8_t *)d_mask, d_alpha, n, (__nv_bfloat16 *)d_out);
+    }
+    return cudaGetLastError() == cudaSuccess ? SQNN_OK : SQNN_E_CUDA;
+}
+
+template <int N_OUT, int N_IN, int BT, typename XT>
+inline int launch_gemv_bt(const DecodeArgs &A, const uint64_t *d_mask, const float *d_alpha, const void *d_x,
+                          int64_t ldx, uint32_t batch, float *d_y, int64_t ldy, uint64_t n, cudaStream_t st)
+{
+    size_t smem = 0;
+    const size_t xbytes = (size_t)n * BT * sizeof(XT);
+    uint32_t warps = xbytes <= 160 * 1024 ? pick_warps(A, A.n_q, xbytes, &smem) : 0;
+    const bool xs = warps != 0;
+    if (!xs) warps = pick_warps(A, A.n_q, 0, &smem);
+    if (!warps) return SQNN_E_UNSUPPORTED;
+    const uint32_t grid = grid_for(A.tiles, warps, 2);
+    if (xs) {
+        auto k = k_decode_gemv<N_OUT, N_IN, BT, XT, true>;
+        if (prepare(k, smem)) return SQNN_E_CUDA;
+        k<<<grid, warps * 32, smem, st>>>(A, (const uint32_t *)d_mask, d_alpha, (const XT *)d_x, ldx, batch, d_y, ldy, (uint32_t)n);
+    } else {
+        auto k = k_decode_gemv<N_OUT, N_IN, BT, XT, false>;
+        if (prepare(k, smem)) return SQNN_E_CUDA;
+        k<<<grid, warps * 32, smem, st>>>(A, (const uint32_t *)d_mask, d_alpha, (const XT *)d_x, ldx, batch, d_y, ldy, (uint32_t)n);
+    }
+    return cudaGetLastError() == cudaSuccess ? SQNN_OK : SQNN_E_CUDA;
+}
+
+template <int N_OUT, int N_IN, typename XT>
+inline int launch_gemv(const DecodeArgs &A, const uint64_t *d_mask, const float *d_alpha, const void *d_x,
+                       int64_t ldx, uint32_t batch, float *d_y, int64_t ldy, uint64_t n, cudaStream_t st)
+{
+    if (batch == 1) return launch_gemv_bt<N_OUT, N_IN, 1, XT>(A, d_mask, d_alpha, d_x, ldx, batch, d_y, ldy, n, st);
+    if (batch == 2) return launch_gemv_bt<N_OUT, N_IN, 2, XT>(A, d_mask, d_alpha, d_x, ldx, batch, d_y, ldy, n, st);
+    if (batch <= 4) return launch_gemv_bt<N_OUT, N_IN, 4, XT>(A, d_mask, d_alpha, d_x, ldx, batch, d_y, ldy, n, st);
+    return launch_gemv_bt<N_OUT, N_IN, 8, XT>(A, d_mask, d_alpha, d_x, ldx, batch, d_y, ldy, n, st);
+}
+
+
+// One network shape = one translation unit (sqnn_shape.cu compiled with -DSQNN_NO / -DSQNN_NI).
+template <int N_OUT, int N_IN>
+int decode_shape(const DecodeArgs &A, sqnn_out_mode mode, const uint64_t *d_mask, const float *d_alpha,
+                 uint64_t n, void *d_out, cudaStream_t st);
+template <int N_OUT, int N_IN>
+int gemv_shape(const DecodeArgs &A, const uint64_t *d_mask, const float *d_alpha, const void *d_x, int x_dtype,
+               int64_t ldx, uint32_t batch, float *d_y, int64_t ldy, uint64_t n, cudaStream_t st);
+
+}  // namespace sqnn
