@@ -84,6 +84,23 @@ SQNN_DEV void flag(uint32_t *status, uint32_t code)
     if (status) atomicMax(status, code);
 }
 
+SQNN_DEV uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+// Asynchronous copy shared -> global by the bulk-copy engine; 16-byte aligned, size % 16 == 0.
+SQNN_DEV void bulk_store(void *gdst, const void *ssrc, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;\n"
+                 :: "l"(gdst), "r"(smem_addr(ssrc)), "r"(bytes) : "memory");
+    asm volatile("cp.async.bulk.commit_group;\n" ::: "memory");
+}
+// Waits until at most PENDING of this thread's bulk copies still read their shared source.
+template <int PENDING>
+SQNN_DEV void bulk_wait_read()
+{
+    asm volatile("cp.async.bulk.wait_group.read %0;\n" :: "n"(PENDING) : "memory");
+}
+SQNN_DEV void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory"); }
+
 // Shared-memory words the tables need, rounded so that what follows stays 16-byte aligned.
 inline __host__ __device__ uint32_t table_words(uint32_t n_in, uint32_t nwp, uint32_t nchunks, uint32_t cb)
 {
@@ -220,8 +237,9 @@ SQNN_DEV void stage_fetch(const DecodeArgs &A, const PlanePtrs &P, TileIn<N_OUT,
 // index, inside the tile's d_patch run, of the lane's first entry; `win` holds the lane's
 // n_patch fields (G fields of w_np bits, least significant first), `cnt` their sum.
 // The fields are rewritten in unary (n_patch ones, then a zero, per slice) so that one flat
-// loop over the lane's entries recovers each entry's slice without nested loops: the j-th one
-// sits at bit b, and b - j zeros (slices) precede it.
+// loop over the lane's entries recovers each entry's slice without nested loops: the one of
+// entry j sits at bit b, and b - j zeros (slices) precede it.  Flips commute, so the loop
+// runs from the last entry down (highest set bit first).
 template <uint32_t G, typename WT>
 SQNN_DEV void apply_patches(const DecodeArgs &A, const PlanePtrs &P, uint32_t n_out, uint32_t *mine,
                             const uint8_t *stage8, uint32_t base, uint32_t total, uint32_t first,
@@ -229,6 +247,10 @@ SQNN_DEV void apply_patches(const DecodeArgs &A, const PlanePtrs &P, uint32_t n_
 {
     const uint32_t w_np = P.w_np;
     const uint32_t fm = (1u << w_np) - 1u;
+    if (first + cnt > total) {                         // counts disagree with the offsets
+        flag(A.status, 2u);
+        return;
+    }
     if (cnt + G <= 8 * sizeof(WT)) {
         WT unary = 0;
         uint32_t at = 0;
@@ -238,25 +260,26 @@ SQNN_DEV void apply_patches(const DecodeArgs &A, const PlanePtrs &P, uint32_t n_
             unary |= (((WT)1 << npi) - (WT)1) << at;
             at += npi + 1;
         }
-        for (uint32_t j = 0; j < cnt; ++j) {
+        uint32_t bad = 0;
+        for (uint32_t j = cnt; j-- > 0;) {
             uint32_t b;
-            if constexpr (sizeof(WT) == 4) b = (uint32_t)__ffs((int)unary) - 1u;
-            else b = (uint32_t)__ffsll((long long)unary) - 1u;
-            unary &= unary - (WT)1;
+            if constexpr (sizeof(WT) == 4) b = 31u - (uint32_t)__clz((int)unary);
+            else b = 63u - (uint32_t)__clzll((long long)unary);
+            unary ^= (WT)1 << b;
             const uint32_t e = first + j;
-            if (e >= total) { flag(A.status, 2u); break; }            // counts disagree with the offsets
             const uint32_t pos = e < STAGE_BYTES ? stage8[e] : P.dp[base + e];
-            if (pos >= n_out) { flag(A.status, 1u); continue; }
             const uint32_t bit = (b - j) * n_out + pos;
-            mine[bit >> 5] ^= 1u << (bit & 31);
+            const uint32_t ok = pos < n_out;
+            bad |= ok ^ 1u;
+            if (ok) atomicXor(mine + (bit >> 5), 1u << (bit & 31));
         }
+        if (bad) flag(A.status, 1u);
     } else {
         uint32_t e = first;
 #pragma unroll 1
         for (uint32_t i = 0; i < G; ++i) {
             const uint32_t npi = (uint32_t)(win >> (i * w_np)) & fm;
             for (uint32_t k = 0; k < npi; ++k, ++e) {
-                if (e >= total) { flag(A.status, 2u); continue; }
                 const uint32_t pos = e < STAGE_BYTES ? stage8[e] : P.dp[base + e];
                 if (pos >= n_out) { flag(A.status, 1u); continue; }
                 const uint32_t bit = i * n_out + pos;
@@ -287,8 +310,9 @@ SQNN_DEV void patch_lane(const DecodeArgs &A, const PlanePtrs &P, uint32_t n_out
 
 // Expands and patches the lane's G slices of one tile (already fetched into `in`, staged d_patch
 // words in `st`) into region[lane * W .. lane * W + W).  `stage` is the warp's STAGE_WORDS
-// words of shared scratch.  Ends with the warp synchronised.
-template <int N_OUT, int N_IN>
+// words of shared scratch.  WAIT_BULK: lane 0 first waits for its pending bulk copy out of
+// `region`, just before the region is overwritten.  Ends with the warp synchronised.
+template <int N_OUT, int N_IN, bool WAIT_BULK = false>
 SQNN_DEV void tile_decode(const DecodeArgs &A, const PlanePtrs &P, const TileIn<N_OUT, N_IN> &in,
                           const uint32_t (&st)[4], uint32_t *region, const uint32_t *tab, uint32_t *stage,
                           uint32_t lane)
@@ -319,6 +343,10 @@ SQNN_DEV void tile_decode(const DecodeArgs &A, const PlanePtrs &P, const TileIn<
 #pragma unroll
             for (uint32_t k = 0; k < NW; ++k) x[i][k] ^= y[k];
         }
+    }
+    if constexpr (WAIT_BULK) {                       // the bulk copy of the previous tile still reads `region`
+        if (lane == 0) bulk_wait_read<0>();
+        __syncwarp();
     }
     // output word k = bits [32k, 32k + 32) of the concatenated entries (entry bits >= n_out are 0)
 #pragma unroll

@@ -21,22 +21,6 @@ SQNN_DEV uint64_t tile_word64(const uint32_t *region, uint32_t q)
     return (uint64_t)v.x | ((uint64_t)v.y << 32);
 }
 
-SQNN_DEV uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-// Asynchronous copy shared -> global by the bulk-copy engine; 16-byte aligned, size % 16 == 0.
-SQNN_DEV void bulk_store(void *gdst, const void *ssrc, uint32_t bytes)
-{
-    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;\n"
-                 :: "l"(gdst), "r"(smem_addr(ssrc)), "r"(bytes) : "memory");
-    asm volatile("cp.async.bulk.commit_group;\n" ::: "memory");
-}
-template <int PENDING>
-SQNN_DEV void bulk_wait_read()
-{
-    asm volatile("cp.async.bulk.wait_group.read %0;\n" :: "n"(PENDING) : "memory");
-}
-SQNN_DEV void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory"); }
-
 template <int N_OUT>
 SQNN_DEV uint32_t words_per_lane(const DecodeArgs &A)
 {
@@ -45,21 +29,22 @@ SQNN_DEV uint32_t words_per_lane(const DecodeArgs &A)
 }
 
 // K1: decoded planes as packed bits.  One warp tile = 16 * W consecutive uint64 of one plane,
-// built in one of two shared-memory regions and written out by a bulk copy while the warp
-// already decodes its next tile into the other region; the global loads of the next tile are
-// issued before the current tile is expanded.  SINK = true: XOR of all those words instead of
+// built in the warp's shared-memory region and written out by a bulk copy while the warp
+// already fetches and expands its next tile (it waits for the copy only when it is about to
+// overwrite the region); the global loads of the next tile are issued before the current tile
+// is expanded.  SINK = true: XOR of all those words instead of
 // storing them.
 template <int N_OUT, int N_IN, bool SINK>
-__global__ void __launch_bounds__(256, 3)
+__global__ void __launch_bounds__(256, 4)
 k_decode_bits(DecodeArgs A, uint64_t *__restrict__ out)
 {
     extern __shared__ __align__(16) uint32_t smem[];
     build_tables(A, smem);
     const uint32_t W = words_per_lane<N_OUT>(A);
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-    const uint32_t per_warp = 2 * 32 * W + STAGE_WORDS;
+    const uint32_t per_warp = 32 * W + STAGE_WORDS;
     uint32_t *mybase = smem + table_words(A.n_in, A.nwp, A.nchunks, A.cb) + warp * per_warp;
-    uint32_t *stage = mybase + 2 * 32 * W;
+    uint32_t *stage = mybase + 32 * W;
     const uint64_t tail_bits = A.mn & 63;
     // tiles that hold at least one real word, per plane; (plane, tile) advance without division
     const uint64_t live = (A.words64 + 16 * W - 1) / (16 * W);
@@ -68,7 +53,6 @@ k_decode_bits(DecodeArgs A, uint64_t *__restrict__ out)
     uint32_t plane = 0;
     while (plane < A.n_q && tile >= live) { tile -= live; ++plane; }
     uint64_t sink = 0;
-    uint32_t par = 0;
     if constexpr (N_OUT != 0) {
         TileIn<N_OUT, N_IN> cur, nxt;
         if (plane < A.n_q) tile_fetch<N_OUT, N_IN>(A.pl[plane], tile, lane, cur);
@@ -79,12 +63,8 @@ k_decode_bits(DecodeArgs A, uint64_t *__restrict__ out)
             if (nplane < A.n_q) tile_fetch<N_OUT, N_IN>(A.pl[nplane], ntile, lane, nxt);
             uint32_t st[4];
             stage_fetch<N_OUT, N_IN>(A, A.pl[plane], cur, lane, st);
-            uint32_t *region = mybase + par * 32 * W;
-            if constexpr (!SINK) {
-                if (lane == 0) bulk_wait_read<1>();      // the copy that last read this region is done
-                __syncwarp();
-            }
-            tile_decode<N_OUT, N_IN>(A, A.pl[plane], cur, st, region, smem, stage, lane);
+            uint32_t *region = mybase;
+            tile_decode<N_OUT, N_IN, !SINK>(A, A.pl[plane], cur, st, region, smem, stage, lane);
             const uint64_t q0 = tile * 16 * W;           // first uint64 of the tile inside the plane
             uint64_t *dst = out + (uint64_t)plane * A.words64 + q0;
             const bool whole = q0 + 16 * W < A.words64 || (q0 + 16 * W == A.words64 && tail_bits == 0);
@@ -101,7 +81,6 @@ k_decode_bits(DecodeArgs A, uint64_t *__restrict__ out)
                 }
                 __syncwarp();
             }
-            par ^= 1;
             cur = nxt;
             tile = ntile;
             plane = nplane;
@@ -338,10 +317,10 @@ inline int launch_decode(const DecodeArgs &A, sqnn_out_mode mode, const uint64_t
 {
     size_t smem = 0;
     if (mode == SQNN_OUT_BITS || mode == SQNN_OUT_SINK) {
-        const uint32_t warps = pick_warps(A, 2, 0, &smem);
+        const uint32_t warps = pick_warps(A, 1, 0, &smem);
         if (!warps) return SQNN_E_UNSUPPORTED;
         const uint64_t live = (A.words64 + 16ull * A.W - 1) / (16ull * A.W);
-        const uint32_t grid = grid_for(live * A.n_q, warps, 3);
+        const uint32_t grid = grid_for(live * A.n_q, warps, 4);
         if (mode == SQNN_OUT_BITS) {
             auto k = k_decode_bits<N_OUT, N_IN, false>;
             if (prepare(k, smem)) return SQNN_E_CUDA;

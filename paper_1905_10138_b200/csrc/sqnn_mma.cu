@@ -1,7 +1,588 @@
-// Fused decode + tcgen05 product for batch >= 16 (placeholder until the kernel lands).
+// K4: decryption fused with the product for batch >= 16 on the 5th-generation tensor cores.
+//
+//   Y[b][r] = sum_c W[r][c] X[b][c],   D (TMEM, fp32) [128 rows of W x N batch columns]
+//                                      += A (shared, bf16, K-major) [128 x 64] . B (shared) [N x 64]^T
+//
+// One CTA owns 128 rows of W and a range of columns.  Per 64-column step
+//   - the decode warps expand the weights of the step into the A stage (bf16, 128-byte rows,
+//     128-byte swizzle) -- the decoded weights exist only in shared memory;
+//   - one thread fetches the matching activations X[bc .. bc+N) x [64 columns] with TMA
+//     (no multicast: every CTA fetches its own tile);
+//   - one thread issues four tcgen05.mma (K = 16 each) that accumulate in tensor memory.
+// Column ranges of different CTAs are summed with fp32 atomics on Y (cleared beforehand).
+//
+// Decoding runs in two phases per 256 columns.  Phase 1, one thread per (row, bit vector):
+// the thread walks the slices that cover its row segment (seed -> XOR tables -> patch flips)
+// and leaves the segment's bits, and the mask bits, in a small shared bit buffer.  Phase 2,
+// one thread per (row, 8 columns): bits -> bf16 values through a per-row table of the 2^n_q
+// sums (+-alpha_1) + (+-alpha_2) + ..., rounded to bf16, zero where the mask is 0.
+//
+// Every wait on an mbarrier is bounded; a wait that gives up sets SQNN_E_TIMEOUT in the status
+// word and makes all roles leave their loops, so the kernel always returns.
 #include "sqnn_launch.h"
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
 namespace sqnn {
-size_t mma_workspace_bytes(const sqnn_desc *, uint32_t) { return 0; }
-int mma_dispatch(const sqnn_desc *, const DecodeArgs &, const uint64_t *, const float *, const void *, int64_t,
-                 uint32_t, float *, int64_t, void *, cudaStream_t) { return SQNN_E_UNSUPPORTED; }
+
+namespace {
+
+constexpr uint32_t ROWS = 128;            // rows of W per CTA = MMA M
+constexpr uint32_t KC = 64;               // columns per pipeline step
+constexpr uint32_t MACRO = 256;           // columns decoded to bits at a time
+constexpr uint32_t STEPS_PER_MACRO = MACRO / KC;
+constexpr uint32_t RB_WORDS = MACRO / 32 + 1;   // words per row of the bit buffer (odd stride)
+constexpr uint32_t DEC_WARPS = 8;
+constexpr uint32_t DEC_THREADS = DEC_WARPS * 32;
+constexpr uint32_t THREADS = DEC_THREADS + 64;  // + TMA warp + MMA warp
+constexpr uint32_t A_STAGE_BYTES = ROWS * KC * 2;
+constexpr uint32_t MAX_STAGES = 4;
+constexpr uint64_t WAIT_LIMIT_CYCLES = 4000000000ull;   // about 2 s at 2 GHz
+
+struct MmaArgs {
+    DecodeArgs A;                 // with small tables (<= 4 KB)
+    const uint32_t *mask32;
+    uint64_t mask_words32;        // number of valid 32-bit mask words
+    const float *alpha;
+    float *y;
+    int64_t ldy;
+    uint64_t m, n;
+    uint32_t batch;               // total batch
+    uint32_t nbt;                 // batch columns per pass (multiple of 16, <= 512)
+    uint32_t tmem_cols;           // power of two >= nbt, >= 32
+    uint32_t stages;
+    uint32_t splits;              // CTAs per row tile
+    uint32_t macros_per_split;
+    uint32_t b_stage_bytes;
+};
+
+// ---------------------------------------------------------------------------------------
+// PTX wrappers
+// ---------------------------------------------------------------------------------------
+SQNN_DEV void mbar_init(uint64_t *bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" :: "r"(smem_addr(bar)), "r"(count) : "memory");
 }
+SQNN_DEV void mbar_arrive(uint64_t *bar)
+{
+    asm volatile("{\n .reg .b64 st;\n mbarrier.arrive.shared::cta.b64 st, [%0];\n}\n" :: "r"(smem_addr(bar)) : "memory");
+}
+SQNN_DEV void mbar_expect_tx(uint64_t *bar, uint32_t bytes)
+{
+    asm volatile("{\n .reg .b64 st;\n mbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1;\n}\n"
+                 :: "r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+SQNN_DEV bool mbar_try(uint64_t *bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+                 : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false if the wait was abandoned (limit reached or another role gave up).
+SQNN_DEV bool mbar_wait(uint64_t *bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t *status)
+{
+    if (mbar_try(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (true) {
+        if (mbar_try(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if ((uint64_t)(clock64() - t0) > WAIT_LIMIT_CYCLES) {
+            *abort_flag = 1u;
+            if (status) atomicMax(status, (uint32_t)(-SQNN_E_TIMEOUT));
+            return false;
+        }
+        __nanosleep(32);
+    }
+}
+SQNN_DEV void tma_load_2d(void *sdst, const CUtensorMap *map, uint64_t *bar, int32_t x, int32_t y)
+{
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];\n"
+                 :: "r"(smem_addr(sdst)), "l"(map), "r"(smem_addr(bar)), "r"(x), "r"(y) : "memory");
+}
+SQNN_DEV void tmem_alloc(uint32_t *slot, uint32_t cols)
+{
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n"
+                 :: "r"(smem_addr(slot)), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+}
+SQNN_DEV void tmem_dealloc(uint32_t taddr, uint32_t cols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" :: "r"(taddr), "r"(cols) : "memory");
+}
+SQNN_DEV void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory"); }
+SQNN_DEV void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory"); }
+SQNN_DEV void mma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+                 " tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
+                 :: "r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// Makes the mbarrier track completion of all MMAs this thread issued so far.
+SQNN_DEV void mma_commit(uint64_t *bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n"
+                 :: "r"(smem_addr(bar)) : "memory");
+}
+SQNN_DEV void tmem_ld8(uint32_t taddr, uint32_t (&v)[8])
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];\n"
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+                 : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+}
+
+// Shared-memory matrix descriptor of a K-major bf16 tile with 128-byte rows and 128-byte
+// swizzle: rows 128 B apart, groups of 8 rows 1024 B apart (stride byte offset), descriptor
+// version 1, layout type 2.  `addr` is the shared address of the first row, advanced by 32 B
+// per K = 16 step inside the swizzled row.
+SQNN_DEV uint64_t smem_desc_sw128(uint32_t addr)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((addr >> 4) & 0x3fffu);
+    d |= (uint64_t)1u << 16;                       // leading byte offset (unused for this layout)
+    d |= (uint64_t)(1024u >> 4) << 32;             // stride byte offset
+    d |= (uint64_t)1u << 46;                       // version
+    d |= (uint64_t)2u << 61;                       // 128-byte swizzle
+    return d;
+}
+// Instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = n.
+SQNN_DEV uint32_t instr_desc_bf16(uint32_t n)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((n >> 3) << 17) | ((ROWS >> 4) << 24);
+}
+
+// Barrier over the decode threads that also ORs a flag, so that all of them take the same exit.
+SQNN_DEV bool decode_barrier_any(uint32_t flagged)
+{
+    uint32_t any;
+    asm volatile("{\n .reg .pred p, q;\n setp.ne.u32 q, %1, 0;\n bar.red.or.pred p, 1, %2, q;\n selp.u32 %0, 1, 0, p;\n}\n"
+                 : "=r"(any) : "r"(flagged), "n"(DEC_THREADS) : "memory");
+    return any != 0;
+}
+
+SQNN_DEV void or_bits(uint32_t *row, uint32_t dst, uint32_t v, uint32_t nb)
+{
+    const uint32_t w = dst >> 5, sh = dst & 31;
+    row[w] |= v << sh;
+    if (sh + nb > 32) row[w + 1] |= v >> (32 - sh);
+}
+
+// Where a row segment stands inside the slice stream of one plane.
+struct Cursor {
+    uint64_t s;      // current slice
+    uint32_t off;    // first position of the slice not yet consumed
+    uint32_t dpo;    // index of the slice's first d_patch entry
+};
+
+SQNN_DEV Cursor cursor_at(const PlanePtrs &P, uint32_t n_out, uint64_t p)
+{
+    Cursor c;
+    c.s = p / n_out;
+    c.off = (uint32_t)(p - c.s * n_out);
+    c.dpo = 0;
+    if (P.w_np != 0) {
+        const uint64_t first = c.s & ~(uint64_t)(SQNN_BLOCK_SLICES - 1);
+        c.dpo = __ldg(P.idx + (c.s >> 7));
+        for (uint64_t t = first; t < c.s; ++t) c.dpo += extract_bits(P.np, t * P.w_np, P.w_np);
+    }
+    return c;
+}
+
+// Phase 1 for one plane: bits [cursor, cursor + cnt) of the decoded plane into row[0 .. RB_WORDS).
+SQNN_DEV void decode_segment(const DecodeArgs &A, const PlanePtrs &P, const uint32_t *tab, Cursor &c,
+                             uint32_t cnt, uint32_t *row)
+{
+    const uint32_t n_out = A.n_out, n_in = A.n_in, nw = A.nw, nwp = A.nwp, nch = A.nchunks, cb = A.cb;
+    const uint32_t cmask = (1u << cb) - 1u;
+#pragma unroll
+    for (uint32_t k = 0; k < RB_WORDS; ++k) row[k] = 0;
+    uint32_t pos = 0;
+    while (pos < cnt) {
+        const uint32_t seed = extract_bits(P.wc, c.s * n_in, n_in);
+        const uint32_t np_s = P.w_np ? extract_bits(P.np, c.s * P.w_np, P.w_np) : 0u;
+        const uint32_t o = c.off;
+        for (uint32_t k = 0; k < nw; ++k) {
+            uint32_t lo = 32 * k;
+            uint32_t nb = n_out - lo < 32 ? n_out - lo : 32;
+            if (lo + nb <= o) continue;
+            uint32_t v = 0;
+            for (uint32_t ch = 0; ch < nch; ++ch)
+                v ^= tab[((ch << cb) | ((seed >> (ch * cb)) & cmask)) * nwp + k];
+            if (lo < o) { v >>= (o - lo); nb -= (o - lo); lo = o; }
+            const uint32_t d = pos + (lo - o);
+            if (d < MACRO) or_bits(row, d, v, nb);
+        }
+        for (uint32_t k = 0; k < np_s; ++k) {
+            const uint32_t at = c.dpo + k;
+            if (at >= P.n_dp) { flag(A.status, 2u); break; }
+            const uint32_t pk = P.dp[at];
+            if (pk >= n_out) { flag(A.status, 1u); continue; }
+            if (pk >= o) {
+                const uint32_t d = pos + pk - o;
+                if (d < MACRO) row[d >> 5] ^= 1u << (d & 31);
+            }
+        }
+        const uint32_t avail = n_out - o;
+        if (pos + avail <= cnt) { pos += avail; ++c.s; c.dpo += np_s; c.off = 0; }
+        else { c.off = o + (cnt - pos); pos = cnt; }
+    }
+}
+
+// 8 bits -> one bit per nibble
+SQNN_DEV uint32_t spread8(uint32_t b)
+{
+    uint32_t x = (b | (b << 12)) & 0x000f000fu;
+    x = (x | (x << 6)) & 0x03030303u;
+    x = (x | (x << 3)) & 0x11111111u;
+    return x;
+}
+
+__global__ void __launch_bounds__(THREADS, 1)
+k_decode_mma(const __grid_constant__ CUtensorMap xmap, const MmaArgs M)
+{
+    extern __shared__ __align__(16) uint8_t smem_raw[];
+    const DecodeArgs &A = M.A;
+    // carve shared memory (A / B stages need 1024-byte alignment for the 128-byte swizzle)
+    uint8_t *base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t *a_stages = base;
+    uint8_t *b_stages = a_stages + M.stages * A_STAGE_BYTES;
+    uint32_t *tab = reinterpret_cast<uint32_t *>(b_stages + (size_t)M.stages * M.b_stage_bytes);
+    const uint32_t n_items = A.n_q + 1;                                  // planes + mask
+    uint32_t *rb = tab + table_words(A.n_in, A.nwp, A.nchunks, A.cb);     // [item][row][RB_WORDS]
+    __nv_bfloat16 *lut = reinterpret_cast<__nv_bfloat16 *>(rb + n_items * ROWS * RB_WORDS);   // [row][16]
+    float *alpha_s = reinterpret_cast<float *>(lut + ROWS * 16);         // [row][8]
+    uint64_t *bars = reinterpret_cast<uint64_t *>(alpha_s + ROWS * 8);
+    uint64_t *full_a = bars, *full_b = bars + MAX_STAGES, *empty = bars + 2 * MAX_STAGES;
+    uint64_t *accum = bars + 3 * MAX_STAGES;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 3 * MAX_STAGES + 1);
+    volatile uint32_t *abort_flag = tmem_slot + 1;
+
+    const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t row_tile = blockIdx.x / M.splits, split = blockIdx.x % M.splits;
+    const uint64_t r0 = (uint64_t)row_tile * ROWS;
+    const uint32_t total_macros = (uint32_t)((M.n + MACRO - 1) / MACRO);
+    const uint32_t macro_begin = split * M.macros_per_split;
+    const uint32_t macro_end = macro_begin + M.macros_per_split < total_macros ? macro_begin + M.macros_per_split : total_macros;
+    const uint32_t total_steps = (uint32_t)((M.n + KC - 1) / KC);
+
+    if (tid == 0) {
+        for (uint32_t s = 0; s < MAX_STAGES; ++s) {
+            mbar_init(full_a + s, DEC_THREADS);
+            mbar_init(full_b + s, 1);
+            mbar_init(empty + s, 1);
+        }
+        mbar_init(accum, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    }
+    if (warp == DEC_WARPS + 1) tmem_alloc(tmem_slot, M.tmem_cols);
+    build_tables(A, tab);                                   // all threads; ends with __syncthreads
+    if (tid < ROWS) {
+        // per-row scales and the table of all 2^n_q weight values (index bit i = plane i, bit 3 = mask)
+        const uint64_t r = r0 + tid;
+        float al[8];
+#pragma unroll
+        for (uint32_t i = 0; i < 8; ++i) {
+            al[i] = (i < A.n_q && r < M.m) ? __ldg(M.alpha + r * A.n_q + i) : 0.0f;
+            alpha_s[tid * 8 + i] = al[i];
+        }
+        for (uint32_t e = 0; e < 16; ++e) {
+            float s = 0.0f;
+            if (e & 8u) {
+#pragma unroll
+                for (uint32_t i = 0; i < 3; ++i)
+                    if (i < A.n_q) s = __fadd_rn(s, ((e >> i) & 1u) ? al[i] : -al[i]);
+            }
+            lut[tid * 16 + e] = __float2bfloat16_rn(s);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    uint32_t step_count = 0;                    // pipeline steps issued so far (all roles count alike)
+    uint32_t accum_parity = 0;
+    for (uint32_t bc = 0; bc < M.batch; bc += M.nbt) {
+        const uint32_t step_begin = macro_begin * STEPS_PER_MACRO;
+        uint32_t step_end = macro_end * STEPS_PER_MACRO;
+        if (step_end > total_steps) step_end = total_steps;
+        const uint32_t nsteps = step_end > step_begin ? step_end - step_begin : 0;
+
+        if (warp < DEC_WARPS) {
+            // ------------------------------ decode warps ------------------------------
+            const uint32_t prow = tid & (ROWS - 1), phalf = tid >> 7;       // phase-1 role
+            const uint64_t r = r0 + prow;
+            const bool live = r < M.m;
+            Cursor cur[4];
+#pragma unroll
+            for (uint32_t q = 0; q < 4; ++q) {
+                const uint32_t item = phalf + 2 * q;                         // plane index (mask = n_q)
+                if (item < A.n_q && live)
+                    cur[q] = cursor_at(A.pl[item], A.n_out, r * M.n + (uint64_t)macro_begin * MACRO);
+            }
+            uint32_t it = step_count;
+            for (uint32_t mc = macro_begin; mc < macro_end; ++mc) {
+                const uint64_t c0 = (uint64_t)mc * MACRO;
+                const uint32_t cnt = (uint32_t)(M.n - c0 < MACRO ? M.n - c0 : MACRO);
+                // phase 1: bits of this thread's (row, item)s
+#pragma unroll
+                for (uint32_t q = 0; q < 5; ++q) {
+                    const uint32_t item = phalf + 2 * q;
+                    if (item > A.n_q) break;
+                    uint32_t *rowbuf = rb + (item * ROWS + prow) * RB_WORDS;
+                    if (!live) {
+#pragma unroll
+                        for (uint32_t k = 0; k < RB_WORDS; ++k) rowbuf[k] = 0;
+                    } else if (item < A.n_q) {
+                        if (q < 4) decode_segment(A, A.pl[item], tab, cur[q < 4 ? q : 0], cnt, rowbuf);
+                    } else {
+                        const uint64_t p0 = r * M.n + c0;
+                        const uint64_t w0 = p0 >> 5;
+                        const uint32_t sh = (uint32_t)(p0 & 31);
+                        uint32_t prev = w0 < M.mask_words32 ? __ldg(M.mask32 + w0) : 0u;
+#pragma unroll
+                        for (uint32_t k = 0; k < RB_WORDS - 1; ++k) {
+                            const uint32_t next = w0 + k + 1 < M.mask_words32 ? __ldg(M.mask32 + w0 + k + 1) : 0u;
+                            uint32_t v = __funnelshift_r(prev, next, sh);
+                            const uint32_t lo = 32 * k;
+                            if (lo >= cnt) v = 0;
+                            else if (lo + 32 > cnt) v &= (1u << (cnt - lo)) - 1u;
+                            rowbuf[k] = v;
+                            prev = next;
+                        }
+                        rowbuf[RB_WORDS - 1] = 0;
+                    }
+                }
+                asm volatile("bar.sync 1, %0;\n" :: "n"(DEC_THREADS) : "memory");
+                // phase 2: four steps of 64 columns
+                const uint32_t steps_here = (cnt + KC - 1) / KC;
+                for (uint32_t ks = 0; ks < steps_here; ++ks, ++it) {
+                    const uint32_t stage = it % M.stages, use = it / M.stages;
+                    if (use > 0 && !mbar_wait(empty + stage, (use - 1) & 1u, abort_flag, A.status)) break;
+                    uint8_t *a_stage = a_stages + stage * A_STAGE_BYTES;
+#pragma unroll
+                    for (uint32_t q = 0; q < 4; ++q) {
+                        const uint32_t id = tid + DEC_THREADS * q;
+                        const uint32_t row = id >> 3, j = id & 7;
+                        const uint32_t byte = ks * 8 + j;
+                        const uint8_t *rb8 = reinterpret_cast<const uint8_t *>(rb);
+                        const uint32_t mb = rb8[((A.n_q * ROWS + row) * RB_WORDS) * 4 + byte];
+                        uint4 out;
+                        if (A.n_q <= 3) {
+                            uint32_t c = spread8(mb) << 3;
+#pragma unroll
+                            for (uint32_t i = 0; i < 3; ++i)
+                                if (i < A.n_q) c |= spread8(rb8[((i * ROWS + row) * RB_WORDS) * 4 + byte]) << i;
+                            const uint16_t *lr = reinterpret_cast<const uint16_t *>(lut) + row * 16;
+                            uint32_t w[4];
+#pragma unroll
+                            for (uint32_t h = 0; h < 4; ++h) {
+                                const uint32_t e0 = (c >> (8 * h)) & 15u, e1 = (c >> (8 * h + 4)) & 15u;
+                                w[h] = (uint32_t)lr[e0] | ((uint32_t)lr[e1] << 16);
+                            }
+                            out = make_uint4(w[0], w[1], w[2], w[3]);
+                        } else {
+                            uint32_t pb[8];
+#pragma unroll
+                            for (uint32_t i = 0; i < 8; ++i)
+                                pb[i] = i < A.n_q ? rb8[((i * ROWS + row) * RB_WORDS) * 4 + byte] : 0u;
+                            uint32_t w[4];
+#pragma unroll
+                            for (uint32_t h = 0; h < 4; ++h) {
+                                uint32_t two = 0;
+#pragma unroll
+                                for (uint32_t e = 0; e < 2; ++e) {
+                                    const uint32_t k = 2 * h + e;
+                                    float s = 0.0f;
+                                    if ((mb >> k) & 1u) {
+#pragma unroll
+                                        for (uint32_t i = 0; i < 8; ++i)
+                                            if (i < A.n_q) {
+                                                const float a = alpha_s[row * 8 + i];
+                                                s = __fadd_rn(s, ((pb[i] >> k) & 1u) ? a : -a);
+                                            }
+                                    }
+                                    two |= (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(s)) << (16 * e);
+                                }
+                                w[h] = two;
+                            }
+                            out = make_uint4(w[0], w[1], w[2], w[3]);
+                        }
+                        *reinterpret_cast<uint4 *>(a_stage + row * 128 + ((j ^ (row & 7)) << 4)) = out;
+                    }
+                    fence_async_smem();                 // generic-proxy writes -> visible to the tensor core
+                    mbar_arrive(full_a + stage);
+                }
+                if (decode_barrier_any(*abort_flag)) break;       // same decision in every decode thread
+            }
+        } else if (warp == DEC_WARPS) {
+            // ------------------------------ TMA producer ------------------------------
+            if (lane == 0) {
+                uint32_t it = step_count;
+                for (uint32_t st = step_begin; st < step_end; ++st, ++it) {
+                    const uint32_t stage = it % M.stages, use = it / M.stages;
+                    if (use > 0 && !mbar_wait(empty + stage, (use - 1) & 1u, abort_flag, A.status)) break;
+                    uint8_t *b_stage = b_stages + (size_t)stage * M.b_stage_bytes;
+                    mbar_expect_tx(full_b + stage, M.b_stage_bytes);
+                    for (uint32_t h = 0; h * 256 < M.nbt; ++h)
+                        tma_load_2d(b_stage + h * 256 * 128, &xmap, full_b + stage, (int32_t)(st * KC),
+                                    (int32_t)(bc + h * 256));
+                }
+            }
+        } else {
+            // ------------------------------ MMA issuer ------------------------------
+            if (lane == 0) {
+                uint32_t it = step_count;
+                const uint32_t nmma = M.nbt > 256 ? 2 : 1;
+                const uint32_t ncols = M.nbt > 256 ? 256 : M.nbt;
+                const uint32_t idesc = instr_desc_bf16(ncols);
+                bool ok = true;
+                for (uint32_t st = step_begin; st < step_end && ok; ++st, ++it) {
+                    const uint32_t stage = it % M.stages, use = it / M.stages;
+                    ok = mbar_wait(full_a + stage, use & 1u, abort_flag, A.status) &&
+                         mbar_wait(full_b + stage, use & 1u, abort_flag, A.status);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t a_addr = smem_addr(a_stages + stage * A_STAGE_BYTES);
+                    const uint32_t b_addr = smem_addr(b_stages + (size_t)stage * M.b_stage_bytes);
+#pragma unroll
+                    for (uint32_t k16 = 0; k16 < KC / 16; ++k16) {
+                        for (uint32_t h = 0; h < nmma; ++h)
+                            mma_bf16(tmem_base + h * 256, smem_desc_sw128(a_addr + k16 * 32),
+                                     smem_desc_sw128(b_addr + h * 256 * 128 + k16 * 32), idesc,
+                                     (st > step_begin || k16 > 0) ? 1u : 0u);
+                    }
+                    mma_commit(empty + stage);          // frees the stage when these MMAs are done
+                }
+                if (ok && nsteps) mma_commit(accum);
+            }
+        }
+        step_count += nsteps;
+
+        // ------------------------------ epilogue ------------------------------
+        if (warp < DEC_WARPS && nsteps) {
+            const bool ready = mbar_wait(accum, accum_parity, abort_flag, A.status);
+            if (__all_sync(0xffffffffu, ready)) {                  // tcgen05.ld needs the whole warp
+                tc_fence_after();
+                const uint32_t quad = warp & 3, half = warp >> 2;
+                const uint64_t r = r0 + quad * 32 + lane;
+                const uint32_t c_begin = half * (M.nbt / 2), c_end = c_begin + M.nbt / 2;
+                for (uint32_t c = c_begin; c < c_end; c += 8) {
+                    uint32_t v[8];
+                    tmem_ld8(tmem_base + ((quad * 32) << 16) + c, v);
+                    if (r < M.m) {
+#pragma unroll
+                        for (uint32_t e = 0; e < 8; ++e)
+                            if (bc + c + e < M.batch)
+                                atomicAdd(M.y + (int64_t)(bc + c + e) * M.ldy + r, __uint_as_float(v[e]));
+                    }
+                }
+            }
+        }
+        if (nsteps) accum_parity ^= 1;
+        tc_fence_before();
+        __syncthreads();                       // accumulators are read before the next pass overwrites them
+        tc_fence_after();
+    }
+    if (warp == DEC_WARPS + 1) tmem_dealloc(tmem_base, M.tmem_cols);
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
+
+// Tables for the per-thread decoder: at most 4 KB.
+void small_tables(DecodeArgs *A)
+{
+    for (uint32_t c = 1; c <= 8; ++c) {
+        const uint32_t cb = (A->n_in + c - 1) / c;
+        if (cb <= 12 && (uint64_t)c * (1ull << cb) * A->nwp * 4 <= 4096) { A->nchunks = c; A->cb = cb; return; }
+    }
+    A->nchunks = 8;
+    A->cb = (A->n_in + 7) / 8;
+}
+
+}  // namespace
+
+size_t mma_workspace_bytes(const sqnn_desc *, uint32_t) { return 0; }
+
+int mma_dispatch(const sqnn_desc *desc, const DecodeArgs &A0, const uint64_t *d_mask, const float *d_alpha,
+                 const void *d_x, int64_t ldx, uint32_t batch, float *d_y, int64_t ldy, void *, cudaStream_t st)
+{
+    if (((uintptr_t)d_x & 15) != 0 || (ldx % 8) != 0) return SQNN_E_UNSUPPORTED;   // TMA: 16-byte base and pitch
+    if (desc->n > 0x7fffffffull || batch > 0x7fffffffu) return SQNN_E_UNSUPPORTED;
+    EncodeTiledFn encode = encode_tiled_fn();
+    if (!encode) return SQNN_E_CUDA;
+
+    MmaArgs M;
+    M.A = A0;
+    small_tables(&M.A);
+    M.mask32 = (const uint32_t *)d_mask;
+    M.mask_words32 = M.A.words64 * 2;
+    M.alpha = d_alpha;
+    M.y = d_y;
+    M.ldy = ldy;
+    M.m = desc->m;
+    M.n = desc->n;
+    M.batch = batch;
+    const uint32_t b16 = (batch + 15) / 16 * 16;
+    M.nbt = b16 > 512 ? 512 : b16;
+    if (M.nbt > 256) M.nbt = 512;                       // two full 256-column MMAs per step
+    M.tmem_cols = 32;
+    while (M.tmem_cols < M.nbt) M.tmem_cols *= 2;
+    M.b_stage_bytes = M.nbt * 128;
+    const size_t fixed = (size_t)table_words(M.A.n_in, M.A.nwp, M.A.nchunks, M.A.cb) * 4 +
+                         (size_t)(M.A.n_q + 1) * ROWS * RB_WORDS * 4 + ROWS * 16 * 2 + ROWS * 8 * 4 +
+                         (3 * MAX_STAGES + 1) * 8 + 16 + 1024;
+    const size_t budget = 220 * 1024;
+    M.stages = MAX_STAGES;
+    while (M.stages > 1 && fixed + (size_t)M.stages * (A_STAGE_BYTES + M.b_stage_bytes) > budget) --M.stages;
+    const size_t smem = fixed + (size_t)M.stages * (A_STAGE_BYTES + M.b_stage_bytes);
+    if (smem > budget) return SQNN_E_UNSUPPORTED;
+
+    const uint32_t row_tiles = (uint32_t)((desc->m + ROWS - 1) / ROWS);
+    const uint32_t total_macros = (uint32_t)((desc->n + MACRO - 1) / MACRO);
+    uint32_t splits = (uint32_t)sm_count() / row_tiles;
+    if (splits < 1) splits = 1;
+    if (splits > total_macros) splits = total_macros;
+    M.macros_per_split = (total_macros + splits - 1) / splits;
+    M.splits = (total_macros + M.macros_per_split - 1) / M.macros_per_split;
+
+    CUtensorMap xmap;
+    const cuuint64_t gdim[2] = {(cuuint64_t)desc->n, (cuuint64_t)batch};
+    const cuuint64_t gstride[1] = {(cuuint64_t)ldx * 2};
+    const cuuint32_t box[2] = {KC, M.nbt > 256 ? 256u : M.nbt};
+    const cuuint32_t estride[2] = {1, 1};
+    if (encode(&xmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(d_x), gdim, gstride, box, estride,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return SQNN_E_CUDA;
+
+    cudaError_t e = (ldy == (int64_t)desc->m)
+        ? cudaMemsetAsync(d_y, 0, (size_t)batch * desc->m * sizeof(float), st)
+        : cudaMemset2DAsync(d_y, (size_t)ldy * sizeof(float), 0, (size_t)desc->m * sizeof(float), batch, st);
+    if (e != cudaSuccess) return SQNN_E_CUDA;
+    if (cudaFuncSetAttribute(k_decode_mma, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return SQNN_E_CUDA;
+    k_decode_mma<<<row_tiles * M.splits, THREADS, smem, st>>>(xmap, M);
+    return cudaGetLastError() == cudaSuccess ? SQNN_OK : SQNN_E_CUDA;
+}
+
+}  // namespace sqnn

@@ -13,7 +13,8 @@ import os
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libsqnn.so")
+# SQNN_LIBRARY overrides the in-tree build (e.g. to try a differently compiled library)
+LIB_PATH = os.environ.get("SQNN_LIBRARY") or os.path.join(_HERE, "libsqnn.so")
 
 MAX_PLANES = 8
 OUT_BITS, OUT_BF16, OUT_SINK = 0, 1, 2

@@ -66,3 +66,57 @@ def test_gemv_respects_row_strides():
     y = ybuf.cpu().numpy()
     assert H.rel_err(y[:, :50], ref) <= TOL_F32
     assert np.all(y[:, 50:] == 7.0)
+
+
+# ----------------------------------------------------------------------------------------------
+# tensor-core path (batch >= 16): weights are rounded to bf16, fp32 accumulation in tensor memory
+# ----------------------------------------------------------------------------------------------
+MMA = [
+    ("cfg2-s-b64", lambda: wl.make_layer(2, m=300, n=9216), 64),          # ragged last row tile
+    ("cfg3-s-b32", lambda: wl.make_layer(3, m=203, n=3000), 32),          # n not a multiple of 64
+    ("cfg4-s-b16", lambda: wl.make_layer(4, m=130, n=16384), 16),
+    ("cfg4-s-b128", lambda: wl.make_layer(4, m=130, n=16384), 128),
+    ("cfg4-s-b512", lambda: wl.make_layer(4, m=130, n=4096), 512),        # two 256-column accumulators
+    ("cfg1-b16", lambda: wl.make_layer(1), 16),
+    ("gen-33x20-q2-b48", lambda: generic_layer(33, 20, 140, 2049 + 7, 0.5, 13, n_q=2), 48),
+    ("gen-96x9-q5-b24", lambda: generic_layer(96, 9, 70, 1000, 0.3, 16, n_q=5), 24),    # arithmetic rescale path
+    ("gen-b300", lambda: generic_layer(100, 10, 129, 520, 0.2, 23), 300),                # padded to 512 columns
+    ("gen-b600", lambda: generic_layer(60, 12, 64, 776, 0.2, 24, n_q=2), 600),           # two passes over the batch
+    ("gen-narrow-n-b16", lambda: generic_layer(40, 12, 300, 24, 0.4, 21), 16),
+]
+
+
+@pytest.mark.parametrize("name,make,batch", MMA, ids=[g[0] for g in MMA])
+def test_fused_tensor_core_product_matches_fp64_oracle(name, make, batch):
+    import torch
+    layer = make()
+    layer.x_dtype = "bf16"
+    x = layer.activations(batch)
+    ref = reference(layer, x)
+    dev = H.DeviceLayer(layer, H.blob_from_library(layer)[0])
+    y = dev.matmul(x, torch.bfloat16)
+    assert y.shape == (batch, layer.m)
+    assert dev.status_value() == 0
+    assert H.rel_err(y, ref) <= TOL_BF16, H.rel_err(y, ref)
+    # tighter: against the same product with the weights rounded to bf16 first, only the fp32
+    # accumulation order differs
+    ref_bits = H.oracle_decode(layer, H.oracle_encode(layer))
+    _, wbf = orc.reconstruct(ref_bits, layer.mask, layer.alpha, want_f32=False)
+    w = (wbf.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    assert H.rel_err(y, x.astype(np.float64) @ w.T) <= 2e-4
+
+
+def test_tensor_core_path_rejects_what_it_cannot_take():
+    import torch
+    from paper_1905_10138_b200 import sqnn
+    layer = wl.make_layer(1)
+    dev = H.DeviceLayer(layer, H.blob_from_library(layer)[0])
+    y = torch.zeros((16, layer.m), dtype=torch.float32, device="cuda")
+    xf = torch.zeros((16, layer.n), dtype=torch.float32, device="cuda")
+    with pytest.raises(sqnn.SqnnError) as e:                       # fp32 activations need batch <= 15
+        sqnn.sqnn_decode_matmul(dev.desc, dev.blob, dev.mask, dev.alpha, xf, y, None, dev.status)
+    assert e.value.status == sqnn.E_UNSUPPORTED
+    xb = torch.zeros((16, layer.n + 3), dtype=torch.bfloat16, device="cuda")[:, : layer.n]
+    with pytest.raises(sqnn.SqnnError) as e:                       # row pitch not a multiple of 16 bytes
+        sqnn.sqnn_decode_matmul(dev.desc, dev.blob, dev.mask, dev.alpha, xb, y, None, dev.status)
+    assert e.value.status == sqnn.E_UNSUPPORTED
