@@ -17,7 +17,6 @@ from __future__ import annotations
 import argparse
 import json
 import os
-import subprocess
 import sys
 import threading
 import time
@@ -47,51 +46,52 @@ def measured_peaks():
 
 
 class ClockSampler:
-    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clock and clock-event (throttle) reasons through NVML (read-only queries) from a
+    thread while the timed region runs."""
 
-    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
-         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-         "clocks_event_reasons.sw_power_cap")
+    REASONS = {"hw_slowdown": 0x8, "sw_power_cap": 0x4, "sw_thermal_slowdown": 0x20,
+               "hw_thermal_slowdown": 0x40}
 
-    def __init__(self, index: int):
-        self.index = index
-        self.lines = []
-        self.proc = None
+    def __init__(self, index: int, period_s: float = 0.002):
+        self.index, self.period = index, period_s
+        self.sm, self.bits, self.smax = [], 0, None
+        self._stop = threading.Event()
+        self._thread = None
+        self.error = None
+
+    def _run(self):
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            visible = os.environ.get("CUDA_VISIBLE_DEVICES")
+            phys = self.index
+            if visible:
+                ids = [v.strip() for v in visible.split(",") if v.strip()]
+                if self.index < len(ids) and ids[self.index].isdigit():
+                    phys = int(ids[self.index])
+            h = pynvml.nvmlDeviceGetHandleByIndex(phys)
+            self.smax = float(pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM))
+            while not self._stop.is_set():
+                self.sm.append(float(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM)))
+                self.bits |= int(pynvml.nvmlDeviceGetCurrentClocksThrottleReasons(h))
+                time.sleep(self.period)
+            pynvml.nvmlShutdown()
+        except Exception as e:                      # noqa: BLE001 - report, never fail the benchmark
+            self.error = repr(e)
 
     def start(self):
-        try:
-            self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-            threading.Thread(target=self._read, daemon=True).start()
-        except OSError:
-            self.proc = None
-
-    def _read(self):
-        for line in self.proc.stdout:
-            self.lines.append(line.strip())
+        self._thread = threading.Thread(target=self._run, daemon=True)
+        self._thread.start()
 
     def stop(self) -> dict:
-        if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.15)
-        self.proc.terminate()
-        sm, smax, reasons = [], None, set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for ln in self.lines:
-            parts = [p.strip() for p in ln.split(",")]
-            if len(parts) < 7:
-                continue
-            try:
-                sm.append(float(parts[0]))
-                smax = float(parts[1])
-            except ValueError:
-                continue
-            for name, val in zip(names, parts[3:7]):
-                if val.lower().startswith("active"):
-                    reasons.add(name)
-        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": smax,
-                "samples": len(sm), "reasons": sorted(reasons)}
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join(timeout=2.0)
+        reasons = sorted(k for k, bit in self.REASONS.items() if self.bits & bit)
+        if self.error:
+            reasons.append("nvml: " + self.error)
+        return {"sm_mhz": float(np.median(self.sm)) if self.sm else None, "sm_max_mhz": self.smax,
+                "samples": len(self.sm), "reasons": reasons}
 
 
 def encode_layer(layer):
@@ -116,6 +116,15 @@ class Flusher:
         self.buf.fill_(self.v)
 
 
+def gpu_spin(torch, cycles=400_000):
+    """Keeps the GPU busy for ~0.2 ms so that the host has queued the timed call before the GPU
+    reaches it (otherwise the event interval would include host launch latency)."""
+    try:
+        torch.cuda._sleep(cycles)
+    except AttributeError:
+        pass
+
+
 def time_steps(torch, fn, steps, warmup, flush):
     """CUDA-event time of each of `steps` calls of fn on the current stream; L2 flushed before each."""
     for _ in range(warmup):
@@ -125,6 +134,7 @@ def time_steps(torch, fn, steps, warmup, flush):
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
     for a, b in ev:
         flush()
+        gpu_spin(torch)
         a.record()
         fn()
         b.record()
@@ -283,8 +293,9 @@ def decode_point(torch, sqnn, wl, i_s, i_m, flush, peaks, steps, warm, m=32768, 
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     words = (layer.mn + 63) // 64
     out = torch.empty(words, dtype=torch.int64, device="cuda")
+    # stream + output (158 MB) exceed L2: timed back to back, no flush
     t = time_steps(torch, lambda: sqnn.sqnn_decode(desc, d_blob, None, None, sqnn.OUT_BITS, out, status),
-                   steps, warm, flush)
+                   steps, warm, lambda: None)
     sink = torch.zeros(2, dtype=torch.int64, device="cuda")
     ts = time_steps(torch, lambda: sqnn.sqnn_decode(desc, d_blob, None, None, sqnn.OUT_SINK, sink, status),
                     steps, warm, flush)

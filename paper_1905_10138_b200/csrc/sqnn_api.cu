@@ -6,6 +6,10 @@
 
 #include <cuda_runtime.h>
 
+#include <map>
+#include <mutex>
+#include <utility>
+
 namespace sqnn {
 
 template <int N_OUT, int N_IN>
@@ -56,6 +60,22 @@ int fill_decode_args(const sqnn_desc *d, const void *d_blob, uint32_t *d_status,
         A->pl[i].w_np = d->w_np[i];
     }
     for (uint32_t i = d->n_q; i < 8; ++i) A->pl[i] = A->pl[0];
+    return SQNN_OK;
+}
+
+int ensure_dynamic_smem(const void *kernel, size_t smem)
+{
+    if (smem <= 48 * 1024) return SQNN_OK;
+    static std::mutex mu;
+    static std::map<std::pair<const void *, int>, size_t> granted;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return SQNN_E_CUDA;
+    std::lock_guard<std::mutex> lock(mu);
+    size_t &have = granted[std::make_pair(kernel, dev)];
+    if (have >= smem) return SQNN_OK;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return SQNN_E_CUDA;
+    have = smem;
     return SQNN_OK;
 }
 

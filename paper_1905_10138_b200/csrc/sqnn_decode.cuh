@@ -112,14 +112,17 @@ inline __host__ __device__ uint32_t table_words(uint32_t n_in, uint32_t nwp, uin
 // are XORed together from the columns directly, every other entry is the XOR of those two.
 SQNN_DEV void build_tables(const DecodeArgs &A, uint32_t *tab)
 {
+    __shared__ uint32_t rows_s[256];                  // rows of M, fetched once with coalesced loads
     const uint32_t nwp = A.nwp, n_in = A.n_in, n_out = A.n_out, cb = A.cb;
     const uint32_t kshift = nwp == 1 ? 0 : nwp == 2 ? 1 : nwp == 4 ? 2 : 3;
     uint32_t *cols = tab + A.nchunks * (1u << cb) * nwp;
+    for (uint32_t j = threadIdx.x; j < n_out; j += blockDim.x) rows_s[j] = __ldg(A.rows + j);
+    __syncthreads();
     for (uint32_t i = threadIdx.x; i < n_in * nwp; i += blockDim.x) {
         const uint32_t t = i >> kshift, k = i & (nwp - 1);
         uint32_t w = 0;
         for (uint32_t j = 32 * k; j < n_out && j < 32 * k + 32; ++j)
-            w |= ((__ldg(A.rows + j) >> t) & 1u) << (j - 32 * k);
+            w |= ((rows_s[j] >> t) & 1u) << (j - 32 * k);
         cols[i] = w;
     }
     __syncthreads();

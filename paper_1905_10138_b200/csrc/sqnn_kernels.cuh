@@ -185,12 +185,23 @@ SQNN_DEV void load_x(const XT *p, float (&v)[BT])
     for (int q = 0; q < BT; ++q) v[q] = to_float(pk.e[q]);
 }
 
+SQNN_DEV void cp_async16(void *sdst, const void *gsrc)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" :: "r"(smem_addr(sdst)), "l"(gsrc) : "memory");
+}
+SQNN_DEV void cp_async_wait_all() { asm volatile("cp.async.wait_all;\n" ::: "memory"); }
+
+// Words of per-warp scratch the GEMV kernel keeps for the scales of the rows a tile touches.
+constexpr uint32_t GEMV_ALPHA_WORDS = 64;
+
 // K3: decryption fused with Y[b][r] = sum_c W[r][c] X[b][c] for small batch, fp32 accumulate.
 // A warp decodes its tile of every plane into shared memory, then walks the row segments the
 // tile covers: lanes take the tile's 32-bit words in turn, visit the set bits of the mask word,
 // rebuild the weight value (+-alpha_1) + (+-alpha_2) + ... and accumulate value * x.  Partial
 // sums of a row segment are reduced over the warp and added to Y with one atomic per (row, b).
-// XS = true: the activations of the current batch chunk sit in shared memory as xs[c][BT].
+// Everything the walk reads is on chip by then: the tile's mask words arrive by cp.async while
+// the tile is decoded, the scales of its rows are fetched up front, and (XS = true) the
+// activations of the current batch chunk sit in shared memory as xs[c][BT].
 template <int N_OUT, int N_IN, int BT, typename XT, bool XS>
 __global__ void __launch_bounds__(256)
 k_decode_gemv(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__restrict__ alpha,
@@ -202,17 +213,35 @@ k_decode_gemv(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__
     const uint32_t W = words_per_lane<N_OUT>(A);
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     const uint32_t n_q = A.n_q;
-    const uint32_t per_warp = n_q * 32 * W + STAGE_WORDS;
+    const uint32_t per_warp = (n_q + 1) * 32 * W + STAGE_WORDS + GEMV_ALPHA_WORDS;
     uint32_t *warp0 = smem + table_words(A.n_in, A.nwp, A.nchunks, A.cb);
     uint32_t *region = warp0 + warp * per_warp;
-    uint32_t *stage = region + n_q * 32 * W;
+    uint32_t *mask_s = region + n_q * 32 * W;
+    uint32_t *stage = mask_s + 32 * W;
+    float *alpha_s = reinterpret_cast<float *>(stage + STAGE_WORDS);
     XT *xs = reinterpret_cast<XT *>(warp0 + nwarps * per_warp);
+    const uint64_t mask_words = A.words64 * 2;
+    const uint64_t alpha_count = (A.mn / n) * n_q;
+    const bool mask_vec = (reinterpret_cast<uintptr_t>(mask32) & 15) == 0;
     for (uint32_t bc = 0; bc < batch; bc += BT) {
         if constexpr (XS) {
             __syncthreads();
-            for (uint32_t i = threadIdx.x; i < n * BT; i += blockDim.x) {
-                const uint32_t c = i / BT, q = i % BT;
-                xs[i] = bc + q < batch ? x[(int64_t)(bc + q) * ldx + c] : XT(0.0f);
+            if (BT == 1 && (reinterpret_cast<uintptr_t>(x + (int64_t)bc * ldx) & 15) == 0) {
+                constexpr uint32_t PER = 16 / sizeof(XT);
+                const uint4 *src = reinterpret_cast<const uint4 *>(x + (int64_t)bc * ldx);
+                uint4 *dst = reinterpret_cast<uint4 *>(xs);
+#pragma unroll 4
+                for (uint32_t v = threadIdx.x; v < n / PER; v += blockDim.x) dst[v] = __ldg(src + v);
+                for (uint32_t c = (n / PER) * PER + threadIdx.x; c < n; c += blockDim.x) xs[c] = x[(int64_t)bc * ldx + c];
+            } else {
+#pragma unroll 4
+                for (uint32_t c = threadIdx.x; c < n; c += blockDim.x) {
+                    XT v[BT];
+#pragma unroll
+                    for (int q = 0; q < BT; ++q) v[q] = bc + q < batch ? x[(int64_t)(bc + q) * ldx + c] : XT(0.0f);
+#pragma unroll
+                    for (int q = 0; q < BT; ++q) xs[c * BT + q] = v[q];
+                }
             }
             __syncthreads();
         }
@@ -221,15 +250,34 @@ k_decode_gemv(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__
             const uint64_t P0 = gw0 * 32;
             if (P0 >= A.mn) continue;
             const uint64_t P1 = (P0 + 1024ull * W < A.mn) ? P0 + 1024ull * W : A.mn;
+            // the tile's mask words: asynchronous 16-byte copies where whole vectors are in range
+            for (uint32_t v = lane; v < 8 * W; v += 32) {
+                if (mask_vec && gw0 + 4 * v + 4 <= mask_words) {
+                    cp_async16(mask_s + 4 * v, mask32 + gw0 + 4 * v);
+                } else {
+#pragma unroll
+                    for (uint32_t e = 0; e < 4; ++e)
+                        mask_s[4 * v + e] = gw0 + 4 * v + e < mask_words ? __ldg(mask32 + gw0 + 4 * v + e) : 0u;
+                }
+            }
+            // scales of the first rows the tile touches (later rows are fetched when reached)
+            const uint64_t r_first = P0 / n;
+            for (uint32_t i = lane; i < GEMV_ALPHA_WORDS; i += 32) {
+                const uint64_t at = r_first * n_q + i;
+                alpha_s[i] = at < alpha_count ? __ldg(alpha + at) : 0.0f;
+            }
             for (uint32_t i = 0; i < n_q; ++i)
                 decode_warp_tile<N_OUT, N_IN>(A, i, tile, region + i * 32 * W, smem, stage, lane);
+            cp_async_wait_all();
             __syncwarp();
-            for (uint64_t r = P0 / n; r * n < P1; ++r) {
+            for (uint64_t r = r_first; r * n < P1; ++r) {
                 const uint64_t a = r * n > P0 ? r * n : P0;
                 const uint64_t b = (r + 1) * n < P1 ? (r + 1) * n : P1;
                 float al[8];
+                const uint32_t ai = (uint32_t)(r - r_first) * n_q;
 #pragma unroll
-                for (uint32_t i = 0; i < 8; ++i) al[i] = i < n_q ? __ldg(alpha + r * n_q + i) : 0.0f;
+                for (uint32_t i = 0; i < 8; ++i)
+                    al[i] = i < n_q ? (ai + i < GEMV_ALPHA_WORDS ? alpha_s[ai + i] : __ldg(alpha + r * n_q + i)) : 0.0f;
                 const uint32_t lw_lo = (uint32_t)((a >> 5) - gw0), lw_hi = (uint32_t)(((b - 1) >> 5) - gw0);
                 const int32_t c_tile = (int32_t)((int64_t)P0 - (int64_t)(r * n));   // column of tile bit 0
                 const uint32_t a_loc = (uint32_t)(a - P0), b_loc = (uint32_t)(b - P0);
@@ -237,7 +285,7 @@ k_decode_gemv(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__
 #pragma unroll
                 for (int q = 0; q < BT; ++q) acc[q] = 0.0f;
                 for (uint32_t lw = lw_lo + lane; lw <= lw_hi; lw += 32) {
-                    uint32_t mk = __ldg(mask32 + gw0 + lw);
+                    uint32_t mk = mask_s[lw];
                     const uint32_t lo = lw * 32;
                     if (lo < a_loc) mk &= 0xffffffffu << (a_loc - lo);
                     if (lo + 32 > b_loc) mk &= 0xffffffffu >> (lo + 32 - b_loc);
@@ -282,10 +330,11 @@ k_decode_gemv(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__
 // launchers
 // ------------------------------------------------------------------------------------------
 // Picks warps per block so the dynamic shared memory fits; returns 0 if not even one warp fits.
-inline uint32_t pick_warps(const DecodeArgs &A, uint32_t regions, size_t extra, size_t *smem_bytes)
+inline uint32_t pick_warps(const DecodeArgs &A, uint32_t regions, size_t extra, size_t *smem_bytes,
+                           uint32_t extra_warp_words = 0)
 {
     const size_t tab = (size_t)table_words(A.n_in, A.nwp, A.nchunks, A.cb) * 4;
-    const size_t per_warp = ((size_t)regions * 32 * A.W + STAGE_WORDS) * 4;
+    const size_t per_warp = ((size_t)regions * 32 * A.W + STAGE_WORDS + extra_warp_words) * 4;
     const size_t limit = 200 * 1024;
     if (tab + per_warp + extra > limit) return 0;
     uint32_t warps = (uint32_t)((limit - tab - extra) / per_warp);
@@ -297,10 +346,7 @@ inline uint32_t pick_warps(const DecodeArgs &A, uint32_t regions, size_t extra, 
 template <typename K>
 inline int prepare(K kernel, size_t smem)
 {
-    if (smem > 48 * 1024 &&
-        cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-        return SQNN_E_CUDA;
-    return SQNN_OK;
+    return ensure_dynamic_smem(reinterpret_cast<const void *>(kernel), smem);
 }
 
 inline uint32_t grid_for(uint64_t warp_tiles, uint32_t warps, uint32_t blocks_per_sm)
@@ -348,9 +394,9 @@ inline int launch_gemv_bt(const DecodeArgs &A, const uint64_t *d_mask, const flo
 {
     size_t smem = 0;
     const size_t xbytes = (size_t)n * BT * sizeof(XT);
-    uint32_t warps = xbytes <= 160 * 1024 ? pick_warps(A, A.n_q, xbytes, &smem) : 0;
+    uint32_t warps = xbytes <= 160 * 1024 ? pick_warps(A, A.n_q + 1, xbytes, &smem, GEMV_ALPHA_WORDS) : 0;
     const bool xs = warps != 0;
-    if (!xs) warps = pick_warps(A, A.n_q, 0, &smem);
+    if (!xs) warps = pick_warps(A, A.n_q + 1, 0, &smem, GEMV_ALPHA_WORDS);
     if (!warps) return SQNN_E_UNSUPPORTED;
     const uint32_t grid = grid_for(A.tiles, warps, 2);
     if (xs) {

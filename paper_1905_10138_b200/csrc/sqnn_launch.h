@@ -6,6 +6,9 @@
 namespace sqnn {
 int fill_decode_args(const sqnn_desc *d, const void *d_blob, uint32_t *d_status, DecodeArgs *A);
 int sm_count();
+// Raises a kernel's dynamic shared-memory limit when `smem` needs it; remembered per kernel and
+// device so that repeated launches cost nothing on the host.
+int ensure_dynamic_smem(const void *kernel, size_t smem);
 size_t mma_workspace_bytes(const sqnn_desc *desc, uint32_t batch);
 int mma_dispatch(const sqnn_desc *desc, const DecodeArgs &A, const uint64_t *d_mask, const float *d_alpha,
                  const void *d_x, int64_t ldx, uint32_t batch, float *d_y, int64_t ldy, void *d_workspace,

@@ -579,8 +579,7 @@ int mma_dispatch(const sqnn_desc *desc, const DecodeArgs &A0, const uint64_t *d_
         ? cudaMemsetAsync(d_y, 0, (size_t)batch * desc->m * sizeof(float), st)
         : cudaMemset2DAsync(d_y, (size_t)ldy * sizeof(float), 0, (size_t)desc->m * sizeof(float), batch, st);
     if (e != cudaSuccess) return SQNN_E_CUDA;
-    if (cudaFuncSetAttribute(k_decode_mma, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-        return SQNN_E_CUDA;
+    if (ensure_dynamic_smem(reinterpret_cast<const void *>(k_decode_mma), smem) != SQNN_OK) return SQNN_E_CUDA;
     k_decode_mma<<<row_tiles * M.splits, THREADS, smem, st>>>(xmap, M);
     return cudaGetLastError() == cudaSuccess ? SQNN_OK : SQNN_E_CUDA;
 }

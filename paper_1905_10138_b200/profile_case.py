@@ -65,6 +65,7 @@ def main():
         if scratch is not None:
             scratch.fill_(it & 0x7F)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda._sleep(400_000)          # let the host queue the call before the GPU gets to it
         e0.record()
         fn()
         e1.record()
