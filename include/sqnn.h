@@ -172,17 +172,22 @@ int sqnn_decode(const sqnn_desc *desc, const void *d_blob, const uint64_t *d_mas
  * reach global memory.  d_x: device, batch rows of n elements (x_dtype SQNN_X_F32 or
  * SQNN_X_BF16), row stride ldx elements.  d_y: device fp32, batch rows of m, row stride ldy;
  * fully overwritten.  batch <= 15 runs the fp32-accumulate GEMV kernel (weights exact);
- * batch >= 16 runs the tcgen05 kernel (weights rounded to bf16, activations must be BF16,
- * fp32 accumulation in tensor memory).  d_workspace: device scratch of at least
- * sqnn_workspace_bytes(desc, batch) bytes, 256-byte aligned, contents undefined before and
- * after (may be NULL when that size is 0).  Errors: INVALID_ARG, UNSUPPORTED (F32 activations
- * with batch >= 16, batch > SQNN_MAX_BATCH), WORKSPACE, CUDA. */
+ * batch >= 16 runs the tcgen05 kernel (weights rounded to bf16, activations must be BF16 with a
+ * 16-byte aligned base and a row pitch that is a multiple of 16 bytes, fp32 accumulation in
+ * tensor memory).  d_workspace: device scratch of at least sqnn_workspace_bytes(desc, batch)
+ * bytes, 256-byte aligned, contents undefined before and after.  For batch >= 16 it receives the
+ * decoded planes as packed bits (1 bit per weight and plane; the rescaled weights themselves
+ * exist only in shared memory), which the tensor-core kernel then reads; it may be NULL, in
+ * which case that kernel decodes the slices itself (same results, slower).  For batch <= 15 it
+ * is not used.  Errors: INVALID_ARG, UNSUPPORTED (F32 activations with batch >= 16, unaligned
+ * activations with batch >= 16, batch > SQNN_MAX_BATCH), WORKSPACE (workspace given but too
+ * small or misaligned), CUDA. */
 int sqnn_decode_matmul(const sqnn_desc *desc, const void *d_blob, const uint64_t *d_mask,
                        const float *d_alpha, const void *d_x, int x_dtype, uint32_t batch,
                        int64_t ldx, float *d_y, int64_t ldy, void *d_workspace,
                        size_t workspace_bytes, uint32_t *d_status, void *cuda_stream);
 
-/* Scratch bytes sqnn_decode_matmul needs for this layer and batch (0 if none). */
+/* Scratch bytes sqnn_decode_matmul can use for this layer and batch (0 if none). */
 size_t sqnn_workspace_bytes(const sqnn_desc *desc, uint32_t batch);
 
 /* Human-readable name of a status code; never NULL. */

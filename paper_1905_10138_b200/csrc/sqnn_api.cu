@@ -109,6 +109,15 @@ static int gemv_dispatch(const DecodeArgs &A, const uint64_t *d_mask, const floa
     return gemv_shape<0, 0>(A, d_mask, d_alpha, d_x, x_dtype, ldx, batch, d_y, ldy, n, st);
 }
 
+int decode_bits_dispatch(const DecodeArgs &A, void *d_out, cudaStream_t st)
+{
+#define SQNN_BITS_CASE(NO, NI) \
+    if (A.n_out == NO && A.n_in == NI) return decode_shape<NO, NI>(A, SQNN_OUT_BITS, nullptr, nullptr, 0, d_out, st);
+    SQNN_FOR_SHAPES(SQNN_BITS_CASE)
+#undef SQNN_BITS_CASE
+    return decode_shape<0, 0>(A, SQNN_OUT_BITS, nullptr, nullptr, 0, d_out, st);
+}
+
 }  // namespace sqnn
 
 using namespace sqnn;
@@ -162,7 +171,10 @@ extern "C" int sqnn_decode_matmul(const sqnn_desc *desc, const void *d_blob, con
     if (batch <= 15)
         return gemv_dispatch(A, d_mask, d_alpha, d_x, x_dtype, ldx, batch, d_y, ldy, desc->m, desc->n, st);
     if (x_dtype != SQNN_X_BF16) return SQNN_E_UNSUPPORTED;
-    const size_t need = mma_workspace_bytes(desc, batch);
-    if (need && (!d_workspace || workspace_bytes < need || ((uintptr_t)d_workspace & 255))) return SQNN_E_WORKSPACE;
+    // With a workspace the planes are decoded to packed bits first (fast tiled decoder) and the
+    // tensor-core kernel reads them from there; without one it decodes inside the kernel (slower).
+    if (d_workspace) {
+        if (workspace_bytes < mma_workspace_bytes(desc, batch) || ((uintptr_t)d_workspace & 255)) return SQNN_E_WORKSPACE;
+    }
     return mma_dispatch(desc, A, d_mask, d_alpha, d_x, ldx, batch, d_y, ldy, d_workspace, st);
 }

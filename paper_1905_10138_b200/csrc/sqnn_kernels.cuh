@@ -202,8 +202,9 @@ constexpr uint32_t GEMV_ALPHA_WORDS = 64;
 // Everything the walk reads is on chip by then: the tile's mask words arrive by cp.async while
 // the tile is decoded, the scales of its rows are fetched up front, and (XS = true) the
 // activations of the current batch chunk sit in shared memory as xs[c][BT].
-template <int N_OUT, int N_IN, int BT, typename XT, bool XS>
-__global__ void __launch_bounds__(256)
+// NQ = number of planes when it is 1, 2 or 3 (scales and plane words stay in registers), 0 = any.
+template <int N_OUT, int N_IN, int BT, typename XT, bool XS, int NQ>
+__global__ void __launch_bounds__(512)
 k_decode_gemv(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__restrict__ alpha,
               const XT *__restrict__ x, int64_t ldx, uint32_t batch, float *__restrict__ y,
               int64_t ldy, uint32_t n)
@@ -273,11 +274,14 @@ k_decode_gemv(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__
             for (uint64_t r = r_first; r * n < P1; ++r) {
                 const uint64_t a = r * n > P0 ? r * n : P0;
                 const uint64_t b = (r + 1) * n < P1 ? (r + 1) * n : P1;
-                float al[8];
+                constexpr int NR = NQ > 0 ? NQ : 1;
+                float al[NR];
                 const uint32_t ai = (uint32_t)(r - r_first) * n_q;
+                if constexpr (NQ > 0) {
 #pragma unroll
-                for (uint32_t i = 0; i < 8; ++i)
-                    al[i] = i < n_q ? (ai + i < GEMV_ALPHA_WORDS ? alpha_s[ai + i] : __ldg(alpha + r * n_q + i)) : 0.0f;
+                    for (int i = 0; i < NQ; ++i)
+                        al[i] = ai + i < GEMV_ALPHA_WORDS ? alpha_s[ai + i] : __ldg(alpha + r * n_q + i);
+                }
                 const uint32_t lw_lo = (uint32_t)((a >> 5) - gw0), lw_hi = (uint32_t)(((b - 1) >> 5) - gw0);
                 const int32_t c_tile = (int32_t)((int64_t)P0 - (int64_t)(r * n));   // column of tile bit 0
                 const uint32_t a_loc = (uint32_t)(a - P0), b_loc = (uint32_t)(b - P0);
@@ -289,17 +293,28 @@ k_decode_gemv(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__
                     const uint32_t lo = lw * 32;
                     if (lo < a_loc) mk &= 0xffffffffu << (a_loc - lo);
                     if (lo + 32 > b_loc) mk &= 0xffffffffu >> (lo + 32 - b_loc);
-                    uint32_t wb[8];
+                    uint32_t wb[NR];
+                    if constexpr (NQ > 0) {
 #pragma unroll
-                    for (uint32_t i = 0; i < 8; ++i) wb[i] = i < n_q ? region[i * 32 * W + lw] : 0u;
+                        for (int i = 0; i < NQ; ++i) wb[i] = region[i * 32 * W + lw];
+                    }
                     const int32_t cbase = c_tile + (int32_t)lo;
                     while (mk) {
-                        const uint32_t k = (uint32_t)__ffs((int)mk) - 1u;
-                        mk &= mk - 1u;
+                        const uint32_t k = 31u - (uint32_t)__clz((int)mk);
+                        mk ^= 1u << k;
                         float v = 0.0f;
+                        if constexpr (NQ > 0) {
 #pragma unroll
-                        for (uint32_t i = 0; i < 8; ++i)
-                            if (i < n_q) v += ((wb[i] >> k) & 1u) ? al[i] : -al[i];
+                            for (int i = 0; i < NQ; ++i) {
+                                const float t = ((wb[i] >> k) & 1u) ? al[i] : -al[i];
+                                v = i == 0 ? t : v + t;
+                            }
+                        } else {
+                            for (uint32_t i = 0; i < n_q; ++i) {
+                                const float a1 = __ldg(alpha + r * n_q + i);
+                                v += ((region[i * 32 * W + lw] >> k) & 1u) ? a1 : -a1;
+                            }
+                        }
                         const int32_t c = cbase + (int32_t)k;
                         if constexpr (XS) {
                             float xv[BT];
@@ -331,14 +346,14 @@ k_decode_gemv(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__
 // ------------------------------------------------------------------------------------------
 // Picks warps per block so the dynamic shared memory fits; returns 0 if not even one warp fits.
 inline uint32_t pick_warps(const DecodeArgs &A, uint32_t regions, size_t extra, size_t *smem_bytes,
-                           uint32_t extra_warp_words = 0)
+                           uint32_t extra_warp_words = 0, uint32_t max_warps = 8)
 {
     const size_t tab = (size_t)table_words(A.n_in, A.nwp, A.nchunks, A.cb) * 4;
     const size_t per_warp = ((size_t)regions * 32 * A.W + STAGE_WORDS + extra_warp_words) * 4;
     const size_t limit = 200 * 1024;
     if (tab + per_warp + extra > limit) return 0;
     uint32_t warps = (uint32_t)((limit - tab - extra) / per_warp);
-    if (warps > 8) warps = 8;
+    if (warps > max_warps) warps = max_warps;
     *smem_bytes = tab + warps * per_warp + extra;
     return warps;
 }
@@ -392,22 +407,30 @@ template <int N_OUT, int N_IN, int BT, typename XT>
 inline int launch_gemv_bt(const DecodeArgs &A, const uint64_t *d_mask, const float *d_alpha, const void *d_x,
                           int64_t ldx, uint32_t batch, float *d_y, int64_t ldy, uint64_t n, cudaStream_t st)
 {
+    // one tile per warp where the layer allows it: warps per block = live tiles / SMs, within [4, 16]
+    const uint64_t live = (A.words64 * 2 + 32ull * A.W - 1) / (32ull * A.W);
+    uint32_t want = (uint32_t)((live + sm_count() - 1) / sm_count());
+    want = want < 4 ? 4 : want > 16 ? 16 : want;
     size_t smem = 0;
     const size_t xbytes = (size_t)n * BT * sizeof(XT);
-    uint32_t warps = xbytes <= 160 * 1024 ? pick_warps(A, A.n_q + 1, xbytes, &smem, GEMV_ALPHA_WORDS) : 0;
+    uint32_t warps = xbytes <= 160 * 1024 ? pick_warps(A, A.n_q + 1, xbytes, &smem, GEMV_ALPHA_WORDS, want) : 0;
     const bool xs = warps != 0;
-    if (!xs) warps = pick_warps(A, A.n_q + 1, 0, &smem, GEMV_ALPHA_WORDS);
+    if (!xs) warps = pick_warps(A, A.n_q + 1, 0, &smem, GEMV_ALPHA_WORDS, want);
     if (!warps) return SQNN_E_UNSUPPORTED;
-    const uint32_t grid = grid_for(A.tiles, warps, 2);
-    if (xs) {
-        auto k = k_decode_gemv<N_OUT, N_IN, BT, XT, true>;
-        if (prepare(k, smem)) return SQNN_E_CUDA;
-        k<<<grid, warps * 32, smem, st>>>(A, (const uint32_t *)d_mask, d_alpha, (const XT *)d_x, ldx, batch, d_y, ldy, (uint32_t)n);
-    } else {
-        auto k = k_decode_gemv<N_OUT, N_IN, BT, XT, false>;
-        if (prepare(k, smem)) return SQNN_E_CUDA;
-        k<<<grid, warps * 32, smem, st>>>(A, (const uint32_t *)d_mask, d_alpha, (const XT *)d_x, ldx, batch, d_y, ldy, (uint32_t)n);
-    }
+    const uint32_t grid = grid_for(live, warps, 2);
+#define SQNN_GEMV_LAUNCH(XSV, NQV)                                                                           \
+    do {                                                                                                     \
+        auto k = k_decode_gemv<N_OUT, N_IN, BT, XT, XSV, NQV>;                                               \
+        if (prepare(k, smem)) return SQNN_E_CUDA;                                                            \
+        k<<<grid, warps * 32, smem, st>>>(A, (const uint32_t *)d_mask, d_alpha, (const XT *)d_x, ldx, batch, \
+                                           d_y, ldy, (uint32_t)n);                                           \
+    } while (0)
+    if (!xs) SQNN_GEMV_LAUNCH(false, 0);
+    else if (A.n_q == 1) SQNN_GEMV_LAUNCH(true, 1);
+    else if (A.n_q == 2) SQNN_GEMV_LAUNCH(true, 2);
+    else if (A.n_q == 3) SQNN_GEMV_LAUNCH(true, 3);
+    else SQNN_GEMV_LAUNCH(true, 0);
+#undef SQNN_GEMV_LAUNCH
     return cudaGetLastError() == cudaSuccess ? SQNN_OK : SQNN_E_CUDA;
 }
 

@@ -56,6 +56,8 @@ struct MmaArgs {
     uint32_t splits;              // CTAs per row tile
     uint32_t macros_per_split;
     uint32_t b_stage_bytes;
+    const uint32_t *bits32;       // decoded planes in the workspace (NULL: decode in this kernel)
+    uint64_t plane_words32;       // 32-bit words per plane in the workspace
 };
 
 // ---------------------------------------------------------------------------------------
@@ -231,6 +233,27 @@ SQNN_DEV void decode_segment(const DecodeArgs &A, const PlanePtrs &P, const uint
     }
 }
 
+// Phase 1 for a vector that already exists as packed bits in global memory (the mask, or a plane
+// decoded into the workspace): bits [p0, p0 + cnt) into row[0 .. RB_WORDS), zero past cnt.
+SQNN_DEV void copy_segment(const uint32_t *__restrict__ src, uint64_t valid_words, uint64_t p0, uint32_t cnt,
+                           uint32_t *row)
+{
+    const uint64_t w0 = p0 >> 5;
+    const uint32_t sh = (uint32_t)(p0 & 31);
+    uint32_t raw[RB_WORDS];
+#pragma unroll
+    for (uint32_t k = 0; k < RB_WORDS; ++k) raw[k] = w0 + k < valid_words ? __ldg(src + w0 + k) : 0u;
+#pragma unroll
+    for (uint32_t k = 0; k < RB_WORDS - 1; ++k) {
+        uint32_t v = __funnelshift_r(raw[k], raw[k + 1], sh);
+        const uint32_t lo = 32 * k;
+        if (lo >= cnt) v = 0;
+        else if (lo + 32 > cnt) v &= (1u << (cnt - lo)) - 1u;
+        row[k] = v;
+    }
+    row[RB_WORDS - 1] = 0;
+}
+
 // 8 bits -> one bit per nibble
 SQNN_DEV uint32_t spread8(uint32_t b)
 {
@@ -321,7 +344,7 @@ k_decode_mma(const __grid_constant__ CUtensorMap xmap, const MmaArgs M)
 #pragma unroll
             for (uint32_t q = 0; q < 4; ++q) {
                 const uint32_t item = phalf + 2 * q;                         // plane index (mask = n_q)
-                if (item < A.n_q && live)
+                if (item < A.n_q && live && !M.bits32)
                     cur[q] = cursor_at(A.pl[item], A.n_out, r * M.n + (uint64_t)macro_begin * MACRO);
             }
             uint32_t it = step_count;
@@ -338,23 +361,13 @@ k_decode_mma(const __grid_constant__ CUtensorMap xmap, const MmaArgs M)
 #pragma unroll
                         for (uint32_t k = 0; k < RB_WORDS; ++k) rowbuf[k] = 0;
                     } else if (item < A.n_q) {
-                        if (q < 4) decode_segment(A, A.pl[item], tab, cur[q < 4 ? q : 0], cnt, rowbuf);
+                        if (M.bits32)
+                            copy_segment(M.bits32 + (uint64_t)item * M.plane_words32, M.plane_words32,
+                                         r * M.n + c0, cnt, rowbuf);
+                        else if (q < 4)
+                            decode_segment(A, A.pl[item], tab, cur[q < 4 ? q : 0], cnt, rowbuf);
                     } else {
-                        const uint64_t p0 = r * M.n + c0;
-                        const uint64_t w0 = p0 >> 5;
-                        const uint32_t sh = (uint32_t)(p0 & 31);
-                        uint32_t prev = w0 < M.mask_words32 ? __ldg(M.mask32 + w0) : 0u;
-#pragma unroll
-                        for (uint32_t k = 0; k < RB_WORDS - 1; ++k) {
-                            const uint32_t next = w0 + k + 1 < M.mask_words32 ? __ldg(M.mask32 + w0 + k + 1) : 0u;
-                            uint32_t v = __funnelshift_r(prev, next, sh);
-                            const uint32_t lo = 32 * k;
-                            if (lo >= cnt) v = 0;
-                            else if (lo + 32 > cnt) v &= (1u << (cnt - lo)) - 1u;
-                            rowbuf[k] = v;
-                            prev = next;
-                        }
-                        rowbuf[RB_WORDS - 1] = 0;
+                        copy_segment(M.mask32, M.mask_words32, r * M.n + c0, cnt, rowbuf);
                     }
                 }
                 asm volatile("bar.sync 1, %0;\n" :: "n"(DEC_THREADS) : "memory");
@@ -521,10 +534,16 @@ void small_tables(DecodeArgs *A)
 
 }  // namespace
 
-size_t mma_workspace_bytes(const sqnn_desc *, uint32_t) { return 0; }
+// Workspace of the two-stage form: the decoded planes as packed bits (1 bit per weight and plane).
+size_t mma_workspace_bytes(const sqnn_desc *desc, uint32_t)
+{
+    const uint64_t words64 = (desc->m * desc->n + 63) / 64;
+    return (size_t)((desc->n_q * words64 * 8 + 255) / 256 * 256);
+}
 
 int mma_dispatch(const sqnn_desc *desc, const DecodeArgs &A0, const uint64_t *d_mask, const float *d_alpha,
-                 const void *d_x, int64_t ldx, uint32_t batch, float *d_y, int64_t ldy, void *, cudaStream_t st)
+                 const void *d_x, int64_t ldx, uint32_t batch, float *d_y, int64_t ldy, void *d_workspace,
+                 cudaStream_t st)
 {
     if (((uintptr_t)d_x & 15) != 0 || (ldx % 8) != 0) return SQNN_E_UNSUPPORTED;   // TMA: 16-byte base and pitch
     if (desc->n > 0x7fffffffull || batch > 0x7fffffffu) return SQNN_E_UNSUPPORTED;
@@ -548,6 +567,8 @@ int mma_dispatch(const sqnn_desc *desc, const DecodeArgs &A0, const uint64_t *d_
     M.tmem_cols = 32;
     while (M.tmem_cols < M.nbt) M.tmem_cols *= 2;
     M.b_stage_bytes = M.nbt * 128;
+    M.bits32 = (const uint32_t *)d_workspace;
+    M.plane_words32 = M.A.words64 * 2;
     const size_t fixed = (size_t)table_words(M.A.n_in, M.A.nwp, M.A.nchunks, M.A.cb) * 4 +
                          (size_t)(M.A.n_q + 1) * ROWS * RB_WORDS * 4 + ROWS * 16 * 2 + ROWS * 8 * 4 +
                          (3 * MAX_STAGES + 1) * 8 + 16 + 1024;
@@ -580,6 +601,11 @@ int mma_dispatch(const sqnn_desc *desc, const DecodeArgs &A0, const uint64_t *d_
         : cudaMemset2DAsync(d_y, (size_t)ldy * sizeof(float), 0, (size_t)desc->m * sizeof(float), batch, st);
     if (e != cudaSuccess) return SQNN_E_CUDA;
     if (ensure_dynamic_smem(reinterpret_cast<const void *>(k_decode_mma), smem) != SQNN_OK) return SQNN_E_CUDA;
+    if (d_workspace) {
+        // stage 1: the decode kernel writes the planes as packed bits into the workspace
+        const int rc = decode_bits_dispatch(A0, d_workspace, st);
+        if (rc != SQNN_OK) return rc;
+    }
     k_decode_mma<<<row_tiles * M.splits, THREADS, smem, st>>>(xmap, M);
     return cudaGetLastError() == cudaSuccess ? SQNN_OK : SQNN_E_CUDA;
 }

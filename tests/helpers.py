@@ -66,14 +66,14 @@ class DeviceLayer:
         torch.cuda.synchronize()
         return out.view(torch.int16).cpu().numpy().view(np.uint16)
 
-    def matmul(self, x_np, dtype):
+    def matmul(self, x_np, dtype, workspace=True):
         """x_np: float32 [batch, n] (already bf16-representable when dtype is bfloat16)."""
         import torch
         x = torch.from_numpy(x_np).cuda().to(dtype)
         batch = x.shape[0]
         y = torch.full((batch, self.layer.m), float("nan"), dtype=torch.float32, device="cuda")
         ws_bytes = sqnn.sqnn_workspace_bytes(self.desc, batch)
-        ws = torch.empty(max(ws_bytes, 256), dtype=torch.uint8, device="cuda")
+        ws = torch.empty(max(ws_bytes, 256), dtype=torch.uint8, device="cuda") if workspace else None
         sqnn.sqnn_decode_matmul(self.desc, self.blob, self.mask, self.alpha, x, y, ws, self.status)
         torch.cuda.synchronize()
         return y.cpu().numpy()

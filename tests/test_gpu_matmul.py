@@ -86,15 +86,18 @@ MMA = [
 ]
 
 
+@pytest.mark.parametrize("workspace", [True, False], ids=["ws", "nows"])
 @pytest.mark.parametrize("name,make,batch", MMA, ids=[g[0] for g in MMA])
-def test_fused_tensor_core_product_matches_fp64_oracle(name, make, batch):
+def test_fused_tensor_core_product_matches_fp64_oracle(name, make, batch, workspace):
+    """workspace=True: planes decoded to packed bits in the workspace first; False: the tensor-core
+    kernel decodes the slices itself."""
     import torch
     layer = make()
     layer.x_dtype = "bf16"
     x = layer.activations(batch)
     ref = reference(layer, x)
     dev = H.DeviceLayer(layer, H.blob_from_library(layer)[0])
-    y = dev.matmul(x, torch.bfloat16)
+    y = dev.matmul(x, torch.bfloat16, workspace=workspace)
     assert y.shape == (batch, layer.m)
     assert dev.status_value() == 0
     assert H.rel_err(y, ref) <= TOL_BF16, H.rel_err(y, ref)
@@ -116,6 +119,11 @@ def test_tensor_core_path_rejects_what_it_cannot_take():
     with pytest.raises(sqnn.SqnnError) as e:                       # fp32 activations need batch <= 15
         sqnn.sqnn_decode_matmul(dev.desc, dev.blob, dev.mask, dev.alpha, xf, y, None, dev.status)
     assert e.value.status == sqnn.E_UNSUPPORTED
+    xok = torch.zeros((16, layer.n), dtype=torch.bfloat16, device="cuda")
+    small = torch.zeros(256, dtype=torch.uint8, device="cuda")
+    with pytest.raises(sqnn.SqnnError) as e:                       # workspace given but too small
+        sqnn.sqnn_decode_matmul(dev.desc, dev.blob, dev.mask, dev.alpha, xok, y, small, dev.status)
+    assert e.value.status == sqnn.E_WORKSPACE
     xb = torch.zeros((16, layer.n + 3), dtype=torch.bfloat16, device="cuda")[:, : layer.n]
     with pytest.raises(sqnn.SqnnError) as e:                       # row pitch not a multiple of 16 bytes
         sqnn.sqnn_decode_matmul(dev.desc, dev.blob, dev.mask, dev.alpha, xb, y, None, dev.status)

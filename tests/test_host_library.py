@@ -184,3 +184,4 @@ def test_device_entry_points_reject_bad_arguments_without_a_gpu():
     assert L.sqnn_decode_matmul(ctypes.byref(d), ctypes.c_void_p(32), None, None, None, 0, 1, 80, None, 16,
                                 None, 0, None, None) == sqnn.E_INVALID_ARG
     assert sqnn.sqnn_workspace_bytes(d, 1) == 0
+    assert sqnn.sqnn_workspace_bytes(d, 16) >= (16 * 80 + 63) // 64 * 8
