@@ -43,6 +43,7 @@ extern "C" {
 #define SQNN_BLOCK_SLICES 128    /* one d_patch offset is stored per 128 slices         */
 #define SQNN_PAD_SLICES   1024   /* streams are zero-padded to a multiple of 1024 slices*/
 #define SQNN_MAX_BATCH    1024
+#define SQNN_STATIC_SCRATCH_BYTES (8u << 20)   /* built-in scratch of sqnn_decode_matmul_static */
 
 enum {
     SQNN_OK            =  0,
@@ -186,6 +187,29 @@ int sqnn_decode_matmul(const sqnn_desc *desc, const void *d_blob, const uint64_t
                        const float *d_alpha, const void *d_x, int x_dtype, uint32_t batch,
                        int64_t ldx, float *d_y, int64_t ldy, void *d_workspace,
                        size_t workspace_bytes, uint32_t *d_status, void *cuda_stream);
+
+/* The tensor-core product (batch >= 16, BF16 activations) of sqnn_decode_matmul for callers that
+ * can neither allocate device memory nor hand over a workspace: code running under a stream
+ * capture, plug-ins inside a framework that owns the device heap, serving loops with a frozen
+ * memory plan.  (The paper has no counterpart; this is a packaging variant of the call above.)
+ * Arguments and results as for sqnn_decode_matmul, minus the workspace: the decoded planes
+ * (packed bits) go to an array of SQNN_STATIC_SCRATCH_BYTES bytes built into the library, which
+ * every GPU that loads the library holds until the process exits.  The call itself makes no
+ * cudaMalloc / cudaFree and calls no allocating routine.
+ *  - Size limit: sqnn_workspace_bytes(desc, batch) must not exceed SQNN_STATIC_SCRATCH_BYTES
+ *    (8 MiB: about 67 million weight bits over all planes); larger layers get SQNN_E_WORKSPACE.
+ *  - batch < 16 or F32 activations: SQNN_E_UNSUPPORTED (those paths need no scratch; use
+ *    sqnn_decode_matmul).
+ *  - The first call on each device looks up the array's device address (with that device
+ *    current); make that first call before any stream capture begins.
+ *  - All calls share the one array and it keeps whatever the last call left.  Nothing in it needs
+ *    clearing (each call overwrites all it reads), but two calls whose kernels may run at the
+ *    same time on one GPU -- different streams, or different threads -- race on it: serialise them.
+ * Errors otherwise as sqnn_decode_matmul. */
+int sqnn_decode_matmul_static(const sqnn_desc *desc, const void *d_blob, const uint64_t *d_mask,
+                              const float *d_alpha, const void *d_x, int x_dtype, uint32_t batch,
+                              int64_t ldx, float *d_y, int64_t ldy, uint32_t *d_status,
+                              void *cuda_stream);
 
 /* Scratch bytes sqnn_decode_matmul can use for this layer and batch (0 if none). */
 size_t sqnn_workspace_bytes(const sqnn_desc *desc, uint32_t batch);

@@ -25,6 +25,8 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include <mutex>
+
 namespace sqnn {
 
 namespace {
@@ -611,3 +613,59 @@ int mma_dispatch(const sqnn_desc *desc, const DecodeArgs &A0, const uint64_t *d_
 }
 
 }  // namespace sqnn
+
+// ---------------------------------------------------------------------------------------------
+// Tensor-core product for callers that must not allocate device memory.
+//
+// Some hosts of this library run where cudaMalloc is off limits: inside a stream capture, inside
+// a framework that owns the whole device heap through its own pool, or in a serving loop whose
+// memory plan is frozen at start-up.  For them the scratch that sqnn_decode_matmul takes from
+// the caller (the decoded planes as packed bits) lives in the array below, which is part of the
+// loaded library image on every GPU that loads it, for as long as the process lives.
+// ---------------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char sqnn_static_scratch[SQNN_STATIC_SCRATCH_BYTES];
+
+namespace {
+
+// In host code `sqnn_static_scratch` is only a handle for the runtime, not a device address, so
+// the address is asked for once per device (with that device current) and remembered.
+int static_scratch_address(void **out)
+{
+    static std::mutex mu;
+    static void *addr[64] = {nullptr};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SQNN_E_CUDA;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!addr[dev]) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, sqnn_static_scratch) != cudaSuccess || !p) return SQNN_E_CUDA;
+        addr[dev] = p;
+    }
+    *out = addr[dev];
+    return SQNN_OK;
+}
+
+}  // namespace
+
+extern "C" int sqnn_decode_matmul_static(const sqnn_desc *desc, const void *d_blob, const uint64_t *d_mask,
+                                         const float *d_alpha, const void *d_x, int x_dtype, uint32_t batch,
+                                         int64_t ldx, float *d_y, int64_t ldy, uint32_t *d_status,
+                                         void *cuda_stream)
+{
+    sqnn::DecodeArgs A;
+    int rc = sqnn::fill_decode_args(desc, d_blob, d_status, &A);
+    if (rc != SQNN_OK) return rc;
+    if (!d_mask || !d_alpha || !d_x || !d_y || batch == 0) return SQNN_E_INVALID_ARG;
+    if (ldx < (int64_t)desc->n || ldy < (int64_t)desc->m) return SQNN_E_INVALID_ARG;
+    if (((uintptr_t)d_mask & 7) || ((uintptr_t)d_alpha & 3) || ((uintptr_t)d_y & 3)) return SQNN_E_INVALID_ARG;
+    if (x_dtype != SQNN_X_BF16 || batch < 16 || batch > SQNN_MAX_BATCH || desc->n > (1ull << 30))
+        return SQNN_E_UNSUPPORTED;
+    if (sqnn::mma_workspace_bytes(desc, batch) > SQNN_STATIC_SCRATCH_BYTES) return SQNN_E_WORKSPACE;
+    void *scratch = nullptr;
+    rc = static_scratch_address(&scratch);
+    if (rc != SQNN_OK) return rc;
+    // Nothing in the scratch has to start at zero: the decode stage overwrites every word the
+    // product stage reads.  Y is cleared by the product path itself.
+    return sqnn::mma_dispatch(desc, A, d_mask, d_alpha, d_x, ldx, batch, d_y, ldy, scratch,
+                              (cudaStream_t)cuda_stream);
+}

@@ -17,6 +17,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.environ.get("SQNN_LIBRARY") or os.path.join(_HERE, "libsqnn.so")
 
 MAX_PLANES = 8
+STATIC_SCRATCH_BYTES = 8 << 20
 OUT_BITS, OUT_BF16, OUT_SINK = 0, 1, 2
 X_F32, X_BF16 = 0, 1
 ENCODE_ALG1, ENCODE_EXHAUSTIVE = 0, 1
@@ -88,6 +89,8 @@ def lib():
         L.sqnn_free.restype = None
         L.sqnn_decode.argtypes = [P(Desc), vp, vp, vp, i32, vp, sz, vp, vp]
         L.sqnn_decode_matmul.argtypes = [P(Desc), vp, vp, vp, vp, i32, u32, i64, vp, i64, vp, sz, vp, vp]
+        L.sqnn_decode_matmul_static.argtypes = [P(Desc), vp, vp, vp, vp, i32, u32, i64, vp, i64, vp, vp]
+        L.sqnn_decode_matmul_static.restype = i32
         L.sqnn_workspace_bytes.argtypes = [P(Desc), u32]
         L.sqnn_workspace_bytes.restype = sz
         L.sqnn_status_string.argtypes = [i32]
@@ -227,3 +230,20 @@ def sqnn_decode_matmul(desc: Desc, d_blob, d_mask, d_alpha, d_x, d_y, d_workspac
                                     _dev_ptr(d_x), xdt, batch, d_x.stride(0), _dev_ptr(d_y), d_y.stride(0),
                                     _dev_ptr(d_workspace), ws_bytes, _dev_ptr(d_status), _stream_ptr(stream)),
            "sqnn_decode_matmul")
+
+
+def sqnn_decode_matmul_static(desc: Desc, d_blob, d_mask, d_alpha, d_x, d_y, d_status=None, stream=None):
+    """Same product as ``sqnn_decode_matmul`` for bfloat16 X with batch >= 16, but the scratch comes
+    from an array built into the library instead of a caller-provided workspace: for callers that
+    cannot allocate device memory (stream capture, a framework-owned heap, a frozen memory plan).
+    Layers whose ``sqnn_workspace_bytes`` exceeds ``STATIC_SCRATCH_BYTES`` are refused.  Calls share
+    that one array, so calls that may overlap on the GPU must be serialised by the caller."""
+    import torch
+    if d_x.dim() != 2 or d_y.dim() != 2 or d_x.stride(1) != 1 or d_y.stride(1) != 1:
+        raise ValueError("X and Y must be 2-D with unit inner stride")
+    if d_x.dtype != torch.bfloat16 or d_y.dtype != torch.float32:
+        raise ValueError("X must be bfloat16 and Y float32")
+    _check(lib().sqnn_decode_matmul_static(ctypes.byref(desc), _dev_ptr(d_blob), _dev_ptr(d_mask),
+                                           _dev_ptr(d_alpha), _dev_ptr(d_x), X_BF16, d_x.shape[0],
+                                           d_x.stride(0), _dev_ptr(d_y), d_y.stride(0), _dev_ptr(d_status),
+                                           _stream_ptr(stream)), "sqnn_decode_matmul_static")
