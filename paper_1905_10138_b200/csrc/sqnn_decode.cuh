@@ -173,10 +173,11 @@ SQNN_DEV void load_entry(const uint32_t *tab, uint32_t e, uint32_t (&x)[NWP])
     }
 }
 
-// d_patch entries a warp stages in shared memory per tile: 128 words, of which up to 3 leading
-// bytes are alignment; entries past that are read from global memory one by one.
-constexpr uint32_t STAGE_WORDS = 128;
-constexpr uint32_t STAGE_BYTES = STAGE_WORDS * 4 - 4;
+// Per-warp scratch of the patch step: 128 words of staged d_patch bytes (one window of up to
+// PATCH_WIN entries, after up to 3 bytes of alignment) and one 16-bit mark per entry of the window.
+constexpr uint32_t PATCH_WIN = 508;
+constexpr uint32_t STAGE_DP_WORDS = 128;
+constexpr uint32_t STAGE_WORDS = STAGE_DP_WORDS + 256;
 
 // Compile-time facts of a network shape.
 template <int N_OUT, int N_IN>
@@ -228,7 +229,7 @@ SQNN_DEV void stage_fetch(const DecodeArgs &A, const PlanePtrs &P, TileIn<N_OUT,
         in.total = 0;
         return;
     }
-    const uint32_t nbytes = in.total < STAGE_BYTES ? in.total : STAGE_BYTES;
+    const uint32_t nbytes = in.total < PATCH_WIN ? in.total : PATCH_WIN;
     const uint32_t nwords = ((in.base & 3u) + nbytes + 3) >> 2;
     const uint32_t *src = reinterpret_cast<const uint32_t *>(P.dp) + (in.base >> 2);
 #pragma unroll
@@ -236,84 +237,91 @@ SQNN_DEV void stage_fetch(const DecodeArgs &A, const PlanePtrs &P, TileIn<N_OUT,
         if (lane + 32 * j < nwords) st[j] = __ldg(src + lane + 32 * j);
 }
 
-// Flips the lane's patched positions in its private words `mine` (Section 3.2).  `first` is the
-// index, inside the tile's d_patch run, of the lane's first entry; `win` holds the lane's
-// n_patch fields (G fields of w_np bits, least significant first), `cnt` their sum.
-// The fields are rewritten in unary (n_patch ones, then a zero, per slice) so that one flat
-// loop over the lane's entries recovers each entry's slice without nested loops: the one of
-// entry j sits at bit b, and b - j zeros (slices) precede it.  Flips commute, so the loop
-// runs from the last entry down (highest set bit first).
+// Flips the patched positions of a tile (Section 3.2), the warp working through the tile's run of
+// d_patch entries 32 at a time.  An entry does not say which slice it belongs to; that follows
+// from the n_patch counts.  Each lane knows where the entries of its own G slices start (a warp
+// scan of the per-lane counts), so it drops a mark "slice id + 1" at the index of each of its
+// slices' first entry; a running maximum over the marks then gives every entry its slice, and
+// the lane holding the entry flips bit slice * n_out + position of the tile with a shared-memory
+// atomic.  Runs longer than PATCH_WIN entries are handled in windows, the running maximum
+// carrying over.  `win` holds the lane's n_patch fields (G fields of w_np bits, lowest first),
+// `st` the first window's d_patch words fetched ahead of time.
 template <uint32_t G, typename WT>
-SQNN_DEV void apply_patches(const DecodeArgs &A, const PlanePtrs &P, uint32_t n_out, uint32_t *mine,
-                            const uint8_t *stage8, uint32_t base, uint32_t total, uint32_t first,
-                            WT win, uint32_t cnt)
+SQNN_DEV void patch_tile(const DecodeArgs &A, const PlanePtrs &P, uint32_t n_out, uint32_t *region,
+                         uint32_t *stage, const uint32_t (&st)[4], uint32_t base, uint32_t total, WT win,
+                         uint32_t lane)
 {
     const uint32_t w_np = P.w_np;
     const uint32_t fm = (1u << w_np) - 1u;
-    if (first + cnt > total) {                         // counts disagree with the offsets
-        flag(A.status, 2u);
-        return;
-    }
-    if (cnt + G <= 8 * sizeof(WT)) {
-        WT unary = 0;
-        uint32_t at = 0;
-#pragma unroll
-        for (uint32_t i = 0; i < G; ++i) {
-            const uint32_t npi = (uint32_t)(win >> (i * w_np)) & fm;
-            unary |= (((WT)1 << npi) - (WT)1) << at;
-            at += npi + 1;
-        }
-        uint32_t bad = 0;
-        for (uint32_t j = cnt; j-- > 0;) {
-            uint32_t b;
-            if constexpr (sizeof(WT) == 4) b = 31u - (uint32_t)__clz((int)unary);
-            else b = 63u - (uint32_t)__clzll((long long)unary);
-            unary ^= (WT)1 << b;
-            const uint32_t e = first + j;
-            const uint32_t pos = e < STAGE_BYTES ? stage8[e] : P.dp[base + e];
-            const uint32_t bit = (b - j) * n_out + pos;
-            const uint32_t ok = pos < n_out;
-            bad |= ok ^ 1u;
-            if (ok) atomicXor(mine + (bit >> 5), 1u << (bit & 31));
-        }
-        if (bad) flag(A.status, 1u);
-    } else {
-        uint32_t e = first;
-#pragma unroll 1
-        for (uint32_t i = 0; i < G; ++i) {
-            const uint32_t npi = (uint32_t)(win >> (i * w_np)) & fm;
-            for (uint32_t k = 0; k < npi; ++k, ++e) {
-                const uint32_t pos = e < STAGE_BYTES ? stage8[e] : P.dp[base + e];
-                if (pos >= n_out) { flag(A.status, 1u); continue; }
-                const uint32_t bit = i * n_out + pos;
-                mine[bit >> 5] ^= 1u << (bit & 31);
-            }
-        }
-    }
-}
-
-template <uint32_t G, typename WT>
-SQNN_DEV void patch_lane(const DecodeArgs &A, const PlanePtrs &P, uint32_t n_out, uint32_t *mine,
-                         const uint32_t *stage, uint32_t base, uint32_t total, WT win, uint32_t lane)
-{
-    const uint32_t fm = (1u << P.w_np) - 1u;
     uint32_t cnt = 0;
 #pragma unroll
-    for (uint32_t i = 0; i < G; ++i) cnt += (uint32_t)(win >> (i * P.w_np)) & fm;
+    for (uint32_t i = 0; i < G; ++i) cnt += (uint32_t)(win >> (i * w_np)) & fm;
     uint32_t incl = cnt;
 #pragma unroll
     for (uint32_t d = 1; d < 32; d <<= 1) {
         const uint32_t v = __shfl_up_sync(0xffffffffu, incl, d);
         if (lane >= d) incl += v;
     }
-    if (cnt != 0)
-        apply_patches<G, WT>(A, P, n_out, mine, reinterpret_cast<const uint8_t *>(stage) + (base & 3u),
-                             base, total, incl - cnt, win, cnt);
+    const uint32_t first = incl - cnt;
+    if (__shfl_sync(0xffffffffu, incl, 31) != total) {      // counts disagree with the offsets
+        flag(A.status, 2u);
+        return;
+    }
+    uint32_t *marks32 = stage + STAGE_DP_WORDS;
+    uint16_t *marks = reinterpret_cast<uint16_t *>(marks32);
+    uint32_t carry = 0, bad = 0;
+    for (uint32_t w0 = 0; w0 < total; w0 += PATCH_WIN) {
+        const uint32_t wn = total - w0 < PATCH_WIN ? total - w0 : PATCH_WIN;
+        const uint32_t ob = (base + w0) & 3u;
+        if (w0 == 0) {
+#pragma unroll
+            for (uint32_t j = 0; j < 4; ++j) stage[lane + 32 * j] = st[j];
+        } else {
+            const uint32_t nwords = (ob + wn + 3) >> 2;
+            const uint32_t *src = reinterpret_cast<const uint32_t *>(P.dp) + ((base + w0) >> 2);
+#pragma unroll
+            for (uint32_t j = 0; j < 4; ++j)
+                if (lane + 32 * j < nwords) stage[lane + 32 * j] = __ldg(src + lane + 32 * j);
+        }
+        for (uint32_t q = lane; q < (wn + 1) / 2; q += 32) marks32[q] = 0;
+        __syncwarp();
+        uint32_t run = first;
+#pragma unroll
+        for (uint32_t i = 0; i < G; ++i) {
+            const uint32_t npi = (uint32_t)(win >> (i * w_np)) & fm;
+            if (npi != 0 && run - w0 < wn) marks[run - w0] = (uint16_t)(lane * G + i + 1);
+            run += npi;
+        }
+        __syncwarp();
+        const uint8_t *bytes = reinterpret_cast<const uint8_t *>(stage) + ob;
+        for (uint32_t e0 = 0; e0 < wn; e0 += 32) {
+            const uint32_t e = e0 + lane;
+            uint32_t v = e < wn ? marks[e] : 0u;
+#pragma unroll
+            for (uint32_t d = 1; d < 32; d <<= 1) {
+                const uint32_t o = __shfl_up_sync(0xffffffffu, v, d);
+                if (lane >= d) v = v > o ? v : o;
+            }
+            v = v > carry ? v : carry;
+            carry = __shfl_sync(0xffffffffu, v, 31);
+            if (e < wn) {
+                const uint32_t pos = bytes[e];
+                if (v == 0 || pos >= n_out) {
+                    bad = 1;
+                } else {
+                    const uint32_t bit = (v - 1) * n_out + pos;
+                    atomicXor(region + (bit >> 5), 1u << (bit & 31));
+                }
+            }
+        }
+        __syncwarp();
+    }
+    if (bad) flag(A.status, 1u);
 }
 
 // Expands and patches the lane's G slices of one tile (already fetched into `in`, staged d_patch
-// words in `st`) into region[lane * W .. lane * W + W).  `stage` is the warp's STAGE_WORDS
-// words of shared scratch.  WAIT_BULK: lane 0 first waits for its pending bulk copy out of
+// words in `st`) into region[lane * W .. lane * W + W); the patch step then works on the whole
+// tile.  `stage` is the warp's STAGE_WORDS words of shared scratch.  WAIT_BULK: lane 0 first waits for its pending bulk copy out of
 // `region`, just before the region is overwritten.  Ends with the warp synchronised.
 template <int N_OUT, int N_IN, bool WAIT_BULK = false>
 SQNN_DEV void tile_decode(const DecodeArgs &A, const PlanePtrs &P, const TileIn<N_OUT, N_IN> &in,
@@ -368,19 +376,17 @@ SQNN_DEV void tile_decode(const DecodeArgs &A, const PlanePtrs &P, const TileIn<
 
     // patches (warp-uniform branch: `total` is the same in every lane)
     if (in.total != 0) {
-#pragma unroll
-        for (uint32_t j = 0; j < 4; ++j) stage[lane + 32 * j] = st[j];
-        __syncwarp();
+        __syncwarp();                                   // every lane's words are in place
         const uint32_t nb = lane * G * P.w_np, sh = nb & 31u;
         if (G * P.w_np <= 32) {
             const uint32_t win = __funnelshift_r(in.np0, in.np1, sh) &
                                  (G * P.w_np == 32 ? 0xffffffffu : (1u << (G * P.w_np)) - 1u);
-            patch_lane<G, uint32_t>(A, P, n_out, mine, stage, in.base, in.total, win, lane);
+            patch_tile<G, uint32_t>(A, P, n_out, region, stage, st, in.base, in.total, win, lane);
         } else {
             uint64_t win = (uint64_t)__funnelshift_r(in.np0, in.np1, sh) |
                            ((uint64_t)__funnelshift_r(in.np1, in.np2, sh) << 32);
             if (G * P.w_np < 64) win &= (1ull << (G * P.w_np)) - 1ull;
-            patch_lane<G, uint64_t>(A, P, n_out, mine, stage, in.base, in.total, win, lane);
+            patch_tile<G, uint64_t>(A, P, n_out, region, stage, st, in.base, in.total, win, lane);
         }
     }
     __syncwarp();
