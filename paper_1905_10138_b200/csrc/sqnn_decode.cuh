@@ -240,22 +240,25 @@ SQNN_DEV void stage_fetch(const DecodeArgs &A, const PlanePtrs &P, TileIn<N_OUT,
 // Flips the patched positions of a tile (Section 3.2), the warp working through the tile's run of
 // d_patch entries 32 at a time.  An entry does not say which slice it belongs to; that follows
 // from the n_patch counts.  Each lane knows where the entries of its own G slices start (a warp
-// scan of the per-lane counts), so it drops a mark "slice id + 1" at the index of each of its
-// slices' first entry; a running maximum over the marks then gives every entry its slice, and
-// the lane holding the entry flips bit slice * n_out + position of the tile with a shared-memory
-// atomic.  Runs longer than PATCH_WIN entries are handled in windows, the running maximum
-// carrying over.  `win` holds the lane's n_patch fields (G fields of w_np bits, lowest first),
+// scan of the per-lane counts), so it drops a mark (the slice's first bit + 1) at the index of each of its
+// slices' first entry; every entry then takes the nearest mark at or before it (a ballot and one
+// shuffle per 32 entries), and the lane holding the entry flips bit slice * n_out + position of
+// the tile with a shared-memory atomic.  Runs longer than PATCH_WIN entries are handled in
+// windows, the last mark carrying over.  `win` holds the lane's n_patch fields (G fields of w_np bits, lowest first),
 // `st` the first window's d_patch words fetched ahead of time.
-template <uint32_t G, typename WT>
-SQNN_DEV void patch_tile(const DecodeArgs &A, const PlanePtrs &P, uint32_t n_out, uint32_t *region,
-                         uint32_t *stage, const uint32_t (&st)[4], uint32_t base, uint32_t total, WT win,
-                         uint32_t lane)
+template <uint32_t G, uint32_t N_OUT, typename WT>
+SQNN_DEV void patch_tile(const DecodeArgs &A, const PlanePtrs &P, uint32_t *region, uint32_t *stage,
+                         const uint32_t (&st)[4], uint32_t base, uint32_t total, WT win, uint32_t lane)
 {
     const uint32_t w_np = P.w_np;
     const uint32_t fm = (1u << w_np) - 1u;
+    uint32_t f[G];
     uint32_t cnt = 0;
 #pragma unroll
-    for (uint32_t i = 0; i < G; ++i) cnt += (uint32_t)(win >> (i * w_np)) & fm;
+    for (uint32_t i = 0; i < G; ++i) {
+        f[i] = (uint32_t)(win >> (i * w_np)) & fm;
+        cnt += f[i];
+    }
     uint32_t incl = cnt;
 #pragma unroll
     for (uint32_t d = 1; d < 32; d <<= 1) {
@@ -269,6 +272,7 @@ SQNN_DEV void patch_tile(const DecodeArgs &A, const PlanePtrs &P, uint32_t n_out
     }
     uint32_t *marks32 = stage + STAGE_DP_WORDS;
     uint16_t *marks = reinterpret_cast<uint16_t *>(marks32);
+    const uint32_t below_me = 0xffffffffu >> (31 - lane);   // lanes 0 .. lane
     uint32_t carry = 0, bad = 0;
     for (uint32_t w0 = 0; w0 < total; w0 += PATCH_WIN) {
         const uint32_t wn = total - w0 < PATCH_WIN ? total - w0 : PATCH_WIN;
@@ -283,35 +287,33 @@ SQNN_DEV void patch_tile(const DecodeArgs &A, const PlanePtrs &P, uint32_t n_out
             for (uint32_t j = 0; j < 4; ++j)
                 if (lane + 32 * j < nwords) stage[lane + 32 * j] = __ldg(src + lane + 32 * j);
         }
-        for (uint32_t q = lane; q < (wn + 1) / 2; q += 32) marks32[q] = 0;
+        // marks of whole 32-entry groups are cleared, so the last group reads zeros past wn
+        for (uint32_t q = lane; q < ((wn + 31) >> 5) * 16; q += 32) marks32[q] = 0;
         __syncwarp();
-        uint32_t run = first;
+        // mark = first tile bit of the slice + 1, dropped at the slice's first entry
+        uint32_t run = first - w0;
 #pragma unroll
         for (uint32_t i = 0; i < G; ++i) {
-            const uint32_t npi = (uint32_t)(win >> (i * w_np)) & fm;
-            if (npi != 0 && run - w0 < wn) marks[run - w0] = (uint16_t)(lane * G + i + 1);
-            run += npi;
+            if (f[i] != 0 && run < wn) marks[run] = (uint16_t)((lane * G + i) * N_OUT + 1);
+            run += f[i];
         }
         __syncwarp();
         const uint8_t *bytes = reinterpret_cast<const uint8_t *>(stage) + ob;
         for (uint32_t e0 = 0; e0 < wn; e0 += 32) {
             const uint32_t e = e0 + lane;
-            uint32_t v = e < wn ? marks[e] : 0u;
-#pragma unroll
-            for (uint32_t d = 1; d < 32; d <<= 1) {
-                const uint32_t o = __shfl_up_sync(0xffffffffu, v, d);
-                if (lane >= d) v = v > o ? v : o;
-            }
-            v = v > carry ? v : carry;
+            uint32_t v = marks[e];
+            // every entry takes the nearest mark at or before it (in this group, else the carry)
+            const uint32_t starts = __ballot_sync(0xffffffffu, v != 0) & below_me;
+            const uint32_t got = __shfl_sync(0xffffffffu, v, (31 - __clz((int)starts)) & 31);
+            v = starts ? got : carry;
             carry = __shfl_sync(0xffffffffu, v, 31);
-            if (e < wn) {
-                const uint32_t pos = bytes[e];
-                if (v == 0 || pos >= n_out) {
-                    bad = 1;
-                } else {
-                    const uint32_t bit = (v - 1) * n_out + pos;
-                    atomicXor(region + (bit >> 5), 1u << (bit & 31));
-                }
+            const uint32_t pos = bytes[e];
+            const bool live = e < wn;
+            const bool ok = live && v != 0 && pos < N_OUT;
+            bad |= (uint32_t)(live && !ok);
+            if (ok) {
+                const uint32_t bit = v - 1 + pos;
+                atomicXor(region + (bit >> 5), 1u << (bit & 31));
             }
         }
         __syncwarp();
@@ -381,12 +383,12 @@ SQNN_DEV void tile_decode(const DecodeArgs &A, const PlanePtrs &P, const TileIn<
         if (G * P.w_np <= 32) {
             const uint32_t win = __funnelshift_r(in.np0, in.np1, sh) &
                                  (G * P.w_np == 32 ? 0xffffffffu : (1u << (G * P.w_np)) - 1u);
-            patch_tile<G, uint32_t>(A, P, n_out, region, stage, st, in.base, in.total, win, lane);
+            patch_tile<G, n_out, uint32_t>(A, P, region, stage, st, in.base, in.total, win, lane);
         } else {
             uint64_t win = (uint64_t)__funnelshift_r(in.np0, in.np1, sh) |
                            ((uint64_t)__funnelshift_r(in.np1, in.np2, sh) << 32);
             if (G * P.w_np < 64) win &= (1ull << (G * P.w_np)) - 1ull;
-            patch_tile<G, uint64_t>(A, P, n_out, region, stage, st, in.base, in.total, win, lane);
+            patch_tile<G, n_out, uint64_t>(A, P, region, stage, st, in.base, in.total, win, lane);
         }
     }
     __syncwarp();

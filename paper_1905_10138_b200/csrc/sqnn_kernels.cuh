@@ -111,11 +111,36 @@ k_decode_bits(DecodeArgs A, uint64_t *__restrict__ out)
     }
 }
 
+SQNN_DEV void cp_async16(void *sdst, const void *gsrc)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" :: "r"(smem_addr(sdst)), "l"(gsrc) : "memory");
+}
+SQNN_DEV void cp_async_wait_all() { asm volatile("cp.async.wait_all;\n" ::: "memory"); }
+
+// Starts the copy of a tile's 32 * W mask words (first word gw0) into shared memory: 16-byte
+// asynchronous copies where a whole vector is in range, plain loads (zero past the end) otherwise.
+// Finish with cp_async_wait_all() and a warp barrier.
+SQNN_DEV void stage_mask_tile(uint32_t *mask_s, const uint32_t *__restrict__ mask32, uint64_t gw0,
+                              uint64_t mask_words, uint32_t W, uint32_t lane, bool vec_ok)
+{
+    for (uint32_t v = lane; v < 8 * W; v += 32) {
+        if (vec_ok && gw0 + 4 * v + 4 <= mask_words) {
+            cp_async16(mask_s + 4 * v, mask32 + gw0 + 4 * v);
+        } else {
+#pragma unroll
+            for (uint32_t e = 0; e < 4; ++e)
+                mask_s[4 * v + e] = gw0 + 4 * v + e < mask_words ? __ldg(mask32 + gw0 + 4 * v + e) : 0u;
+        }
+    }
+}
+
 // K2: decoded, masked, rescaled weights as bf16.  Lane j of an iteration writes the 8 weights
 // of byte j of a 32-byte group of the tile's bit run, so a warp stores 512 contiguous bytes.
-template <int N_OUT, int N_IN>
+// The tile's mask words arrive by cp.async while the tile is decoded; a lane keeps the scales
+// of the row it is in.  NQ = number of planes when it is 1, 2 or 3, 0 = any.
+template <int N_OUT, int N_IN, int NQ>
 __global__ void __launch_bounds__(256)
-k_decode_bf16(DecodeArgs A, const uint8_t *__restrict__ mask8, const float *__restrict__ alpha,
+k_decode_bf16(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__restrict__ alpha,
               uint64_t n, __nv_bfloat16 *__restrict__ out)
 {
     extern __shared__ __align__(16) uint32_t smem[];
@@ -123,49 +148,75 @@ k_decode_bf16(DecodeArgs A, const uint8_t *__restrict__ mask8, const float *__re
     const uint32_t W = words_per_lane<N_OUT>(A);
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     const uint32_t n_q = A.n_q;
-    const uint32_t per_warp = n_q * 32 * W + STAGE_WORDS;
+    const uint32_t per_warp = (n_q + 1) * 32 * W + STAGE_WORDS;
     uint32_t *region = smem + table_words(A.n_in, A.nwp, A.nchunks, A.cb) + warp * per_warp;
-    uint32_t *stage = region + n_q * 32 * W;
+    uint32_t *mask_s = region + n_q * 32 * W;
+    uint32_t *stage = mask_s + 32 * W;
+    const uint8_t *mask_s8 = reinterpret_cast<const uint8_t *>(mask_s);
     const uint32_t tile_bytes = 128 * W;                 // bytes of bits per tile and plane
+    const uint64_t mask_words = A.words64 * 2;
+    const bool mask_vec = (reinterpret_cast<uintptr_t>(mask32) & 15) == 0;
+    constexpr int NR = NQ > 0 ? NQ : 1;
     for (uint64_t tile = (uint64_t)blockIdx.x * nwarps + warp; tile < A.tiles; tile += (uint64_t)gridDim.x * nwarps) {
         const uint64_t p_tile = tile * (uint64_t)tile_bytes * 8;
         if (p_tile >= A.mn) continue;
+        stage_mask_tile(mask_s, mask32, tile * 32 * W, mask_words, W, lane, mask_vec);
         for (uint32_t i = 0; i < n_q; ++i)
             decode_warp_tile<N_OUT, N_IN>(A, i, tile, region + i * 32 * W, smem, stage, lane);
+        cp_async_wait_all();
         __syncwarp();
         uint64_t p = p_tile + 8ull * lane;               // first weight of this lane's group
         uint64_t r = p / n;
         uint64_t c = p - r * n;
+        float al[NR];
+        uint64_t r_al = ~0ull;
         for (uint32_t t = lane; t < tile_bytes; t += 32, p += 256, c += 256) {
             if (p >= A.mn) break;
             while (c >= n) { c -= n; ++r; }
-            const uint32_t mk = mask8[p >> 3];
-            uint32_t bits[8];
+            const uint32_t mk = mask_s8[t];
+            if (NQ > 0 && c + 8 <= n && p + 8 <= A.mn) {
+                if (r != r_al) {
 #pragma unroll
-            for (uint32_t i = 0; i < 8; ++i)
-                bits[i] = i < n_q ? reinterpret_cast<const uint8_t *>(region + i * 32 * W)[t] : 0u;
-            __align__(16) __nv_bfloat16 v[8];
-            uint64_t rr = r, cc = c;
+                    for (int i = 0; i < NR; ++i) al[i] = __ldg(alpha + r * n_q + i);
+                    r_al = r;
+                }
+                uint32_t bits[NR];
 #pragma unroll
-            for (uint32_t k = 0; k < 8; ++k) {
-                if (cc >= n) { cc -= n; ++rr; }
-                float s = 0.0f;
-                if ((mk >> k) & 1u) {
+                for (int i = 0; i < NR; ++i) bits[i] = reinterpret_cast<const uint8_t *>(region + i * 32 * W)[t];
+                uint32_t w[4];
 #pragma unroll
-                    for (uint32_t i = 0; i < 8; ++i) {
-                        if (i < n_q) {
+                for (uint32_t h = 0; h < 4; ++h) {
+                    float two[2];
+#pragma unroll
+                    for (uint32_t e = 0; e < 2; ++e) {
+                        const uint32_t k = 2 * h + e;
+                        float s = 0.0f;
+#pragma unroll
+                        for (int i = 0; i < NR; ++i) {
+                            const float term = ((bits[i] >> k) & 1u) ? al[i] : -al[i];
+                            s = i == 0 ? term : __fadd_rn(s, term);
+                        }
+                        two[e] = ((mk >> k) & 1u) ? s : 0.0f;
+                    }
+                    const __nv_bfloat162 pk = __floats2bfloat162_rn(two[0], two[1]);
+                    w[h] = *reinterpret_cast<const uint32_t *>(&pk);
+                }
+                *reinterpret_cast<uint4 *>(out + p) = make_uint4(w[0], w[1], w[2], w[3]);
+            } else {
+                uint64_t rr = r, cc = c;
+                for (uint32_t k = 0; k < 8 && p + k < A.mn; ++k) {
+                    if (cc >= n) { cc -= n; ++rr; }
+                    float s = 0.0f;
+                    if ((mk >> k) & 1u) {
+                        for (uint32_t i = 0; i < n_q; ++i) {
                             const float a = __ldg(alpha + rr * n_q + i);
-                            s = __fadd_rn(s, ((bits[i] >> k) & 1u) ? a : -a);
+                            const uint32_t bi = reinterpret_cast<const uint8_t *>(region + i * 32 * W)[t];
+                            s = __fadd_rn(s, ((bi >> k) & 1u) ? a : -a);
                         }
                     }
+                    out[p + k] = __float2bfloat16_rn(s);
+                    ++cc;
                 }
-                v[k] = __float2bfloat16_rn(s);
-                ++cc;
-            }
-            if (p + 8 <= A.mn) {
-                *reinterpret_cast<uint4 *>(out + p) = *reinterpret_cast<const uint4 *>(v);
-            } else {
-                for (uint32_t k = 0; k < 8 && p + k < A.mn; ++k) out[p + k] = v[k];
             }
         }
         __syncwarp();
@@ -184,12 +235,6 @@ SQNN_DEV void load_x(const XT *p, float (&v)[BT])
 #pragma unroll
     for (int q = 0; q < BT; ++q) v[q] = to_float(pk.e[q]);
 }
-
-SQNN_DEV void cp_async16(void *sdst, const void *gsrc)
-{
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" :: "r"(smem_addr(sdst)), "l"(gsrc) : "memory");
-}
-SQNN_DEV void cp_async_wait_all() { asm volatile("cp.async.wait_all;\n" ::: "memory"); }
 
 // Words of per-warp scratch the GEMV kernel keeps for the scales of the rows a tile touches.
 constexpr uint32_t GEMV_ALPHA_WORDS = 64;
@@ -251,16 +296,7 @@ k_decode_gemv(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__
             const uint64_t P0 = gw0 * 32;
             if (P0 >= A.mn) continue;
             const uint64_t P1 = (P0 + 1024ull * W < A.mn) ? P0 + 1024ull * W : A.mn;
-            // the tile's mask words: asynchronous 16-byte copies where whole vectors are in range
-            for (uint32_t v = lane; v < 8 * W; v += 32) {
-                if (mask_vec && gw0 + 4 * v + 4 <= mask_words) {
-                    cp_async16(mask_s + 4 * v, mask32 + gw0 + 4 * v);
-                } else {
-#pragma unroll
-                    for (uint32_t e = 0; e < 4; ++e)
-                        mask_s[4 * v + e] = gw0 + 4 * v + e < mask_words ? __ldg(mask32 + gw0 + 4 * v + e) : 0u;
-                }
-            }
+            stage_mask_tile(mask_s, mask32, gw0, mask_words, W, lane, mask_vec);
             // scales of the first rows the tile touches (later rows are fetched when reached)
             const uint64_t r_first = P0 / n;
             for (uint32_t i = lane; i < GEMV_ALPHA_WORDS; i += 32) {
@@ -393,12 +429,21 @@ inline int launch_decode(const DecodeArgs &A, sqnn_out_mode mode, const uint64_t
             k<<<grid, warps * 32, smem, st>>>(A, (uint64_t *)d_out);
         }
     } else {
-        const uint32_t warps = pick_warps(A, A.n_q, 0, &smem);
+        const uint32_t warps = pick_warps(A, A.n_q + 1, 0, &smem);
         if (!warps) return SQNN_E_UNSUPPORTED;
-        const uint32_t grid = grid_for(A.tiles, warps, 4);
-        auto k = k_decode_bf16<N_OUT, N_IN>;
-        if (prepare(k, smem)) return SQNN_E_CUDA;
-        k<<<grid, warps * 32, smem, st>>>(A, (const uint8_t *)d_mask, d_alpha, n, (__nv_bfloat16 *)d_out);
+        const uint64_t live = (A.words64 * 2 + 32ull * A.W - 1) / (32ull * A.W);
+        const uint32_t grid = grid_for(live, warps, 4);
+#define SQNN_BF16_LAUNCH(NQV)                                                                            \
+    do {                                                                                                 \
+        auto k = k_decode_bf16<N_OUT, N_IN, NQV>;                                                        \
+        if (prepare(k, smem)) return SQNN_E_CUDA;                                                        \
+        k<<<grid, warps * 32, smem, st>>>(A, (const uint32_t *)d_mask, d_alpha, n, (__nv_bfloat16 *)d_out); \
+    } while (0)
+        if (A.n_q == 1) SQNN_BF16_LAUNCH(1);
+        else if (A.n_q == 2) SQNN_BF16_LAUNCH(2);
+        else if (A.n_q == 3) SQNN_BF16_LAUNCH(3);
+        else SQNN_BF16_LAUNCH(0);
+#undef SQNN_BF16_LAUNCH
     }
     return cudaGetLastError() == cudaSuccess ? SQNN_OK : SQNN_E_CUDA;
 }
