@@ -299,6 +299,12 @@ def decode_point(torch, sqnn, wl, i_s, i_m, flush, peaks, steps, warm, m=32768, 
     sink = torch.zeros(2, dtype=torch.int64, device="cuda")
     ts = time_steps(torch, lambda: sqnn.sqnn_decode(desc, d_blob, None, None, sqnn.OUT_SINK, sink, status),
                     steps, warm, flush)
+    # context for the roofline: this kernel writes 5.5 x what it reads, and a write-only stream
+    # (a plain fill of 1 GiB) runs well below the copy peak on this part
+    big = torch.empty(1 << 30, dtype=torch.uint8, device="cuda")
+    tf = time_steps(torch, lambda: big.fill_(1), 5, 3, lambda: None)
+    write_only_gbs = (1 << 30) / (float(np.median(tf)) * 1e-3) / 1e9
+    del big
     sec = float(np.median(t)) * 1e-3
     in_bytes = stream_bytes(stats, layer, False)
     alg = in_bytes + layer.mn / 8
@@ -306,7 +312,9 @@ def decode_point(torch, sqnn, wl, i_s, i_m, flush, peaks, steps, warm, m=32768, 
             "compressed_stream_gbs": in_bytes / sec / 1e9,
             "roofline": {"bound": "hbm", "achieved": alg / sec / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                          "frac": alg / sec / 1e9 / peaks["hbm_gbs"], "traffic": None, "kernel": "k_decode_bits",
-                         "algorithmic_bytes": alg, "peaks": peaks["source"]},
+                         "algorithmic_bytes": alg, "peaks": peaks["source"],
+                         "write_only_fill_gbs": write_only_gbs,
+                         "frac_of_write_only_fill": alg / sec / 1e9 / write_only_gbs},
             "sink_us": float(np.median(ts)) * 1e3, "sink_stream_gbs": in_bytes / (float(np.median(ts)) * 1e-3) / 1e9,
             "bits_per_weight_eq1": stats["bpw_eq1"], "bits_per_weight_stored": stats["bpw_actual"],
             "status": int(status.item())}

@@ -287,8 +287,8 @@ SQNN_DEV void patch_tile(const DecodeArgs &A, const PlanePtrs &P, uint32_t *regi
             for (uint32_t j = 0; j < 4; ++j)
                 if (lane + 32 * j < nwords) stage[lane + 32 * j] = __ldg(src + lane + 32 * j);
         }
-        // marks of whole 32-entry groups are cleared, so the last group reads zeros past wn
-        for (uint32_t q = lane; q < ((wn + 31) >> 5) * 16; q += 32) marks32[q] = 0;
+        // marks of whole 64-entry groups are cleared, so the last group reads zeros past wn
+        for (uint32_t q = lane; q < ((wn + 63) >> 6) * 32; q += 32) marks32[q] = 0;
         __syncwarp();
         // mark = first tile bit of the slice + 1, dropped at the slice's first entry
         uint32_t run = first - w0;
@@ -299,20 +299,29 @@ SQNN_DEV void patch_tile(const DecodeArgs &A, const PlanePtrs &P, uint32_t *regi
         }
         __syncwarp();
         const uint8_t *bytes = reinterpret_cast<const uint8_t *>(stage) + ob;
-        for (uint32_t e0 = 0; e0 < wn; e0 += 32) {
-            const uint32_t e = e0 + lane;
-            uint32_t v = marks[e];
-            // every entry takes the nearest mark at or before it (in this group, else the carry)
-            const uint32_t starts = __ballot_sync(0xffffffffu, v != 0) & below_me;
-            const uint32_t got = __shfl_sync(0xffffffffu, v, (31 - __clz((int)starts)) & 31);
-            v = starts ? got : carry;
-            carry = __shfl_sync(0xffffffffu, v, 31);
-            const uint32_t pos = bytes[e];
-            const bool live = e < wn;
-            const bool ok = live && v != 0 && pos < N_OUT;
-            bad |= (uint32_t)(live && !ok);
-            if (ok) {
-                const uint32_t bit = v - 1 + pos;
+        // two groups of 32 entries per round (two independent chains of shared-memory reads and
+        // shuffles); every entry takes the nearest mark at or before it, else the carry
+        for (uint32_t e0 = 0; e0 < wn; e0 += 64) {
+            const uint32_t ea = e0 + lane, eb = ea + 32;
+            uint32_t va = marks[ea], vb = marks[eb];
+            const uint32_t pa = bytes[ea], pb = bytes[eb];
+            const uint32_t sa = __ballot_sync(0xffffffffu, va != 0) & below_me;
+            const uint32_t sb = __ballot_sync(0xffffffffu, vb != 0) & below_me;
+            const uint32_t ga = __shfl_sync(0xffffffffu, va, (31 - __clz((int)sa)) & 31);
+            const uint32_t gb = __shfl_sync(0xffffffffu, vb, (31 - __clz((int)sb)) & 31);
+            va = sa ? ga : carry;
+            const uint32_t ca = __shfl_sync(0xffffffffu, va, 31);
+            vb = sb ? gb : ca;
+            carry = __shfl_sync(0xffffffffu, vb, 31);
+            const bool la = ea < wn, lb = eb < wn;
+            const bool oka = la && va != 0 && pa < N_OUT, okb = lb && vb != 0 && pb < N_OUT;
+            bad |= (uint32_t)((la && !oka) || (lb && !okb));
+            if (oka) {
+                const uint32_t bit = va - 1 + pa;
+                atomicXor(region + (bit >> 5), 1u << (bit & 31));
+            }
+            if (okb) {
+                const uint32_t bit = vb - 1 + pb;
                 atomicXor(region + (bit >> 5), 1u << (bit & 31));
             }
         }

@@ -35,7 +35,7 @@ SQNN_DEV uint32_t words_per_lane(const DecodeArgs &A)
 // is expanded.  SINK = true: XOR of all those words instead of
 // storing them.
 template <int N_OUT, int N_IN, bool SINK>
-__global__ void __launch_bounds__(256, 4)
+__global__ void __launch_bounds__(512, 2)
 k_decode_bits(DecodeArgs A, uint64_t *__restrict__ out)
 {
     extern __shared__ __align__(16) uint32_t smem[];
@@ -46,10 +46,14 @@ k_decode_bits(DecodeArgs A, uint64_t *__restrict__ out)
     uint32_t *mybase = smem + table_words(A.n_in, A.nwp, A.nchunks, A.cb) + warp * per_warp;
     uint32_t *stage = mybase + 32 * W;
     const uint64_t tail_bits = A.mn & 63;
-    // tiles that hold at least one real word, per plane; (plane, tile) advance without division
-    const uint64_t live = (A.words64 + 16 * W - 1) / (16 * W);
-    const uint64_t stride = (uint64_t)gridDim.x * nwarps;
-    uint64_t tile = (uint64_t)blockIdx.x * nwarps + warp;
+    // tiles that hold at least one real word, per plane (the launcher keeps the count below 2^31);
+    // (plane, tile) advance without division
+    const uint32_t live = (uint32_t)((A.words64 + 16 * W - 1) / (16 * W));
+    // tiles before this one lie wholly inside the plane and end on a whole word
+    const uint32_t full_tiles = (uint32_t)(A.words64 / (16 * W)) -
+                                ((tail_bits != 0 && A.words64 % (16 * W) == 0) ? 1u : 0u);
+    const uint32_t stride = gridDim.x * nwarps;
+    uint32_t tile = blockIdx.x * nwarps + warp;
     uint32_t plane = 0;
     while (plane < A.n_q && tile >= live) { tile -= live; ++plane; }
     uint64_t sink = 0;
@@ -57,7 +61,7 @@ k_decode_bits(DecodeArgs A, uint64_t *__restrict__ out)
         TileIn<N_OUT, N_IN> cur, nxt;
         if (plane < A.n_q) tile_fetch<N_OUT, N_IN>(A.pl[plane], tile, lane, cur);
         while (plane < A.n_q) {
-            uint64_t ntile = tile + stride;
+            uint32_t ntile = tile + stride;
             uint32_t nplane = plane;
             while (nplane < A.n_q && ntile >= live) { ntile -= live; ++nplane; }
             if (nplane < A.n_q) tile_fetch<N_OUT, N_IN>(A.pl[nplane], ntile, lane, nxt);
@@ -65,10 +69,10 @@ k_decode_bits(DecodeArgs A, uint64_t *__restrict__ out)
             stage_fetch<N_OUT, N_IN>(A, A.pl[plane], cur, lane, st);
             uint32_t *region = mybase;
             tile_decode<N_OUT, N_IN, !SINK>(A, A.pl[plane], cur, st, region, smem, stage, lane);
-            const uint64_t q0 = tile * 16 * W;           // first uint64 of the tile inside the plane
-            uint64_t *dst = out + (uint64_t)plane * A.words64 + q0;
-            const bool whole = q0 + 16 * W < A.words64 || (q0 + 16 * W == A.words64 && tail_bits == 0);
-            if (!SINK && whole && (reinterpret_cast<uintptr_t>(dst) & 15) == 0) {
+            uint64_t *pbase = out + (uint64_t)plane * A.words64;
+            const uint64_t q0 = (uint64_t)tile * (16 * W);   // first uint64 of the tile inside the plane
+            uint64_t *dst = pbase + q0;
+            if (!SINK && tile < full_tiles && (reinterpret_cast<uintptr_t>(pbase) & 15) == 0) {
                 fence_async_smem();
                 __syncwarp();
                 if (lane == 0) bulk_store(dst, region, 128 * W);
@@ -89,7 +93,7 @@ k_decode_bits(DecodeArgs A, uint64_t *__restrict__ out)
         while (plane < A.n_q) {
             uint32_t *region = mybase;
             decode_warp_tile<0, 0>(A, plane, tile, region, smem, stage, lane);
-            const uint64_t q0 = tile * 16 * W;
+            const uint64_t q0 = (uint64_t)tile * (16 * W);
             uint64_t *dst = out + (uint64_t)plane * A.words64 + q0;
             for (uint32_t q = lane; q < 16 * W; q += 32) {
                 if (q0 + q >= A.words64) break;
@@ -249,23 +253,26 @@ constexpr uint32_t GEMV_ALPHA_WORDS = 64;
 // activations of the current batch chunk sit in shared memory as xs[c][BT].
 // NQ = number of planes when it is 1, 2 or 3 (scales and plane words stay in registers), 0 = any.
 template <int N_OUT, int N_IN, int BT, typename XT, bool XS, int NQ>
-__global__ void __launch_bounds__(512)
+__global__ void __launch_bounds__(640)
 k_decode_gemv(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__restrict__ alpha,
               const XT *__restrict__ x, int64_t ldx, uint32_t batch, float *__restrict__ y,
-              int64_t ldy, uint32_t n)
+              int64_t ldy, uint32_t n, uint32_t wpt)
 {
     extern __shared__ __align__(16) uint32_t smem[];
     build_tables(A, smem);
     const uint32_t W = words_per_lane<N_OUT>(A);
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     const uint32_t n_q = A.n_q;
-    const uint32_t per_warp = (n_q + 1) * 32 * W + STAGE_WORDS + GEMV_ALPHA_WORDS;
+    // `wpt` warps form a group that shares one tile: the planes (and the mask / scale staging)
+    // are dealt out over the group's warps, then all of them walk the tile's words
+    const uint32_t group = warp / wpt, sub = warp - group * wpt, ngroups = nwarps / wpt;
+    const uint32_t per_group = (n_q + 1) * 32 * W + GEMV_ALPHA_WORDS;
     uint32_t *warp0 = smem + table_words(A.n_in, A.nwp, A.nchunks, A.cb);
-    uint32_t *region = warp0 + warp * per_warp;
+    uint32_t *region = warp0 + group * per_group;
     uint32_t *mask_s = region + n_q * 32 * W;
-    uint32_t *stage = mask_s + 32 * W;
-    float *alpha_s = reinterpret_cast<float *>(stage + STAGE_WORDS);
-    XT *xs = reinterpret_cast<XT *>(warp0 + nwarps * per_warp);
+    float *alpha_s = reinterpret_cast<float *>(mask_s + 32 * W);
+    uint32_t *stage = warp0 + ngroups * per_group + warp * STAGE_WORDS;
+    XT *xs = reinterpret_cast<XT *>(warp0 + ngroups * per_group + nwarps * STAGE_WORDS);
     const uint64_t mask_words = A.words64 * 2;
     const uint64_t alpha_count = (A.mn / n) * n_q;
     const bool mask_vec = (reinterpret_cast<uintptr_t>(mask32) & 15) == 0;
@@ -291,22 +298,25 @@ k_decode_gemv(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__
             }
             __syncthreads();
         }
-        for (uint64_t tile = (uint64_t)blockIdx.x * nwarps + warp; tile < A.tiles; tile += (uint64_t)gridDim.x * nwarps) {
+        for (uint64_t tile = (uint64_t)blockIdx.x * ngroups + group; tile < A.tiles; tile += (uint64_t)gridDim.x * ngroups) {
             const uint64_t gw0 = tile * 32 * W;          // first 32-bit word of the tile
             const uint64_t P0 = gw0 * 32;
             if (P0 >= A.mn) continue;
             const uint64_t P1 = (P0 + 1024ull * W < A.mn) ? P0 + 1024ull * W : A.mn;
-            stage_mask_tile(mask_s, mask32, gw0, mask_words, W, lane, mask_vec);
-            // scales of the first rows the tile touches (later rows are fetched when reached)
             const uint64_t r_first = P0 / n;
-            for (uint32_t i = lane; i < GEMV_ALPHA_WORDS; i += 32) {
-                const uint64_t at = r_first * n_q + i;
-                alpha_s[i] = at < alpha_count ? __ldg(alpha + at) : 0.0f;
+            if (sub == n_q % wpt) {
+                stage_mask_tile(mask_s, mask32, gw0, mask_words, W, lane, mask_vec);
+                // scales of the first rows the tile touches (later rows are fetched when reached)
+                for (uint32_t i = lane; i < GEMV_ALPHA_WORDS; i += 32) {
+                    const uint64_t at = r_first * n_q + i;
+                    alpha_s[i] = at < alpha_count ? __ldg(alpha + at) : 0.0f;
+                }
             }
-            for (uint32_t i = 0; i < n_q; ++i)
+            for (uint32_t i = sub; i < n_q; i += wpt)
                 decode_warp_tile<N_OUT, N_IN>(A, i, tile, region + i * 32 * W, smem, stage, lane);
             cp_async_wait_all();
-            __syncwarp();
+            if (wpt == 1) __syncwarp();
+            else asm volatile("bar.sync %0, %1;\n" :: "r"(1 + group), "r"(32 * wpt) : "memory");
             for (uint64_t r = r_first; r * n < P1; ++r) {
                 const uint64_t a = r * n > P0 ? r * n : P0;
                 const uint64_t b = (r + 1) * n < P1 ? (r + 1) * n : P1;
@@ -324,7 +334,7 @@ k_decode_gemv(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__
                 float acc[BT];
 #pragma unroll
                 for (int q = 0; q < BT; ++q) acc[q] = 0.0f;
-                for (uint32_t lw = lw_lo + lane; lw <= lw_hi; lw += 32) {
+                for (uint32_t lw = lw_lo + sub * 32 + lane; lw <= lw_hi; lw += 32 * wpt) {
                     uint32_t mk = mask_s[lw];
                     const uint32_t lo = lw * 32;
                     if (lo < a_loc) mk &= 0xffffffffu << (a_loc - lo);
@@ -372,7 +382,8 @@ k_decode_gemv(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__
                     if (lane == 0 && bc + q < batch) atomicAdd(y + (int64_t)(bc + q) * ldy + r, s);
                 }
             }
-            __syncwarp();
+            if (wpt == 1) __syncwarp();                  // the group is done with its regions
+            else asm volatile("bar.sync %0, %1;\n" :: "r"(1 + group), "r"(32 * wpt) : "memory");
         }
     }
 }
@@ -382,11 +393,10 @@ k_decode_gemv(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__
 // ------------------------------------------------------------------------------------------
 // Picks warps per block so the dynamic shared memory fits; returns 0 if not even one warp fits.
 inline uint32_t pick_warps(const DecodeArgs &A, uint32_t regions, size_t extra, size_t *smem_bytes,
-                           uint32_t extra_warp_words = 0, uint32_t max_warps = 8)
+                           uint32_t extra_warp_words = 0, uint32_t max_warps = 8, size_t limit = 200 * 1024)
 {
     const size_t tab = (size_t)table_words(A.n_in, A.nwp, A.nchunks, A.cb) * 4;
     const size_t per_warp = ((size_t)regions * 32 * A.W + STAGE_WORDS + extra_warp_words) * 4;
-    const size_t limit = 200 * 1024;
     if (tab + per_warp + extra > limit) return 0;
     uint32_t warps = (uint32_t)((limit - tab - extra) / per_warp);
     if (warps > max_warps) warps = max_warps;
@@ -414,10 +424,12 @@ inline int launch_decode(const DecodeArgs &A, sqnn_out_mode mode, const uint64_t
 {
     size_t smem = 0;
     if (mode == SQNN_OUT_BITS || mode == SQNN_OUT_SINK) {
-        const uint32_t warps = pick_warps(A, 1, 0, &smem);
+        // half of the shared memory per block, so that two blocks of up to 16 warps share an SM
+        const uint32_t warps = pick_warps(A, 1, 0, &smem, 0, 16, 100 * 1024);
         if (!warps) return SQNN_E_UNSUPPORTED;
         const uint64_t live = (A.words64 + 16ull * A.W - 1) / (16ull * A.W);
-        const uint32_t grid = grid_for(live * A.n_q, warps, 4);
+        if (live * A.n_q >= (1ull << 31)) return SQNN_E_UNSUPPORTED;
+        const uint32_t grid = grid_for(live * A.n_q, warps, 2);
         if (mode == SQNN_OUT_BITS) {
             auto k = k_decode_bits<N_OUT, N_IN, false>;
             if (prepare(k, smem)) return SQNN_E_CUDA;
@@ -452,23 +464,34 @@ template <int N_OUT, int N_IN, int BT, typename XT>
 inline int launch_gemv_bt(const DecodeArgs &A, const uint64_t *d_mask, const float *d_alpha, const void *d_x,
                           int64_t ldx, uint32_t batch, float *d_y, int64_t ldy, uint64_t n, cudaStream_t st)
 {
-    // one tile per warp where the layer allows it: warps per block = live tiles / SMs, within [4, 16]
+    // Aim at ~32 warps per SM: with few tiles, up to 4 warps share a tile; a block holds up to
+    // 15 tile groups (named barriers) and 20 warps.
     const uint64_t live = (A.words64 * 2 + 32ull * A.W - 1) / (32ull * A.W);
-    uint32_t want = (uint32_t)((live + sm_count() - 1) / sm_count());
-    want = want < 4 ? 4 : want > 16 ? 16 : want;
-    size_t smem = 0;
+    const uint32_t sms = (uint32_t)sm_count();
+    uint32_t wpt = 1;
+    // (only while a row still gives every lane of the group at least two words)
+    while (wpt < 4 && live * wpt * 2 <= 32ull * sms && n >= 2048ull * wpt * 2) wpt *= 2;
+    uint32_t groups = (uint32_t)((live + sms - 1) / sms);
+    const uint32_t max_groups = 20 / wpt < 15 ? 20 / wpt : 15;
+    groups = groups < 1 ? 1 : groups > max_groups ? max_groups : groups;
+    if (wpt == 1 && groups < 4) groups = 4;
+    const size_t tab = (size_t)table_words(A.n_in, A.nwp, A.nchunks, A.cb) * 4;
+    const size_t per_group = ((size_t)(A.n_q + 1) * 32 * A.W + GEMV_ALPHA_WORDS + (size_t)wpt * STAGE_WORDS) * 4;
+    const size_t limit = 200 * 1024;
     const size_t xbytes = (size_t)n * BT * sizeof(XT);
-    uint32_t warps = xbytes <= 160 * 1024 ? pick_warps(A, A.n_q + 1, xbytes, &smem, GEMV_ALPHA_WORDS, want) : 0;
-    const bool xs = warps != 0;
-    if (!xs) warps = pick_warps(A, A.n_q + 1, 0, &smem, GEMV_ALPHA_WORDS, want);
-    if (!warps) return SQNN_E_UNSUPPORTED;
-    const uint32_t grid = grid_for(live, warps, 2);
+    bool xs = xbytes <= 160 * 1024 && tab + per_group + xbytes <= limit;
+    const size_t extra = xs ? xbytes : 0;
+    if (tab + per_group + extra > limit) return SQNN_E_UNSUPPORTED;
+    while (groups > 1 && tab + groups * per_group + extra > limit) --groups;
+    const size_t smem = tab + groups * per_group + extra;
+    const uint32_t warps = groups * wpt;
+    const uint32_t grid = grid_for(live, groups, 2);
 #define SQNN_GEMV_LAUNCH(XSV, NQV)                                                                           \
     do {                                                                                                     \
         auto k = k_decode_gemv<N_OUT, N_IN, BT, XT, XSV, NQV>;                                               \
         if (prepare(k, smem)) return SQNN_E_CUDA;                                                            \
         k<<<grid, warps * 32, smem, st>>>(A, (const uint32_t *)d_mask, d_alpha, (const XT *)d_x, ldx, batch, \
-                                           d_y, ldy, (uint32_t)n);                                           \
+                                           d_y, ldy, (uint32_t)n, wpt);                                      \
     } while (0)
     if (!xs) SQNN_GEMV_LAUNCH(false, 0);
     else if (A.n_q == 1) SQNN_GEMV_LAUNCH(true, 1);
