@@ -142,6 +142,21 @@ def time_steps(torch, fn, steps, warmup, flush):
     return [a.elapsed_time(b) for a, b in ev]          # ms
 
 
+def max_over_ranks(dist, value: float, device) -> float:
+    """Slowest rank's value (the job is as slow as its slowest replica); identity without a group."""
+    if dist is None:
+        return float(value)
+    import torch
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_rate(world: int, units_per_rank: float, slowest_ms_per_step: float) -> float:
+    """Replicas only: every rank processes `units_per_rank` per step, the job takes the slowest rank's time."""
+    return world * units_per_rank / (slowest_ms_per_step * 1e-3)
+
+
 def stream_bytes(stats, layer, with_mask):
     b = (stats["bits_wc"] + stats["bits_npatch"] + stats["bits_dpatch"] + stats["bits_index"]) / 8
     if with_mask:
@@ -200,25 +215,19 @@ def run_ours(args):
     clocks = sampler.stop()
     total_ms = float(sum(times))
     if dist:
-        t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
         dist.barrier()
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(dist, total_ms, "cuda")
     torch.cuda.synchronize()
     assert int(status.item()) == 0, "device status word set"
     units = layer.mn * layer.n_q
     ms_per_step = total_ms / args.steps
-    value = world * units / (ms_per_step * 1e-3)
+    value = whole_job_rate(world, units, ms_per_step)
 
     e2e_times = time_steps(torch, step_e2e, args.steps, args.warmup, flush)
-    e2e_ms = float(sum(e2e_times))
-    if dist:
-        t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = max_over_ranks(dist, float(sum(e2e_times)), "cuda")
     h2d = int(h_blob.numel() + h_mask.numel() * 8 + h_alpha.numel() * 4 + h_x.numel() * 2)
     d2h = int(h_y.numel() * 4)
-    e2e = {"value": world * units / (e2e_ms / args.steps * 1e-3), "unit": UNIT,
+    e2e = {"value": whole_job_rate(world, units, e2e_ms / args.steps), "unit": UNIT,
            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
 
     # roofline of the dominant kernel (fused decode-GEMV).  It is bound by plain ALU work: one
