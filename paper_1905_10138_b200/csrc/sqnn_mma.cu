@@ -14,8 +14,9 @@
 // Decoding runs in two phases per 256 columns.  Phase 1, one thread per (row, bit vector):
 // the thread walks the slices that cover its row segment (seed -> XOR tables -> patch flips)
 // and leaves the segment's bits, and the mask bits, in a small shared bit buffer.  Phase 2,
-// one thread per (row, 8 columns): bits -> bf16 values through a per-row table of the 2^n_q
-// sums (+-alpha_1) + (+-alpha_2) + ..., rounded to bf16, zero where the mask is 0.
+// one thread per (row, 32 columns): the thread clears its part of the stage and then writes only
+// the unpruned positions, each value taken from a per-row table of the 2^n_q sums
+// (+-alpha_1) + (+-alpha_2) + ..., rounded to bf16.
 //
 // Every wait on an mbarrier is bounded; a wait that gives up sets SQNN_E_TIMEOUT in the status
 // word and makes all roles leave their loops, so the kernel always returns.
@@ -33,10 +34,10 @@ namespace {
 
 constexpr uint32_t ROWS = 128;            // rows of W per CTA = MMA M
 constexpr uint32_t KC = 64;               // columns per pipeline step
-constexpr uint32_t MACRO = 256;           // columns decoded to bits at a time
+constexpr uint32_t MACRO = 512;           // columns decoded to bits at a time
 constexpr uint32_t STEPS_PER_MACRO = MACRO / KC;
 constexpr uint32_t RB_WORDS = MACRO / 32 + 1;   // words per row of the bit buffer (odd stride)
-constexpr uint32_t DEC_WARPS = 8;
+constexpr uint32_t DEC_WARPS = 16;
 constexpr uint32_t DEC_THREADS = DEC_WARPS * 32;
 constexpr uint32_t THREADS = DEC_THREADS + 64;  // + TMA warp + MMA warp
 constexpr uint32_t A_STAGE_BYTES = ROWS * KC * 2;
@@ -256,15 +257,6 @@ SQNN_DEV void copy_segment(const uint32_t *__restrict__ src, uint64_t valid_word
     row[RB_WORDS - 1] = 0;
 }
 
-// 8 bits -> one bit per nibble
-SQNN_DEV uint32_t spread8(uint32_t b)
-{
-    uint32_t x = (b | (b << 12)) & 0x000f000fu;
-    x = (x | (x << 6)) & 0x03030303u;
-    x = (x | (x << 3)) & 0x11111111u;
-    return x;
-}
-
 __global__ void __launch_bounds__(THREADS, 1)
 k_decode_mma(const __grid_constant__ CUtensorMap xmap, const MmaArgs M)
 {
@@ -339,13 +331,13 @@ k_decode_mma(const __grid_constant__ CUtensorMap xmap, const MmaArgs M)
 
         if (warp < DEC_WARPS) {
             // ------------------------------ decode warps ------------------------------
-            const uint32_t prow = tid & (ROWS - 1), phalf = tid >> 7;       // phase-1 role
+            const uint32_t prow = tid & (ROWS - 1), pq = tid >> 7;          // phase-1 role: row, item class
             const uint64_t r = r0 + prow;
             const bool live = r < M.m;
-            Cursor cur[4];
+            Cursor cur[3];
 #pragma unroll
-            for (uint32_t q = 0; q < 4; ++q) {
-                const uint32_t item = phalf + 2 * q;                         // plane index (mask = n_q)
+            for (uint32_t q = 0; q < 3; ++q) {
+                const uint32_t item = pq + 4 * q;                            // plane index (mask = n_q)
                 if (item < A.n_q && live && !M.bits32)
                     cur[q] = cursor_at(A.pl[item], A.n_out, r * M.n + (uint64_t)macro_begin * MACRO);
             }
@@ -355,8 +347,8 @@ k_decode_mma(const __grid_constant__ CUtensorMap xmap, const MmaArgs M)
                 const uint32_t cnt = (uint32_t)(M.n - c0 < MACRO ? M.n - c0 : MACRO);
                 // phase 1: bits of this thread's (row, item)s
 #pragma unroll
-                for (uint32_t q = 0; q < 5; ++q) {
-                    const uint32_t item = phalf + 2 * q;
+                for (uint32_t q = 0; q < 3; ++q) {
+                    const uint32_t item = pq + 4 * q;
                     if (item > A.n_q) break;
                     uint32_t *rowbuf = rb + (item * ROWS + prow) * RB_WORDS;
                     if (!live) {
@@ -366,8 +358,8 @@ k_decode_mma(const __grid_constant__ CUtensorMap xmap, const MmaArgs M)
                         if (M.bits32)
                             copy_segment(M.bits32 + (uint64_t)item * M.plane_words32, M.plane_words32,
                                          r * M.n + c0, cnt, rowbuf);
-                        else if (q < 4)
-                            decode_segment(A, A.pl[item], tab, cur[q < 4 ? q : 0], cnt, rowbuf);
+                        else
+                            decode_segment(A, A.pl[item], tab, cur[q], cnt, rowbuf);
                     } else {
                         copy_segment(M.mask32, M.mask_words32, r * M.n + c0, cnt, rowbuf);
                     }
@@ -379,55 +371,43 @@ k_decode_mma(const __grid_constant__ CUtensorMap xmap, const MmaArgs M)
                     const uint32_t stage = it % M.stages, use = it / M.stages;
                     if (use > 0 && !mbar_wait(empty + stage, (use - 1) & 1u, abort_flag, A.status)) break;
                     uint8_t *a_stage = a_stages + stage * A_STAGE_BYTES;
+                    {
+                        // one thread per (row, 16 columns): clear its 32 bytes of the stage, then
+                        // write only the unpruned weights (most positions are zero)
+                        const uint32_t row = tid >> 2, quarter = tid & 3;
+                        const uint32_t wi = ks * 2 + (quarter >> 1), sh16 = (quarter & 1) * 16;
+                        uint32_t mw = (rb[(A.n_q * ROWS + row) * RB_WORDS + wi] >> sh16) & 0xffffu;
+                        uint8_t *arow = a_stage + row * 128;
+                        const uint32_t sw = row & 7;
 #pragma unroll
-                    for (uint32_t q = 0; q < 4; ++q) {
-                        const uint32_t id = tid + DEC_THREADS * q;
-                        const uint32_t row = id >> 3, j = id & 7;
-                        const uint32_t byte = ks * 8 + j;
-                        const uint8_t *rb8 = reinterpret_cast<const uint8_t *>(rb);
-                        const uint32_t mb = rb8[((A.n_q * ROWS + row) * RB_WORDS) * 4 + byte];
-                        uint4 out;
+                        for (uint32_t q = 0; q < 2; ++q)
+                            *reinterpret_cast<uint4 *>(arow + (((quarter * 2 + q) ^ sw) << 4)) = make_uint4(0, 0, 0, 0);
                         if (A.n_q <= 3) {
-                            uint32_t c = spread8(mb) << 3;
+                            uint32_t bw[3];
 #pragma unroll
                             for (uint32_t i = 0; i < 3; ++i)
-                                if (i < A.n_q) c |= spread8(rb8[((i * ROWS + row) * RB_WORDS) * 4 + byte]) << i;
+                                bw[i] = i < A.n_q ? rb[(i * ROWS + row) * RB_WORDS + wi] >> sh16 : 0u;
                             const uint16_t *lr = reinterpret_cast<const uint16_t *>(lut) + row * 16;
-                            uint32_t w[4];
-#pragma unroll
-                            for (uint32_t h = 0; h < 4; ++h) {
-                                const uint32_t e0 = (c >> (8 * h)) & 15u, e1 = (c >> (8 * h + 4)) & 15u;
-                                w[h] = (uint32_t)lr[e0] | ((uint32_t)lr[e1] << 16);
+                            while (mw) {
+                                const uint32_t k = 31u - (uint32_t)__clz((int)mw);
+                                mw ^= 1u << k;
+                                const uint32_t e = 8u | ((bw[0] >> k) & 1u) | (((bw[1] >> k) & 1u) << 1) |
+                                                   (((bw[2] >> k) & 1u) << 2);
+                                *reinterpret_cast<uint16_t *>(arow + (((quarter * 2 + (k >> 3)) ^ sw) << 4) + (k & 7) * 2) = lr[e];
                             }
-                            out = make_uint4(w[0], w[1], w[2], w[3]);
                         } else {
-                            uint32_t pb[8];
-#pragma unroll
-                            for (uint32_t i = 0; i < 8; ++i)
-                                pb[i] = i < A.n_q ? rb8[((i * ROWS + row) * RB_WORDS) * 4 + byte] : 0u;
-                            uint32_t w[4];
-#pragma unroll
-                            for (uint32_t h = 0; h < 4; ++h) {
-                                uint32_t two = 0;
-#pragma unroll
-                                for (uint32_t e = 0; e < 2; ++e) {
-                                    const uint32_t k = 2 * h + e;
-                                    float s = 0.0f;
-                                    if ((mb >> k) & 1u) {
-#pragma unroll
-                                        for (uint32_t i = 0; i < 8; ++i)
-                                            if (i < A.n_q) {
-                                                const float a = alpha_s[row * 8 + i];
-                                                s = __fadd_rn(s, ((pb[i] >> k) & 1u) ? a : -a);
-                                            }
-                                    }
-                                    two |= (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(s)) << (16 * e);
+                            while (mw) {
+                                const uint32_t k = 31u - (uint32_t)__clz((int)mw);
+                                mw ^= 1u << k;
+                                float sum = 0.0f;
+                                for (uint32_t i = 0; i < A.n_q; ++i) {
+                                    const float a = alpha_s[row * 8 + i];
+                                    sum = __fadd_rn(sum, ((rb[(i * ROWS + row) * RB_WORDS + wi] >> (sh16 + k)) & 1u) ? a : -a);
                                 }
-                                w[h] = two;
+                                *reinterpret_cast<uint16_t *>(arow + (((quarter * 2 + (k >> 3)) ^ sw) << 4) + (k & 7) * 2) =
+                                    __bfloat16_as_ushort(__float2bfloat16_rn(sum));
                             }
-                            out = make_uint4(w[0], w[1], w[2], w[3]);
                         }
-                        *reinterpret_cast<uint4 *>(a_stage + row * 128 + ((j ^ (row & 7)) << 4)) = out;
                     }
                     fence_async_smem();                 // generic-proxy writes -> visible to the tensor core
                     mbar_arrive(full_a + stage);
@@ -483,10 +463,9 @@ k_decode_mma(const __grid_constant__ CUtensorMap xmap, const MmaArgs M)
             const bool ready = mbar_wait(accum, accum_parity, abort_flag, A.status);
             if (__all_sync(0xffffffffu, ready)) {                  // tcgen05.ld needs the whole warp
                 tc_fence_after();
-                const uint32_t quad = warp & 3, half = warp >> 2;
+                const uint32_t quad = warp & 3, part = warp >> 2;       // TMEM lane quarter, column class
                 const uint64_t r = r0 + quad * 32 + lane;
-                const uint32_t c_begin = half * (M.nbt / 2), c_end = c_begin + M.nbt / 2;
-                for (uint32_t c = c_begin; c < c_end; c += 8) {
+                for (uint32_t c = part * 8; c < M.nbt; c += 8 * (DEC_WARPS / 4)) {
                     uint32_t v[8];
                     tmem_ld8(tmem_base + ((quad * 32) << 16) + c, v);
                     if (r < M.m) {
