@@ -61,6 +61,10 @@ struct MmaArgs {
     uint32_t b_stage_bytes;
     const uint32_t *bits32;       // decoded planes in the workspace (NULL: decode in this kernel)
     uint64_t plane_words32;       // 32-bit words per plane in the workspace
+    uint32_t per_plane;           // 1: one sign tile and one accumulator per plane, scales in the epilogue
+    uint32_t tma_bits;            // 1: the bit buffer is filled by TMA (rows of the packed planes 16-byte aligned)
+    uint32_t rbp;                 // words per row of the bit buffer
+    uint32_t rb_bufs;             // bit buffers (2 with TMA)
 };
 
 // ---------------------------------------------------------------------------------------
@@ -99,7 +103,6 @@ SQNN_DEV bool mbar_wait(uint64_t *bar, uint32_t parity, volatile uint32_t *abort
             if (status) atomicMax(status, (uint32_t)(-SQNN_E_TIMEOUT));
             return false;
         }
-        __nanosleep(32);
     }
 }
 SQNN_DEV void tma_load_2d(void *sdst, const CUtensorMap *map, uint64_t *bar, int32_t x, int32_t y)
@@ -257,24 +260,37 @@ SQNN_DEV void copy_segment(const uint32_t *__restrict__ src, uint64_t valid_word
     row[RB_WORDS - 1] = 0;
 }
 
+SQNN_DEV void tma_load_3d(void *sdst, const CUtensorMap *map, uint64_t *bar, int32_t x, int32_t y, int32_t z)
+{
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];\n"
+                 :: "r"(smem_addr(sdst)), "l"(map), "r"(smem_addr(bar)), "r"(x), "r"(y), "r"(z) : "memory");
+}
+
 __global__ void __launch_bounds__(THREADS, 1)
-k_decode_mma(const __grid_constant__ CUtensorMap xmap, const MmaArgs M)
+k_decode_mma(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap pmap,
+             const __grid_constant__ CUtensorMap kmap, const MmaArgs M)
 {
     extern __shared__ __align__(16) uint8_t smem_raw[];
     const DecodeArgs &A = M.A;
+    const uint32_t n_items = A.n_q + 1;                                  // planes + mask
+    const uint32_t a_tiles = M.per_plane ? A.n_q : 1;                    // A tiles per stage
+    const uint32_t rbp = M.rbp;                                          // words per row of the bit buffer
     // carve shared memory (A / B stages need 1024-byte alignment for the 128-byte swizzle)
     uint8_t *base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t *a_stages = base;
-    uint8_t *b_stages = a_stages + M.stages * A_STAGE_BYTES;
-    uint32_t *tab = reinterpret_cast<uint32_t *>(b_stages + (size_t)M.stages * M.b_stage_bytes);
-    const uint32_t n_items = A.n_q + 1;                                  // planes + mask
-    uint32_t *rb = tab + table_words(A.n_in, A.nwp, A.nchunks, A.cb);     // [item][row][RB_WORDS]
-    __nv_bfloat16 *lut = reinterpret_cast<__nv_bfloat16 *>(rb + n_items * ROWS * RB_WORDS);   // [row][16]
+    const uint32_t a_stage_bytes = a_tiles * A_STAGE_BYTES;
+    uint8_t *b_stages = a_stages + M.stages * a_stage_bytes;
+    uint32_t *rb = reinterpret_cast<uint32_t *>(b_stages + (size_t)M.stages * M.b_stage_bytes);   // [buf][item][row][rbp]
+    const uint32_t rb_buf_words = n_items * ROWS * rbp;
+    uint32_t *tab = rb + M.rb_bufs * rb_buf_words;
+    uint2 *lut256 = reinterpret_cast<uint2 *>(tab + table_words(A.n_in, A.nwp, A.nchunks, A.cb));   // [256]
+    __nv_bfloat16 *lut = reinterpret_cast<__nv_bfloat16 *>(lut256 + 256);                             // [row][16]
     float *alpha_s = reinterpret_cast<float *>(lut + ROWS * 16);         // [row][8]
     uint64_t *bars = reinterpret_cast<uint64_t *>(alpha_s + ROWS * 8);
     uint64_t *full_a = bars, *full_b = bars + MAX_STAGES, *empty = bars + 2 * MAX_STAGES;
     uint64_t *accum = bars + 3 * MAX_STAGES;
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 3 * MAX_STAGES + 1);
+    uint64_t *bits_full = accum + 1, *bits_empty = accum + 3;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(accum + 5);
     volatile uint32_t *abort_flag = tmem_slot + 1;
 
     const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -292,11 +308,23 @@ k_decode_mma(const __grid_constant__ CUtensorMap xmap, const MmaArgs M)
             mbar_init(empty + s, 1);
         }
         mbar_init(accum, 1);
+        for (uint32_t s = 0; s < 2; ++s) {
+            mbar_init(bits_full + s, 1);
+            mbar_init(bits_empty + s, DEC_THREADS);
+        }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
     if (warp == DEC_WARPS + 1) tmem_alloc(tmem_slot, M.tmem_cols);
-    build_tables(A, tab);                                   // all threads; ends with __syncthreads
+    if (!M.bits32) build_tables(A, tab);                    // only the in-kernel decoder needs them
+    if (tid < 256) {
+        // 4 weights of one plane at a time: index = mask nibble << 4 | bit nibble -> 4 bf16 of -1, 0, +1
+        uint32_t h[4];
+#pragma unroll
+        for (uint32_t k = 0; k < 4; ++k)
+            h[k] = ((tid >> (4 + k)) & 1u) ? (((tid >> k) & 1u) ? 0x3f80u : 0xbf80u) : 0u;
+        lut256[tid] = make_uint2(h[0] | (h[1] << 16), h[2] | (h[3] << 16));
+    }
     if (tid < ROWS) {
         // per-row scales and the table of all 2^n_q weight values (index bit i = plane i, bit 3 = mask)
         const uint64_t r = r0 + tid;
@@ -322,12 +350,14 @@ k_decode_mma(const __grid_constant__ CUtensorMap xmap, const MmaArgs M)
     const uint32_t tmem_base = *tmem_slot;
 
     uint32_t step_count = 0;                    // pipeline steps issued so far (all roles count alike)
+    uint32_t macro_count = 0;                   // bit-buffer fills so far
     uint32_t accum_parity = 0;
     for (uint32_t bc = 0; bc < M.batch; bc += M.nbt) {
         const uint32_t step_begin = macro_begin * STEPS_PER_MACRO;
         uint32_t step_end = macro_end * STEPS_PER_MACRO;
         if (step_end > total_steps) step_end = total_steps;
         const uint32_t nsteps = step_end > step_begin ? step_end - step_begin : 0;
+        const uint32_t nmacros = macro_end > macro_begin ? macro_end - macro_begin : 0;
 
         if (warp < DEC_WARPS) {
             // ------------------------------ decode warps ------------------------------
@@ -341,44 +371,86 @@ k_decode_mma(const __grid_constant__ CUtensorMap xmap, const MmaArgs M)
                 if (item < A.n_q && live && !M.bits32)
                     cur[q] = cursor_at(A.pl[item], A.n_out, r * M.n + (uint64_t)macro_begin * MACRO);
             }
-            uint32_t it = step_count;
-            for (uint32_t mc = macro_begin; mc < macro_end; ++mc) {
+            uint32_t it = step_count, mi = macro_count;
+            for (uint32_t mc = macro_begin; mc < macro_end; ++mc, ++mi) {
                 const uint64_t c0 = (uint64_t)mc * MACRO;
                 const uint32_t cnt = (uint32_t)(M.n - c0 < MACRO ? M.n - c0 : MACRO);
-                // phase 1: bits of this thread's (row, item)s
+                const uint32_t buf = M.tma_bits ? (mi & 1u) : 0u;
+                const uint32_t *rbb = rb + buf * rb_buf_words;
+                bool stop = false;
+                // phase 1: the bit vectors of the 128 rows x MACRO columns into the bit buffer
+                if (M.tma_bits) {
+                    // the TMA thread fetches them as 128 x 64-byte boxes; wait for this buffer
+                    stop = !mbar_wait(bits_full + buf, (mi >> 1) & 1u, abort_flag, A.status);
+                } else if (M.bits32) {
+                    // planes exist as packed bits but rows are not 16-byte aligned: 16 consecutive
+                    // lanes copy the 16 words of one row segment, 32 rows per pass
+                    const uint32_t j = tid & 15;
 #pragma unroll
-                for (uint32_t q = 0; q < 3; ++q) {
-                    const uint32_t item = pq + 4 * q;
-                    if (item > A.n_q) break;
-                    uint32_t *rowbuf = rb + (item * ROWS + prow) * RB_WORDS;
-                    if (!live) {
+                    for (uint32_t pass = 0; pass < ROWS / 32; ++pass) {
+                        const uint32_t rl = pass * 32 + (tid >> 4);
+                        const uint64_t rr = r0 + rl;
+                        const uint64_t p0 = rr * M.n + c0;
+                        const uint64_t w = (p0 >> 5) + j;
+                        const uint32_t sh = (uint32_t)(p0 & 31);
+                        const uint32_t lo = 32 * j;
+                        uint32_t keep = 0;                        // bits of this word that lie in [0, cnt)
+                        if (rr < M.m && lo < cnt) keep = lo + 32 > cnt ? (1u << (cnt - lo)) - 1u : 0xffffffffu;
+                        for (uint32_t item = 0; item <= A.n_q; ++item) {
+                            const uint32_t *src = item < A.n_q ? M.bits32 + (uint64_t)item * M.plane_words32 : M.mask32;
+                            const uint64_t valid = item < A.n_q ? M.plane_words32 : M.mask_words32;
+                            uint32_t v = 0;
+                            if (keep) {
+                                const uint32_t lo_w = w < valid ? __ldg(src + w) : 0u;
+                                const uint32_t hi_w = w + 1 < valid ? __ldg(src + w + 1) : 0u;
+                                v = __funnelshift_r(lo_w, hi_w, sh) & keep;
+                            }
+                            rb[(item * ROWS + rl) * rbp + j] = v;
+                        }
+                    }
+                } else {
 #pragma unroll
-                        for (uint32_t k = 0; k < RB_WORDS; ++k) rowbuf[k] = 0;
-                    } else if (item < A.n_q) {
-                        if (M.bits32)
-                            copy_segment(M.bits32 + (uint64_t)item * M.plane_words32, M.plane_words32,
-                                         r * M.n + c0, cnt, rowbuf);
-                        else
+                    for (uint32_t q = 0; q < 3; ++q) {
+                        const uint32_t item = pq + 4 * q;
+                        if (item > A.n_q) break;
+                        uint32_t *rowbuf = rb + (item * ROWS + prow) * rbp;
+                        if (!live) {
+#pragma unroll
+                            for (uint32_t k = 0; k < RB_WORDS; ++k) rowbuf[k] = 0;
+                        } else if (item < A.n_q) {
                             decode_segment(A, A.pl[item], tab, cur[q], cnt, rowbuf);
-                    } else {
-                        copy_segment(M.mask32, M.mask_words32, r * M.n + c0, cnt, rowbuf);
+                        } else {
+                            copy_segment(M.mask32, M.mask_words32, r * M.n + c0, cnt, rowbuf);
+                        }
                     }
                 }
-                asm volatile("bar.sync 1, %0;\n" :: "n"(DEC_THREADS) : "memory");
-                // phase 2: four steps of 64 columns
-                const uint32_t steps_here = (cnt + KC - 1) / KC;
+                if (!M.tma_bits) asm volatile("bar.sync 1, %0;\n" :: "n"(DEC_THREADS) : "memory");
+                // phase 2: steps of 64 columns; one thread per (row, 16 columns)
+                const uint32_t steps_here = stop ? 0u : (cnt + KC - 1) / KC;
+                const uint32_t row = tid >> 2, quarter = tid & 3, sw = row & 7;
                 for (uint32_t ks = 0; ks < steps_here; ++ks, ++it) {
                     const uint32_t stage = it % M.stages, use = it / M.stages;
                     if (use > 0 && !mbar_wait(empty + stage, (use - 1) & 1u, abort_flag, A.status)) break;
-                    uint8_t *a_stage = a_stages + stage * A_STAGE_BYTES;
-                    {
-                        // one thread per (row, 16 columns): clear its 32 bytes of the stage, then
-                        // write only the unpruned weights (most positions are zero)
-                        const uint32_t row = tid >> 2, quarter = tid & 3;
-                        const uint32_t wi = ks * 2 + (quarter >> 1), sh16 = (quarter & 1) * 16;
-                        uint32_t mw = (rb[(A.n_q * ROWS + row) * RB_WORDS + wi] >> sh16) & 0xffffu;
+                    uint8_t *a_stage = a_stages + stage * a_stage_bytes;
+                    const uint32_t wi = ks * 2 + (quarter >> 1), sh16 = (quarter & 1) * 16;
+                    uint32_t mw = (rbb[(A.n_q * ROWS + row) * rbp + wi] >> sh16) & 0xffffu;
+                    if (M.per_plane) {
+                        // sign tiles, one per plane: -1 / 0 / +1 in bf16 (the scales are applied to
+                        // the accumulators afterwards), four weights per table read
+                        for (uint32_t i = 0; i < A.n_q; ++i) {
+                            const uint32_t bw = (rbb[(i * ROWS + row) * rbp + wi] >> sh16) & 0xffffu;
+                            uint2 e[4];
+#pragma unroll
+                            for (uint32_t q = 0; q < 4; ++q)
+                                e[q] = lut256[(((mw >> (4 * q)) & 15u) << 4) | ((bw >> (4 * q)) & 15u)];
+                            uint8_t *arow = a_stage + i * A_STAGE_BYTES + row * 128;
+                            *reinterpret_cast<uint4 *>(arow + (((quarter * 2) ^ sw) << 4)) = make_uint4(e[0].x, e[0].y, e[1].x, e[1].y);
+                            *reinterpret_cast<uint4 *>(arow + (((quarter * 2 + 1) ^ sw) << 4)) = make_uint4(e[2].x, e[2].y, e[3].x, e[3].y);
+                        }
+                    } else {
+                        // one tile of rescaled weights: clear the thread's 32 bytes, then write only
+                        // the unpruned positions (most are zero)
                         uint8_t *arow = a_stage + row * 128;
-                        const uint32_t sw = row & 7;
 #pragma unroll
                         for (uint32_t q = 0; q < 2; ++q)
                             *reinterpret_cast<uint4 *>(arow + (((quarter * 2 + q) ^ sw) << 4)) = make_uint4(0, 0, 0, 0);
@@ -386,7 +458,7 @@ k_decode_mma(const __grid_constant__ CUtensorMap xmap, const MmaArgs M)
                             uint32_t bw[3];
 #pragma unroll
                             for (uint32_t i = 0; i < 3; ++i)
-                                bw[i] = i < A.n_q ? rb[(i * ROWS + row) * RB_WORDS + wi] >> sh16 : 0u;
+                                bw[i] = i < A.n_q ? rbb[(i * ROWS + row) * rbp + wi] >> sh16 : 0u;
                             const uint16_t *lr = reinterpret_cast<const uint16_t *>(lut) + row * 16;
                             while (mw) {
                                 const uint32_t k = 31u - (uint32_t)__clz((int)mw);
@@ -402,7 +474,7 @@ k_decode_mma(const __grid_constant__ CUtensorMap xmap, const MmaArgs M)
                                 float sum = 0.0f;
                                 for (uint32_t i = 0; i < A.n_q; ++i) {
                                     const float a = alpha_s[row * 8 + i];
-                                    sum = __fadd_rn(sum, ((rb[(i * ROWS + row) * RB_WORDS + wi] >> (sh16 + k)) & 1u) ? a : -a);
+                                    sum = __fadd_rn(sum, ((rbb[(i * ROWS + row) * rbp + wi] >> (sh16 + k)) & 1u) ? a : -a);
                                 }
                                 *reinterpret_cast<uint16_t *>(arow + (((quarter * 2 + (k >> 3)) ^ sw) << 4) + (k & 7) * 2) =
                                     __bfloat16_as_ushort(__float2bfloat16_rn(sum));
@@ -412,20 +484,38 @@ k_decode_mma(const __grid_constant__ CUtensorMap xmap, const MmaArgs M)
                     fence_async_smem();                 // generic-proxy writes -> visible to the tensor core
                     mbar_arrive(full_a + stage);
                 }
+                if (M.tma_bits) mbar_arrive(bits_empty + buf);     // this thread is done with the buffer
                 if (decode_barrier_any(*abort_flag)) break;       // same decision in every decode thread
             }
         } else if (warp == DEC_WARPS) {
             // ------------------------------ TMA producer ------------------------------
             if (lane == 0) {
-                uint32_t it = step_count;
-                for (uint32_t st = step_begin; st < step_end; ++st, ++it) {
-                    const uint32_t stage = it % M.stages, use = it / M.stages;
-                    if (use > 0 && !mbar_wait(empty + stage, (use - 1) & 1u, abort_flag, A.status)) break;
-                    uint8_t *b_stage = b_stages + (size_t)stage * M.b_stage_bytes;
-                    mbar_expect_tx(full_b + stage, M.b_stage_bytes);
-                    for (uint32_t h = 0; h * 256 < M.nbt; ++h)
-                        tma_load_2d(b_stage + h * 256 * 128, &xmap, full_b + stage, (int32_t)(st * KC),
-                                    (int32_t)(bc + h * 256));
+                uint32_t it = step_count, mi = macro_count;
+                bool ok = true;
+                auto fetch_bits = [&](uint32_t mc, uint32_t mix) {
+                    const uint32_t buf = mix & 1u, useb = mix >> 1;
+                    if (useb > 0 && !mbar_wait(bits_empty + buf, (useb - 1) & 1u, abort_flag, A.status)) return false;
+                    uint8_t *dst = reinterpret_cast<uint8_t *>(rb + buf * rb_buf_words);
+                    mbar_expect_tx(bits_full + buf, n_items * ROWS * 64);
+                    for (uint32_t i = 0; i < A.n_q; ++i)
+                        tma_load_3d(dst + i * ROWS * 64, &pmap, bits_full + buf, (int32_t)(mc * (MACRO / 8)), (int32_t)r0, (int32_t)i);
+                    tma_load_2d(dst + A.n_q * ROWS * 64, &kmap, bits_full + buf, (int32_t)(mc * (MACRO / 8)), (int32_t)r0);
+                    return true;
+                };
+                if (M.tma_bits && nmacros) ok = fetch_bits(macro_begin, mi);
+                for (uint32_t mc = macro_begin; mc < macro_end && ok; ++mc, ++mi) {
+                    if (M.tma_bits && mc + 1 < macro_end) ok = fetch_bits(mc + 1, mi + 1);
+                    uint32_t st_lo = mc * STEPS_PER_MACRO, st_hi = st_lo + STEPS_PER_MACRO;
+                    if (st_hi > step_end) st_hi = step_end;
+                    for (uint32_t st = st_lo; st < st_hi && ok; ++st, ++it) {
+                        const uint32_t stage = it % M.stages, use = it / M.stages;
+                        if (use > 0 && !mbar_wait(empty + stage, (use - 1) & 1u, abort_flag, A.status)) { ok = false; break; }
+                        uint8_t *b_stage = b_stages + (size_t)stage * M.b_stage_bytes;
+                        mbar_expect_tx(full_b + stage, M.b_stage_bytes);
+                        for (uint32_t h = 0; h * 256 < M.nbt; ++h)
+                            tma_load_2d(b_stage + h * 256 * 128, &xmap, full_b + stage, (int32_t)(st * KC),
+                                        (int32_t)(bc + h * 256));
+                    }
                 }
             }
         } else {
@@ -442,14 +532,17 @@ k_decode_mma(const __grid_constant__ CUtensorMap xmap, const MmaArgs M)
                          mbar_wait(full_b + stage, use & 1u, abort_flag, A.status);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint32_t a_addr = smem_addr(a_stages + stage * A_STAGE_BYTES);
+                    const uint32_t a_addr = smem_addr(a_stages + stage * a_stage_bytes);
                     const uint32_t b_addr = smem_addr(b_stages + (size_t)stage * M.b_stage_bytes);
+                    for (uint32_t t = 0; t < a_tiles; ++t) {
 #pragma unroll
-                    for (uint32_t k16 = 0; k16 < KC / 16; ++k16) {
-                        for (uint32_t h = 0; h < nmma; ++h)
-                            mma_bf16(tmem_base + h * 256, smem_desc_sw128(a_addr + k16 * 32),
-                                     smem_desc_sw128(b_addr + h * 256 * 128 + k16 * 32), idesc,
-                                     (st > step_begin || k16 > 0) ? 1u : 0u);
+                        for (uint32_t k16 = 0; k16 < KC / 16; ++k16) {
+                            for (uint32_t h = 0; h < nmma; ++h)
+                                mma_bf16(tmem_base + t * M.nbt + h * 256,
+                                         smem_desc_sw128(a_addr + t * A_STAGE_BYTES + k16 * 32),
+                                         smem_desc_sw128(b_addr + h * 256 * 128 + k16 * 32), idesc,
+                                         (st > step_begin || k16 > 0) ? 1u : 0u);
+                        }
                     }
                     mma_commit(empty + stage);          // frees the stage when these MMAs are done
                 }
@@ -457,6 +550,7 @@ k_decode_mma(const __grid_constant__ CUtensorMap xmap, const MmaArgs M)
             }
         }
         step_count += nsteps;
+        macro_count += nmacros;
 
         // ------------------------------ epilogue ------------------------------
         if (warp < DEC_WARPS && nsteps) {
@@ -464,15 +558,32 @@ k_decode_mma(const __grid_constant__ CUtensorMap xmap, const MmaArgs M)
             if (__all_sync(0xffffffffu, ready)) {                  // tcgen05.ld needs the whole warp
                 tc_fence_after();
                 const uint32_t quad = warp & 3, part = warp >> 2;       // TMEM lane quarter, column class
-                const uint64_t r = r0 + quad * 32 + lane;
+                const uint32_t rl = quad * 32 + lane;
+                const uint64_t r = r0 + rl;
                 for (uint32_t c = part * 8; c < M.nbt; c += 8 * (DEC_WARPS / 4)) {
-                    uint32_t v[8];
-                    tmem_ld8(tmem_base + ((quad * 32) << 16) + c, v);
+                    float out[8];
+                    if (M.per_plane) {
+                        // Y = sum over planes of alpha[r][i] * (sign tile i . X)
+#pragma unroll
+                        for (uint32_t e = 0; e < 8; ++e) out[e] = 0.0f;
+                        for (uint32_t i = 0; i < A.n_q; ++i) {
+                            uint32_t v[8];
+                            tmem_ld8(tmem_base + ((quad * 32) << 16) + i * M.nbt + c, v);
+                            const float a = alpha_s[rl * 8 + i];
+#pragma unroll
+                            for (uint32_t e = 0; e < 8; ++e) out[e] = fmaf(a, __uint_as_float(v[e]), out[e]);
+                        }
+                    } else {
+                        uint32_t v[8];
+                        tmem_ld8(tmem_base + ((quad * 32) << 16) + c, v);
+#pragma unroll
+                        for (uint32_t e = 0; e < 8; ++e) out[e] = __uint_as_float(v[e]);
+                    }
                     if (r < M.m) {
 #pragma unroll
                         for (uint32_t e = 0; e < 8; ++e)
                             if (bc + c + e < M.batch)
-                                atomicAdd(M.y + (int64_t)(bc + c + e) * M.ldy + r, __uint_as_float(v[e]));
+                                atomicAdd(M.y + (int64_t)(bc + c + e) * M.ldy + r, out[e]);
                     }
                 }
             }
@@ -545,18 +656,34 @@ int mma_dispatch(const sqnn_desc *desc, const DecodeArgs &A0, const uint64_t *d_
     const uint32_t b16 = (batch + 15) / 16 * 16;
     M.nbt = b16 > 512 ? 512 : b16;
     if (M.nbt > 256) M.nbt = 512;                       // two full 256-column MMAs per step
-    M.tmem_cols = 32;
-    while (M.tmem_cols < M.nbt) M.tmem_cols *= 2;
     M.b_stage_bytes = M.nbt * 128;
     M.bits32 = (const uint32_t *)d_workspace;
     M.plane_words32 = M.A.words64 * 2;
-    const size_t fixed = (size_t)table_words(M.A.n_in, M.A.nwp, M.A.nchunks, M.A.cb) * 4 +
-                         (size_t)(M.A.n_q + 1) * ROWS * RB_WORDS * 4 + ROWS * 16 * 2 + ROWS * 8 * 4 +
-                         (3 * MAX_STAGES + 1) * 8 + 16 + 1024;
+    // One sign tile and one accumulator per plane (exact weights, cheap expansion) while the
+    // accumulators fit tensor memory; otherwise one tile of rescaled bf16 weights.
+    M.per_plane = (uint64_t)M.A.n_q * M.nbt <= 512 ? 1u : 0u;
+    // The bit buffer is filled by TMA when the rows of the packed planes start on 16-byte boundaries.
+    M.tma_bits = (d_workspace && desc->n % 128 == 0 && ((uintptr_t)d_mask & 15) == 0) ? 1u : 0u;
     const size_t budget = 220 * 1024;
+    size_t fixed = 0, per_stage = 0;
+    for (;;) {
+        M.rbp = M.tma_bits ? 16 : RB_WORDS;
+        M.rb_bufs = M.tma_bits ? 2 : 1;
+        const uint32_t a_tiles = M.per_plane ? M.A.n_q : 1;
+        M.tmem_cols = 32;
+        while (M.tmem_cols < a_tiles * M.nbt) M.tmem_cols *= 2;
+        fixed = (size_t)M.rb_bufs * (M.A.n_q + 1) * ROWS * M.rbp * 4 +
+                (size_t)table_words(M.A.n_in, M.A.nwp, M.A.nchunks, M.A.cb) * 4 + 256 * 8 + ROWS * 16 * 2 +
+                ROWS * 8 * 4 + (3 * MAX_STAGES + 5) * 8 + 16 + 1024;
+        per_stage = (size_t)a_tiles * A_STAGE_BYTES + M.b_stage_bytes;
+        if (fixed + 2 * per_stage <= budget) break;
+        if (M.per_plane) { M.per_plane = 0; continue; }        // too many planes for two stages
+        if (M.tma_bits) { M.tma_bits = 0; continue; }          // single bit buffer
+        break;
+    }
     M.stages = MAX_STAGES;
-    while (M.stages > 1 && fixed + (size_t)M.stages * (A_STAGE_BYTES + M.b_stage_bytes) > budget) --M.stages;
-    const size_t smem = fixed + (size_t)M.stages * (A_STAGE_BYTES + M.b_stage_bytes);
+    while (M.stages > 1 && fixed + (size_t)M.stages * per_stage > budget) --M.stages;
+    const size_t smem = fixed + (size_t)M.stages * per_stage;
     if (smem > budget) return SQNN_E_UNSUPPORTED;
 
     const uint32_t row_tiles = (uint32_t)((desc->m + ROWS - 1) / ROWS);
@@ -567,15 +694,30 @@ int mma_dispatch(const sqnn_desc *desc, const DecodeArgs &A0, const uint64_t *d_
     M.macros_per_split = (total_macros + splits - 1) / splits;
     M.splits = (total_macros + M.macros_per_split - 1) / M.macros_per_split;
 
-    CUtensorMap xmap;
+    CUtensorMap xmap, pmap, kmap;
     const cuuint64_t gdim[2] = {(cuuint64_t)desc->n, (cuuint64_t)batch};
     const cuuint64_t gstride[1] = {(cuuint64_t)ldx * 2};
     const cuuint32_t box[2] = {KC, M.nbt > 256 ? 256u : M.nbt};
-    const cuuint32_t estride[2] = {1, 1};
+    const cuuint32_t estride[3] = {1, 1, 1};
     if (encode(&xmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(d_x), gdim, gstride, box, estride,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return SQNN_E_CUDA;
+    pmap = xmap;
+    kmap = xmap;
+    if (M.tma_bits) {
+        // packed planes as bytes: [plane][row][n / 8], and the mask [row][n / 8]; boxes of 128 rows x 64 bytes
+        const cuuint64_t pdim[3] = {(cuuint64_t)(desc->n / 8), (cuuint64_t)desc->m, (cuuint64_t)M.A.n_q};
+        const cuuint64_t pstride[2] = {(cuuint64_t)(desc->n / 8), (cuuint64_t)(M.A.words64 * 8)};
+        const cuuint32_t pbox[3] = {MACRO / 8, ROWS, 1};
+        if (encode(&pmap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, d_workspace, pdim, pstride, pbox, estride,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS ||
+            encode(&kmap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint64_t *>(d_mask), pdim, pstride, pbox, estride,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return SQNN_E_CUDA;
+    }
 
     cudaError_t e = (ldy == (int64_t)desc->m)
         ? cudaMemsetAsync(d_y, 0, (size_t)batch * desc->m * sizeof(float), st)
@@ -587,7 +729,7 @@ int mma_dispatch(const sqnn_desc *desc, const DecodeArgs &A0, const uint64_t *d_
         const int rc = decode_bits_dispatch(A0, d_workspace, st);
         if (rc != SQNN_OK) return rc;
     }
-    k_decode_mma<<<row_tiles * M.splits, THREADS, smem, st>>>(xmap, M);
+    k_decode_mma<<<row_tiles * M.splits, THREADS, smem, st>>>(xmap, pmap, kmap, M);
     return cudaGetLastError() == cudaSuccess ? SQNN_OK : SQNN_E_CUDA;
 }
 
