@@ -5,18 +5,23 @@
 //
 // One CTA owns 128 rows of W and a range of columns.  Per 64-column step
 //   - the decode warps expand the weights of the step into the A stage (bf16, 128-byte rows,
-//     128-byte swizzle) -- the decoded weights exist only in shared memory;
+//     128-byte swizzle) -- the expanded weights exist only in shared memory;
 //   - one thread fetches the matching activations X[bc .. bc+N) x [64 columns] with TMA
 //     (no multicast: every CTA fetches its own tile);
-//   - one thread issues four tcgen05.mma (K = 16 each) that accumulate in tensor memory.
+//   - one thread issues tcgen05.mma (K = 16 each) that accumulate in tensor memory.
 // Column ranges of different CTAs are summed with fp32 atomics on Y (cleared beforehand).
 //
-// Decoding runs in two phases per 256 columns.  Phase 1, one thread per (row, bit vector):
-// the thread walks the slices that cover its row segment (seed -> XOR tables -> patch flips)
-// and leaves the segment's bits, and the mask bits, in a small shared bit buffer.  Phase 2,
-// one thread per (row, 32 columns): the thread clears its part of the stage and then writes only
-// the unpruned positions, each value taken from a per-row table of the 2^n_q sums
-// (+-alpha_1) + (+-alpha_2) + ..., rounded to bf16.
+// Two forms of the A stage.  While n_q * N fits the 512 columns of tensor memory, every plane
+// gets its own tile of -1 / 0 / +1 (mask and sign only, four weights per table read) and its own
+// accumulator, and the epilogue forms sum_i alpha[r][i] * D_i: the weights stay exact and the
+// expansion is a few instructions per weight.  Otherwise one tile holds the rescaled weights
+// (+-alpha_1) + (+-alpha_2) + ... rounded to bf16, written sparsely from a per-row value table.
+//
+// Where the bits come from.  With a workspace the planes have been decoded to packed bits by the
+// tiled decode kernel; 128 x 512-bit boxes of them (and of the mask) are brought in by TMA when
+// rows start on 16-byte boundaries, by coalesced loads otherwise.  Without a workspace one thread
+// per (row, bit vector) walks the slices that cover its row segment (seed -> XOR tables -> patch
+// flips) itself.
 //
 // Every wait on an mbarrier is bounded; a wait that gives up sets SQNN_E_TIMEOUT in the status
 // word and makes all roles leave their loops, so the kernel always returns.
@@ -525,25 +530,33 @@ k_decode_mma(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ C
                 const uint32_t nmma = M.nbt > 256 ? 2 : 1;
                 const uint32_t ncols = M.nbt > 256 ? 256 : M.nbt;
                 const uint32_t idesc = instr_desc_bf16(ncols);
+                // descriptors differ only in the start-address field (units of 16 bytes): keep the
+                // constant part and add offsets, so that issuing an MMA costs a few instructions
+                const uint64_t a_desc0 = smem_desc_sw128(smem_addr(a_stages));
+                const uint64_t b_desc0 = smem_desc_sw128(smem_addr(b_stages));
+                const uint32_t a_stage16 = a_stage_bytes >> 4, b_stage16 = M.b_stage_bytes >> 4;
                 bool ok = true;
+                uint32_t acc = 0;                       // 0 for the very first MMA of every accumulator
                 for (uint32_t st = step_begin; st < step_end && ok; ++st, ++it) {
                     const uint32_t stage = it % M.stages, use = it / M.stages;
                     ok = mbar_wait(full_a + stage, use & 1u, abort_flag, A.status) &&
                          mbar_wait(full_b + stage, use & 1u, abort_flag, A.status);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint32_t a_addr = smem_addr(a_stages + stage * a_stage_bytes);
-                    const uint32_t b_addr = smem_addr(b_stages + (size_t)stage * M.b_stage_bytes);
+                    const uint64_t a_desc = a_desc0 + (uint64_t)(stage * a_stage16);
+                    const uint64_t b_desc = b_desc0 + (uint64_t)(stage * b_stage16);
                     for (uint32_t t = 0; t < a_tiles; ++t) {
+                        for (uint32_t h = 0; h < nmma; ++h) {
+                            const uint32_t d = tmem_base + t * M.nbt + h * 256;
+                            const uint64_t ad = a_desc + (uint64_t)(t * (A_STAGE_BYTES >> 4));
+                            const uint64_t bd = b_desc + (uint64_t)(h * (256 * 128 >> 4));
+                            mma_bf16(d, ad, bd, idesc, acc);
 #pragma unroll
-                        for (uint32_t k16 = 0; k16 < KC / 16; ++k16) {
-                            for (uint32_t h = 0; h < nmma; ++h)
-                                mma_bf16(tmem_base + t * M.nbt + h * 256,
-                                         smem_desc_sw128(a_addr + t * A_STAGE_BYTES + k16 * 32),
-                                         smem_desc_sw128(b_addr + h * 256 * 128 + k16 * 32), idesc,
-                                         (st > step_begin || k16 > 0) ? 1u : 0u);
+                            for (uint32_t k16 = 1; k16 < KC / 16; ++k16)
+                                mma_bf16(d, ad + 2 * k16, bd + 2 * k16, idesc, 1u);
                         }
                     }
+                    acc = 1;
                     mma_commit(empty + stage);          // frees the stage when these MMAs are done
                 }
                 if (ok && nsteps) mma_commit(accum);
