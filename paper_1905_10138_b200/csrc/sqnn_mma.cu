@@ -90,9 +90,12 @@ SQNN_DEV void mbar_expect_tx(uint64_t *bar, uint32_t bytes)
 }
 SQNN_DEV bool mbar_try(uint64_t *bar, uint32_t parity)
 {
+    // The last operand lets the hardware park the thread for up to ~1 ms while the phase is
+    // pending (it wakes as soon as the phase completes), so that waiting threads do not take
+    // issue slots from working ones; the caller's loop still bounds the total wait.
     uint32_t ok;
-    asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
-                 : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity) : "memory");
+    asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n selp.u32 %0, 1, 0, p;\n}\n"
+                 : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity), "r"(1000000u) : "memory");
     return ok != 0;
 }
 // Bounded wait.  Returns false if the wait was abandoned (limit reached or another role gave up).
