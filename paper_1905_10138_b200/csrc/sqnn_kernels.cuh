@@ -240,6 +240,11 @@ SQNN_DEV void load_x(const XT *p, float (&v)[BT])
     for (int q = 0; q < BT; ++q) v[q] = to_float(pk.e[q]);
 }
 
+// Words of a row segment a lane works on at the same time in the GEMV kernel (build-time tunable).
+#ifndef SQNN_GEMV_WORDS_PER_ROUND
+#define SQNN_GEMV_WORDS_PER_ROUND 2
+#endif
+
 // Words of per-warp scratch the GEMV kernel keeps for the scales of the rows a tile touches.
 constexpr uint32_t GEMV_ALPHA_WORDS = 64;
 
@@ -259,7 +264,6 @@ k_decode_gemv(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__
               int64_t ldy, uint32_t n, uint32_t wpt)
 {
     extern __shared__ __align__(16) uint32_t smem[];
-    build_tables(A, smem);
     const uint32_t W = words_per_lane<N_OUT>(A);
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     const uint32_t n_q = A.n_q;
@@ -276,9 +280,32 @@ k_decode_gemv(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__
     const uint64_t mask_words = A.words64 * 2;
     const uint64_t alpha_count = (A.mn / n) * n_q;
     const bool mask_vec = (reinterpret_cast<uintptr_t>(mask32) & 15) == 0;
+    const uint64_t tile_first = (uint64_t)blockIdx.x * ngroups + group, tile_step = (uint64_t)gridDim.x * ngroups;
+
+    // What a tile needs from global memory besides the activations -- its mask words, the scales
+    // of its first rows and this warp's seeds / patch offsets -- is requested before the tables
+    // are built, so that the two latencies overlap; later tiles are requested one tile ahead.
+    auto request = [&](uint64_t tile) {
+        const uint64_t gw0 = tile * 32 * W;
+        if (gw0 * 32 >= A.mn) return;
+        if (sub == n_q % wpt) {
+            stage_mask_tile(mask_s, mask32, gw0, mask_words, W, lane, mask_vec);
+            const uint64_t r_first = gw0 * 32 / n;
+            for (uint32_t i = lane; i < GEMV_ALPHA_WORDS; i += 32) {
+                const uint64_t at = r_first * n_q + i;
+                alpha_s[i] = at < alpha_count ? __ldg(alpha + at) : 0.0f;
+            }
+        }
+    };
+    TileIn<N_OUT ? N_OUT : 40, N_OUT ? N_IN : 12> pre;      // seeds of plane `sub` of the next tile
+    if constexpr (N_OUT != 0) {
+        if (tile_first < A.tiles && sub < n_q) tile_fetch<N_OUT, N_IN>(A.pl[sub], tile_first, lane, pre);
+    }
+    if (tile_first < A.tiles) request(tile_first);
+
     for (uint32_t bc = 0; bc < batch; bc += BT) {
         if constexpr (XS) {
-            __syncthreads();
+            if (bc != 0) __syncthreads();
             if (BT == 1 && (reinterpret_cast<uintptr_t>(x + (int64_t)bc * ldx) & 15) == 0) {
                 constexpr uint32_t PER = 16 / sizeof(XT);
                 const uint4 *src = reinterpret_cast<const uint4 *>(x + (int64_t)bc * ldx);
@@ -296,24 +323,29 @@ k_decode_gemv(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__
                     for (int q = 0; q < BT; ++q) xs[c * BT + q] = v[q];
                 }
             }
-            __syncthreads();
         }
-        for (uint64_t tile = (uint64_t)blockIdx.x * ngroups + group; tile < A.tiles; tile += (uint64_t)gridDim.x * ngroups) {
+        if (bc == 0) build_tables(A, smem);              // ends with a block barrier
+        else __syncthreads();
+        for (uint64_t tile = tile_first; tile < A.tiles; tile += tile_step) {
             const uint64_t gw0 = tile * 32 * W;          // first 32-bit word of the tile
             const uint64_t P0 = gw0 * 32;
             if (P0 >= A.mn) continue;
             const uint64_t P1 = (P0 + 1024ull * W < A.mn) ? P0 + 1024ull * W : A.mn;
             const uint64_t r_first = P0 / n;
-            if (sub == n_q % wpt) {
-                stage_mask_tile(mask_s, mask32, gw0, mask_words, W, lane, mask_vec);
-                // scales of the first rows the tile touches (later rows are fetched when reached)
-                for (uint32_t i = lane; i < GEMV_ALPHA_WORDS; i += 32) {
-                    const uint64_t at = r_first * n_q + i;
-                    alpha_s[i] = at < alpha_count ? __ldg(alpha + at) : 0.0f;
+            if (bc != 0 || tile != tile_first) request(tile);       // not requested ahead of time
+            if constexpr (N_OUT != 0) {
+                for (uint32_t i = sub; i < n_q; i += wpt) {
+                    TileIn<N_OUT, N_IN> in;
+                    if (i == sub && bc == 0 && tile == tile_first) in = pre;
+                    else tile_fetch<N_OUT, N_IN>(A.pl[i], tile, lane, in);
+                    uint32_t st[4];
+                    stage_fetch<N_OUT, N_IN>(A, A.pl[i], in, lane, st);
+                    tile_decode<N_OUT, N_IN>(A, A.pl[i], in, st, region + i * 32 * W, smem, stage, lane);
                 }
+            } else {
+                for (uint32_t i = sub; i < n_q; i += wpt)
+                    decode_warp_tile<N_OUT, N_IN>(A, i, tile, region + i * 32 * W, smem, stage, lane);
             }
-            for (uint32_t i = sub; i < n_q; i += wpt)
-                decode_warp_tile<N_OUT, N_IN>(A, i, tile, region + i * 32 * W, smem, stage, lane);
             cp_async_wait_all();
             if (wpt == 1) __syncwarp();
             else asm volatile("bar.sync %0, %1;\n" :: "r"(1 + group), "r"(32 * wpt) : "memory");
@@ -334,43 +366,71 @@ k_decode_gemv(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__
                 float acc[BT];
 #pragma unroll
                 for (int q = 0; q < BT; ++q) acc[q] = 0.0f;
-                for (uint32_t lw = lw_lo + sub * 32 + lane; lw <= lw_hi; lw += 32 * wpt) {
-                    uint32_t mk = mask_s[lw];
-                    const uint32_t lo = lw * 32;
-                    if (lo < a_loc) mk &= 0xffffffffu << (a_loc - lo);
-                    if (lo + 32 > b_loc) mk &= 0xffffffffu >> (lo + 32 - b_loc);
-                    uint32_t wb[NR];
-                    if constexpr (NQ > 0) {
+                // a lane takes up to four of the segment's words at a time and visits one set mask
+                // bit of each per round: four independent chains of shared-memory reads
+                constexpr uint32_t K = SQNN_GEMV_WORDS_PER_ROUND;
+                const uint32_t wstep = 32 * wpt;
+                for (uint32_t lw0 = lw_lo + sub * 32 + lane; lw0 <= lw_hi; lw0 += wstep * K) {
+                    uint32_t mk[K], wb[K][NR];
+                    int32_t cb[K];
+                    uint32_t any = 0;
 #pragma unroll
-                        for (int i = 0; i < NQ; ++i) wb[i] = region[i * 32 * W + lw];
-                    }
-                    const int32_t cbase = c_tile + (int32_t)lo;
-                    while (mk) {
-                        const uint32_t k = 31u - (uint32_t)__clz((int)mk);
-                        mk ^= 1u << k;
-                        float v = 0.0f;
-                        if constexpr (NQ > 0) {
+                    for (uint32_t j = 0; j < K; ++j) {
+                        const uint32_t lw = lw0 + j * wstep;
+                        mk[j] = 0;
+                        cb[j] = c_tile + (int32_t)a_loc;    // a valid column for the idle slots
 #pragma unroll
-                            for (int i = 0; i < NQ; ++i) {
-                                const float t = ((wb[i] >> k) & 1u) ? al[i] : -al[i];
-                                v = i == 0 ? t : v + t;
-                            }
-                        } else {
-                            for (uint32_t i = 0; i < n_q; ++i) {
-                                const float a1 = __ldg(alpha + r * n_q + i);
-                                v += ((region[i * 32 * W + lw] >> k) & 1u) ? a1 : -a1;
+                        for (int i = 0; i < NR; ++i) wb[j][i] = 0;
+                        if (lw <= lw_hi) {
+                            uint32_t m = mask_s[lw];
+                            const uint32_t lo = lw * 32;
+                            if (lo < a_loc) m &= 0xffffffffu << (a_loc - lo);
+                            if (lo + 32 > b_loc) m &= 0xffffffffu >> (lo + 32 - b_loc);
+                            mk[j] = m;
+                            cb[j] = c_tile + (int32_t)lo;
+                            if constexpr (NQ > 0) {
+#pragma unroll
+                                for (int i = 0; i < NQ; ++i) wb[j][i] = region[i * 32 * W + lw];
+                            } else {
+                                wb[j][0] = lw;
                             }
                         }
-                        const int32_t c = cbase + (int32_t)k;
-                        if constexpr (XS) {
-                            float xv[BT];
-                            load_x<BT, XT>(xs + (uint32_t)c * BT, xv);
+                        any |= mk[j];
+                    }
+                    while (any) {
+                        any = 0;
+                        // branch-free: an exhausted word contributes value 0 at a valid column
 #pragma unroll
-                            for (int q = 0; q < BT; ++q) acc[q] = fmaf(v, xv[q], acc[q]);
-                        } else {
+                        for (uint32_t j = 0; j < K; ++j) {
+                            const bool live = mk[j] != 0;
+                            const uint32_t k = live ? 31u - (uint32_t)__clz((int)mk[j]) : 0u;
+                            mk[j] &= ~(1u << k);
+                            float v = 0.0f;
+                            if constexpr (NQ > 0) {
 #pragma unroll
-                            for (int q = 0; q < BT; ++q)
-                                if (bc + q < batch) acc[q] = fmaf(v, to_float(x[(int64_t)(bc + q) * ldx + c]), acc[q]);
+                                for (int i = 0; i < NQ; ++i) {
+                                    const float t = ((wb[j][i] >> k) & 1u) ? al[i] : -al[i];
+                                    v = i == 0 ? t : v + t;
+                                }
+                            } else {
+                                for (uint32_t i = 0; i < n_q; ++i) {
+                                    const float a1 = __ldg(alpha + r * n_q + i);
+                                    v += ((region[i * 32 * W + wb[j][0]] >> k) & 1u) ? a1 : -a1;
+                                }
+                            }
+                            v = live ? v : 0.0f;
+                            const int32_t c = cb[j] + (int32_t)k;
+                            if constexpr (XS) {
+                                float xv[BT];
+                                load_x<BT, XT>(xs + (uint32_t)c * BT, xv);
+#pragma unroll
+                                for (int q = 0; q < BT; ++q) acc[q] = fmaf(v, xv[q], acc[q]);
+                            } else {
+#pragma unroll
+                                for (int q = 0; q < BT; ++q)
+                                    if (bc + q < batch) acc[q] = fmaf(v, to_float(x[(int64_t)(bc + q) * ldx + c]), acc[q]);
+                            }
+                            any |= mk[j];
                         }
                     }
                 }
