@@ -122,6 +122,13 @@ typedef struct sqnn_desc {
 int sqnn_encode_host(const sqnn_xornet *net, const sqnn_planes *layer, uint32_t flags,
                      void **blob, size_t *blob_bytes, sqnn_stats *stats);
 
+/* As sqnn_encode_host, but the seeds are given: wc[i][s] is the seed of slice s of plane i (for
+ * instance from sqnn_search_seeds).  n_patch and d_patch follow by expanding each seed and
+ * comparing on the care bits (Algorithm 1, its last three steps).  Any seed gives a lossless blob;
+ * better seeds give fewer patches.  Errors: INVALID_ARG (also a seed >= 2^n_in), NOMEM. */
+int sqnn_encode_seeds_host(const sqnn_xornet *net, const sqnn_planes *layer, const uint32_t *const *wc,
+                           void **blob, size_t *blob_bytes, sqnn_stats *stats);
+
 /* Packs logical per-plane arrays (the three parts of the format, Section 3.2) into a blob:
  * wc[i][s] seed of slice s (bit t = w^c[t]), np[i][s] = n_patch, dp[i] = all d_patch entries of
  * plane i in slice order.  Arrays are host, length l, l and sum(np[i]).  Errors: INVALID_ARG
@@ -210,6 +217,16 @@ int sqnn_decode_matmul_static(const sqnn_desc *desc, const void *d_blob, const u
                               const float *d_alpha, const void *d_x, int x_dtype, uint32_t batch,
                               int64_t ldx, float *d_y, int64_t ldy, uint32_t *d_status,
                               void *cuda_stream);
+
+/* Exhaustive seed search on the device (Section 5.2, "minimizing n_patch for small n_in"): for every
+ * slice of every plane all 2^n_in seeds are expanded and the one with the fewest wrong care bits is
+ * kept, the smallest seed among equals.  net: host.  d_planes / d_mask: device, packed as in
+ * sqnn_planes.  d_wc / d_np: device outputs, n_q * l entries each (plane-major, l = ceil(mn/n_out)):
+ * the seed and its number of wrong care bits (= n_patch).  Queues on the stream, allocates nothing.
+ * Cost grows as 2^n_in per slice.  Errors: INVALID_ARG, UNSUPPORTED (n_in > 20), CUDA. */
+int sqnn_search_seeds(const sqnn_xornet *net, uint64_t m, uint64_t n, uint32_t n_q,
+                      const uint64_t *d_planes, const uint64_t *d_mask, uint32_t *d_wc, uint16_t *d_np,
+                      void *cuda_stream);
 
 /* Scratch bytes sqnn_decode_matmul can use for this layer and batch (0 if none). */
 size_t sqnn_workspace_bytes(const sqnn_desc *desc, uint32_t batch);

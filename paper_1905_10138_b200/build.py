@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libsqnn.so")
-SOURCES = ["sqnn_host.cpp", "sqnn_api.cu", "sqnn_mma.cu"]
+SOURCES = ["sqnn_host.cpp", "sqnn_api.cu", "sqnn_mma.cu", "sqnn_search.cu"]
 SHAPE_SOURCE = "sqnn_shape.cu"
 # (n_out, n_in) with compile-time kernels -- the list in csrc/sqnn_shapes.h -- plus the run-time shape (0, 0)
 SHAPES = [(40, 12), (40, 16), (60, 12), (80, 8), (80, 16), (100, 10), (200, 10), (0, 0)]

@@ -254,35 +254,37 @@ const char *sqnn_status_string(int status)
     }
 }
 
-int sqnn_encode_host(const sqnn_xornet *net, const sqnn_planes *layer, uint32_t flags,
-                     void **blob, size_t *blob_bytes, sqnn_stats *stats)
+// Shared by sqnn_encode_host and sqnn_encode_seeds_host: seeds come from Algorithm 1, from the
+// exhaustive search, or from the caller (given != NULL); patch counts and positions follow by
+// expanding each seed and comparing on the care bits.
+static int encode_impl(const sqnn_xornet *net, const sqnn_planes *layer, bool exhaustive,
+                       const uint32_t *const *given, void **blob, size_t *blob_bytes, sqnn_stats *stats)
 {
-    if (!net_ok(net) || !layer || !blob || !blob_bytes) return SQNN_E_INVALID_ARG;
-    if (!layer->planes || !layer->mask || layer->n_q < 1 || layer->n_q > SQNN_MAX_PLANES)
-        return SQNN_E_INVALID_ARG;
-    if (layer->m == 0 || layer->n == 0 || layer->m > ((uint64_t)1 << 40) / layer->n)
-        return SQNN_E_INVALID_ARG;
-    const bool exhaustive = (flags & SQNN_ENCODE_EXHAUSTIVE) != 0;
-    if (exhaustive && net->n_in > 20) return SQNN_E_INVALID_ARG;
     try {
         const uint64_t mn = layer->m * layer->n;
         const uint32_t n_out = net->n_out, n_in = net->n_in, n_q = layer->n_q;
         const uint64_t l = (mn + n_out - 1) / n_out;
         const uint64_t words = (mn + 63) / 64;
         std::vector<uint64_t> tab;
-        if (exhaustive) build_outputs(net->rows, n_out, n_in, tab);
+        if (exhaustive && !given) build_outputs(net->rows, n_out, n_in, tab);
         std::vector<PlaneArrays> pa(n_q);
         for (uint32_t i = 0; i < n_q; ++i) {
             const uint64_t *plane = layer->planes + (uint64_t)i * words;
             pa[i].wc.assign(l, 0);
             pa[i].np.assign(l, 0);
+            bool bad_seed = false;
             // pass 1: seed and patch count of every slice (slices are independent)
 #pragma omp parallel for schedule(dynamic, 4096)
             for (int64_t s = 0; s < (int64_t)l; ++s) {
                 SliceBits sb;
                 load_slice(plane, layer->mask, mn, n_out, (uint64_t)s, sb);
-                const uint32_t seed = exhaustive ? encode_exhaustive(tab, n_in, sb)
-                                                 : encode_alg1(net->rows, n_out, sb);
+                uint32_t seed;
+                if (given) {
+                    seed = given[i][s];
+                    if (n_in < 32 && (seed >> n_in)) { bad_seed = true; seed = 0; }
+                } else {
+                    seed = exhaustive ? encode_exhaustive(tab, n_in, sb) : encode_alg1(net->rows, n_out, sb);
+                }
                 uint64_t out[4];
                 expand(net->rows, n_out, seed, out);
                 int wrong = 0;
@@ -290,6 +292,7 @@ int sqnn_encode_host(const sqnn_xornet *net, const sqnn_planes *layer, uint32_t 
                 pa[i].wc[s] = seed;
                 pa[i].np[s] = (uint16_t)wrong;
             }
+            if (bad_seed) return SQNN_E_INVALID_ARG;
             // pass 2: positions of the wrong care bits, written at the running offset
             std::vector<uint64_t> start(l + 1, 0);
             for (uint64_t s = 0; s < l; ++s) start[s + 1] = start[s] + pa[i].np[s];
@@ -325,6 +328,30 @@ int sqnn_encode_host(const sqnn_xornet *net, const sqnn_planes *layer, uint32_t 
     } catch (const std::bad_alloc &) {
         return SQNN_E_NOMEM;
     }
+}
+
+static bool layer_ok(const sqnn_planes *layer)
+{
+    return layer && layer->planes && layer->mask && layer->n_q >= 1 && layer->n_q <= SQNN_MAX_PLANES &&
+           layer->m != 0 && layer->n != 0 && layer->m <= ((uint64_t)1 << 40) / layer->n;
+}
+
+int sqnn_encode_host(const sqnn_xornet *net, const sqnn_planes *layer, uint32_t flags,
+                     void **blob, size_t *blob_bytes, sqnn_stats *stats)
+{
+    if (!net_ok(net) || !layer_ok(layer) || !blob || !blob_bytes) return SQNN_E_INVALID_ARG;
+    const bool exhaustive = (flags & SQNN_ENCODE_EXHAUSTIVE) != 0;
+    if (exhaustive && net->n_in > 20) return SQNN_E_INVALID_ARG;
+    return encode_impl(net, layer, exhaustive, nullptr, blob, blob_bytes, stats);
+}
+
+int sqnn_encode_seeds_host(const sqnn_xornet *net, const sqnn_planes *layer, const uint32_t *const *wc,
+                           void **blob, size_t *blob_bytes, sqnn_stats *stats)
+{
+    if (!net_ok(net) || !layer_ok(layer) || !wc || !blob || !blob_bytes) return SQNN_E_INVALID_ARG;
+    for (uint32_t i = 0; i < layer->n_q; ++i)
+        if (!wc[i]) return SQNN_E_INVALID_ARG;
+    return encode_impl(net, layer, false, wc, blob, blob_bytes, stats);
 }
 
 int sqnn_pack_host(const sqnn_xornet *net, uint64_t m, uint64_t n, uint32_t n_q,

@@ -4,6 +4,7 @@
     python -m paper_1905_10138_b200.profile_case sink    --sweep 2 2
     python -m paper_1905_10138_b200.profile_case bf16    --cfg 3
     python -m paper_1905_10138_b200.profile_case matmul  --cfg 2 --batch 1
+    python -m paper_1905_10138_b200.profile_case search  --cfg 2          (exhaustive seed search)
 
 --cfg 1..4 picks a layer of the benchmark configurations (optionally --rows / --cols smaller),
 --sweep I_S I_M a point of the decode-only sweep (prune rate index, network index).
@@ -20,7 +21,7 @@ def main():
     import torch
     from . import sqnn, workloads as wl
     ap = argparse.ArgumentParser()
-    ap.add_argument("what", choices=["decode", "sink", "bf16", "matmul"])
+    ap.add_argument("what", choices=["decode", "sink", "bf16", "matmul", "search"])
     ap.add_argument("--cfg", type=int, default=0)
     ap.add_argument("--sweep", type=int, nargs=2, default=None)
     ap.add_argument("--rows", type=int, default=None)
@@ -49,6 +50,14 @@ def main():
     elif a.what == "sink":
         out = torch.empty(2, dtype=torch.int64, device="cuda")
         fn = lambda: sqnn.sqnn_decode(desc, d_blob, None, None, sqnn.OUT_SINK, out, status)
+    elif a.what == "search":
+        slices = (layer.mn + layer.n_out - 1) // layer.n_out
+        d_planes = torch.from_numpy(planes_words.view(np.int64)).cuda()
+        d_wc = torch.empty(layer.n_q * slices, dtype=torch.int32, device="cuda")
+        d_np = torch.empty(layer.n_q * slices, dtype=torch.int16, device="cuda")
+        rows = wl.network_rows(layer.M)
+        fn = lambda: sqnn.sqnn_search_seeds(rows, layer.n_in, layer.m, layer.n, layer.n_q, d_planes, d_mask,
+                                            d_wc, d_np)
     elif a.what == "bf16":
         out = torch.empty((layer.m, layer.n), dtype=torch.bfloat16, device="cuda")
         fn = lambda: sqnn.sqnn_decode(desc, d_blob, d_mask, d_alpha, sqnn.OUT_BF16, out, status)
@@ -71,6 +80,9 @@ def main():
         e1.record()
         torch.cuda.synchronize()
         times.append(e0.elapsed_time(e1) * 1e3)
+    if a.what == "search":
+        found = d_np.cpu().numpy().view(np.uint16).reshape(layer.n_q, -1).astype(np.int64).sum(axis=1)
+        print(f"exhaustive search patches per plane {found.tolist()} vs Algorithm 1 {stats['patches'][:layer.n_q]}")
     print(f"{a.what} {layer.name} {layer.m}x{layer.n} n_q={layer.n_q} M {layer.n_out}x{layer.n_in}: "
           f"us per iteration {['%.1f' % t for t in times]}  patches {stats['patches'][:layer.n_q]} "
           f"stored bits/weight {stats['bpw_actual']:.4f}  status {int(status.item())}")

@@ -81,6 +81,10 @@ def lib():
                                       ctypes.c_int, ctypes.c_size_t)
         P = ctypes.POINTER
         L.sqnn_encode_host.argtypes = [P(XorNet), P(Planes), u32, P(vp), P(sz), P(Stats)]
+        L.sqnn_encode_seeds_host.argtypes = [P(XorNet), P(Planes), P(vp), P(vp), P(sz), P(Stats)]
+        L.sqnn_encode_seeds_host.restype = i32
+        L.sqnn_search_seeds.argtypes = [P(XorNet), u64, u64, u32, vp, vp, vp, vp, vp]
+        L.sqnn_search_seeds.restype = i32
         L.sqnn_pack_host.argtypes = [P(XorNet), u64, u64, u32, P(vp), P(vp), P(vp), P(vp), P(sz)]
         L.sqnn_unpack_host.argtypes = [vp, sz, u32, P(vp), P(vp), P(vp), P(u64)]
         L.sqnn_describe_host.argtypes = [vp, sz, P(Desc)]
@@ -143,6 +147,28 @@ def sqnn_encode_host(rows, n_in, m, n, n_q, planes_words, mask_words, flags=ENCO
     _check(lib().sqnn_encode_host(ctypes.byref(net), ctypes.byref(layer), flags, ctypes.byref(blob),
                                   ctypes.byref(nbytes), ctypes.byref(st)), "sqnn_encode_host")
     return _take(blob, nbytes.value), st.as_dict(n_q)
+
+
+def sqnn_encode_seeds_host(rows, n_in, m, n, n_q, planes_words, mask_words, wc):
+    """As sqnn_encode_host with the seeds given: wc is a list (one per plane) of uint32 [l]."""
+    net, _keep = _net(rows, n_in)
+    planes_words = np.ascontiguousarray(planes_words, dtype=np.uint64)
+    mask_words = np.ascontiguousarray(mask_words, dtype=np.uint64)
+    wc = [np.ascontiguousarray(a, dtype=np.uint32) for a in wc]
+    layer = Planes(m, n, n_q, planes_words.ctypes.data, mask_words.ctypes.data)
+    arr = (ctypes.c_void_p * n_q)(*[a.ctypes.data for a in wc])
+    blob, nbytes, st = ctypes.c_void_p(), ctypes.c_size_t(), Stats()
+    _check(lib().sqnn_encode_seeds_host(ctypes.byref(net), ctypes.byref(layer), arr, ctypes.byref(blob),
+                                        ctypes.byref(nbytes), ctypes.byref(st)), "sqnn_encode_seeds_host")
+    return _take(blob, nbytes.value), st.as_dict(n_q)
+
+
+def sqnn_search_seeds(rows, n_in, m, n, n_q, d_planes, d_mask, d_wc, d_np, stream=None):
+    """Exhaustive seed search on the device.  d_planes / d_mask: CUDA int64 tensors (packed bits);
+    d_wc: CUDA int32 [n_q * l]; d_np: CUDA int16 [n_q * l].  Queues on ``stream``."""
+    net, _keep = _net(rows, n_in)
+    _check(lib().sqnn_search_seeds(ctypes.byref(net), m, n, n_q, _dev_ptr(d_planes), _dev_ptr(d_mask),
+                                   _dev_ptr(d_wc), _dev_ptr(d_np), _stream_ptr(stream)), "sqnn_search_seeds")
 
 
 def sqnn_pack_host(rows, n_in, m, n, wc, np_, dp):
