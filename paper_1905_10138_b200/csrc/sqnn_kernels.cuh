@@ -371,7 +371,7 @@ k_decode_gemv(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__
                 constexpr uint32_t K = SQNN_GEMV_WORDS_PER_ROUND;
                 const uint32_t wstep = 32 * wpt;
                 for (uint32_t lw0 = lw_lo + sub * 32 + lane; lw0 <= lw_hi; lw0 += wstep * K) {
-                    uint32_t mk[K], wb[K][NR];
+                    uint32_t mk[K], wb[K][NR], k_idle[K];
                     int32_t cb[K];
                     uint32_t any = 0;
 #pragma unroll
@@ -379,12 +379,16 @@ k_decode_gemv(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__
                         const uint32_t lw = lw0 + j * wstep;
                         mk[j] = 0;
                         cb[j] = c_tile + (int32_t)a_loc;    // a valid column for the idle slots
+                        k_idle[j] = 0;
 #pragma unroll
                         for (int i = 0; i < NR; ++i) wb[j][i] = 0;
                         if (lw <= lw_hi) {
                             uint32_t m = mask_s[lw];
                             const uint32_t lo = lw * 32;
-                            if (lo < a_loc) m &= 0xffffffffu << (a_loc - lo);
+                            if (lo < a_loc) {
+                                m &= 0xffffffffu << (a_loc - lo);
+                                k_idle[j] = a_loc - lo;     // bit 0 of this word belongs to the row before
+                            }
                             if (lo + 32 > b_loc) m &= 0xffffffffu >> (lo + 32 - b_loc);
                             mk[j] = m;
                             cb[j] = c_tile + (int32_t)lo;
@@ -399,11 +403,12 @@ k_decode_gemv(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__
                     }
                     while (any) {
                         any = 0;
-                        // branch-free: an exhausted word contributes value 0 at a valid column
+                        // branch-free: an exhausted word contributes value 0 at a column of this row
+                        // (0 * x must not meet an x read from outside the row: it could be Inf or NaN)
 #pragma unroll
                         for (uint32_t j = 0; j < K; ++j) {
                             const bool live = mk[j] != 0;
-                            const uint32_t k = live ? 31u - (uint32_t)__clz((int)mk[j]) : 0u;
+                            const uint32_t k = live ? 31u - (uint32_t)__clz((int)mk[j]) : k_idle[j];
                             mk[j] &= ~(1u << k);
                             float v = 0.0f;
                             if constexpr (NQ > 0) {

@@ -68,6 +68,24 @@ def test_gemv_respects_row_strides():
     assert np.all(y[:, 50:] == 7.0)
 
 
+def test_gemv_never_reads_activations_outside_a_row():
+    """Rows that start inside a 32-bit word (n not a multiple of 32), activations read from global
+    memory (too wide for shared memory) with NaN between the rows of X: a read at a column
+    outside [0, n) would poison Y even if its weight were zero."""
+    import torch
+    from paper_1905_10138_b200 import sqnn
+    layer = generic_layer(100, 10, 24, 5150, 0.3, 31)
+    x = layer.activations(8)
+    ref = reference(layer, x)
+    dev = H.DeviceLayer(layer, H.blob_from_library(layer)[0])
+    xbuf = torch.full((10, 5150 + 64), float("nan"), dtype=torch.float32, device="cuda")
+    xbuf[1:9, 32:32 + 5150] = torch.from_numpy(x).cuda()
+    ybuf = torch.full((8, 24), float("nan"), dtype=torch.float32, device="cuda")
+    sqnn.sqnn_decode_matmul(dev.desc, dev.blob, dev.mask, dev.alpha, xbuf[1:9, 32:32 + 5150], ybuf, None, dev.status)
+    torch.cuda.synchronize()
+    assert H.rel_err(ybuf.cpu().numpy(), ref) <= TOL_F32
+
+
 # ----------------------------------------------------------------------------------------------
 # tensor-core path (batch >= 16): weights are rounded to bf16, fp32 accumulation in tensor memory
 # ----------------------------------------------------------------------------------------------
