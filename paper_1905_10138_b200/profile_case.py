@@ -24,6 +24,8 @@ def main():
     ap.add_argument("what", choices=["decode", "sink", "bf16", "matmul", "search"])
     ap.add_argument("--cfg", type=int, default=0)
     ap.add_argument("--sweep", type=int, nargs=2, default=None)
+    ap.add_argument("--repeat", type=int, default=0,
+                    help="also time REPEAT calls inside one event interval (finer than one event tick)")
     ap.add_argument("--rows", type=int, default=None)
     ap.add_argument("--cols", type=int, default=None)
     ap.add_argument("--batch", type=int, default=1)
@@ -80,11 +82,27 @@ def main():
         e1.record()
         torch.cuda.synchronize()
         times.append(e0.elapsed_time(e1) * 1e3)
+    if a.repeat > 0:
+        def interval(f):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda._sleep(2_000_000)
+            e0.record()
+            for _ in range(a.repeat):
+                f()
+            e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) * 1e3 / a.repeat
+        if scratch is not None:
+            both = min(interval(lambda: (scratch.fill_(1), fn())) for _ in range(3))
+            alone = min(interval(lambda: scratch.fill_(1)) for _ in range(3))
+            print(f"{a.repeat} x (flush + call) {both:.2f} us each, flush alone {alone:.2f}: call {both - alone:.2f} us (cold L2)")
+        else:
+            print(f"{a.repeat} calls back to back: {min(interval(fn) for _ in range(3)):.2f} us each (warm L2)")
     if a.what == "search":
         found = d_np.cpu().numpy().view(np.uint16).reshape(layer.n_q, -1).astype(np.int64).sum(axis=1)
         print(f"exhaustive search patches per plane {found.tolist()} vs Algorithm 1 {stats['patches'][:layer.n_q]}")
     print(f"{a.what} {layer.name} {layer.m}x{layer.n} n_q={layer.n_q} M {layer.n_out}x{layer.n_in}: "
-          f"us per iteration {['%.1f' % t for t in times]}  patches {stats['patches'][:layer.n_q]} "
+          f"us per iteration {['%.1f' % t for t in times[:8]]} mean after the first {np.mean(times[1:]) if len(times) > 1 else times[0]:.2f}  patches {stats['patches'][:layer.n_q]} "
           f"stored bits/weight {stats['bpw_actual']:.4f}  status {int(status.item())}")
 
 
