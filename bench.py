@@ -250,7 +250,9 @@ def run_ours(args):
                       "parallelism": "replicas only" if world > 1 else "single GPU",
                       "bits_per_weight_eq1": stats["bpw_eq1"], "bits_per_weight_stored": stats["bpw_actual"],
                       "patches": stats["patches"][0]},
-           "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps, "roofline": roofline}
+           "clocks": clocks, "e2e": e2e,
+           "gpu_launches": 2 * args.steps,      # per step: the kernel clearing Y and the fused decode-GEMV
+           "roofline": roofline}
 
     if rank == 0 and not args.quick:
         out["extra"] = extras(torch, sqnn, wl, layer, desc, d_blob, d_mask, d_alpha, status, flush, peaks, args)

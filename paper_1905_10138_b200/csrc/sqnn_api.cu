@@ -93,15 +93,28 @@ int sm_count()
 }
 
 
+// Clears Y[b][r] (row stride ldy); dependents may be launched as soon as every block has started.
+__global__ void k_clear_y(float *__restrict__ y, int64_t ldy, uint64_t m, uint64_t cells)
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < cells; i += (uint64_t)gridDim.x * blockDim.x) {
+        const uint64_t b = i / m;
+        y[(int64_t)b * ldy + (int64_t)(i - b * m)] = 0.0f;
+    }
+}
+
 static int gemv_dispatch(const DecodeArgs &A, const uint64_t *d_mask, const float *d_alpha, const void *d_x,
                          int x_dtype, int64_t ldx, uint32_t batch, float *d_y, int64_t ldy, uint64_t m, uint64_t n,
                          cudaStream_t st)
 {
-    // Y is accumulated with atomics: clear it first.
-    cudaError_t e = (ldy == (int64_t)m)
-        ? cudaMemsetAsync(d_y, 0, (size_t)batch * m * sizeof(float), st)
-        : cudaMemset2DAsync(d_y, (size_t)ldy * sizeof(float), 0, (size_t)m * sizeof(float), batch, st);
-    if (e != cudaSuccess) return SQNN_E_CUDA;
+    // Y is accumulated with atomics: clear it first.  The clearing kernel lets the product kernel
+    // start at once (programmatic dependent launch); that one waits for the cleared Y only before
+    // its first atomic, so its launch and its first fetches overlap the clearing.
+    const uint64_t cells = (uint64_t)batch * m;
+    uint64_t blocks = (cells + 1023) / 1024;
+    if (blocks > (uint64_t)sm_count()) blocks = (uint64_t)sm_count();
+    k_clear_y<<<(uint32_t)blocks, 256, 0, st>>>(d_y, ldy, m, cells);
+    if (cudaGetLastError() != cudaSuccess) return SQNN_E_CUDA;
 #define SQNN_GEMV_CASE(NO, NI) \
     if (A.n_out == NO && A.n_in == NI) return gemv_shape<NO, NI>(A, d_mask, d_alpha, d_x, x_dtype, ldx, batch, d_y, ldy, n, st);
     SQNN_FOR_SHAPES(SQNN_GEMV_CASE)

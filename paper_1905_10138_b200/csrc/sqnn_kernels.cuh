@@ -349,6 +349,9 @@ k_decode_gemv(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__
             cp_async_wait_all();
             if (wpt == 1) __syncwarp();
             else asm volatile("bar.sync %0, %1;\n" :: "r"(1 + group), "r"(32 * wpt) : "memory");
+            // Y is cleared by the kernel before this one in the stream; under a programmatic dependent
+            // launch this is where its results are awaited (a no-op otherwise)
+            asm volatile("griddepcontrol.wait;" ::: "memory");
             for (uint64_t r = r_first; r * n < P1; ++r) {
                 const uint64_t a = r * n > P0 ? r * n : P0;
                 const uint64_t b = (r + 1) * n < P1 ? (r + 1) * n : P1;
@@ -548,15 +551,30 @@ inline int launch_gemv_bt(const DecodeArgs &A, const uint64_t *d_mask, const flo
     const size_t extra = xs ? xbytes : 0;
     if (tab + per_group + extra > limit) return SQNN_E_UNSUPPORTED;
     while (groups > 1 && tab + groups * per_group + extra > limit) --groups;
-    const size_t smem = tab + groups * per_group + extra;
+    size_t smem = tab + groups * per_group + extra;
     const uint32_t warps = groups * wpt;
     const uint32_t grid = grid_for(live, groups, 2);
+    // A grid that fits one block per SM asks for more than half of an SM's shared memory, so that
+    // no two of its blocks are placed on the same SM while other SMs stay empty.
+    if (grid <= sms && smem < 116 * 1024) smem = 116 * 1024;
+    // The kernel may start while the kernel before it in the stream (the one clearing Y) still
+    // runs; it waits for that kernel's results before its first atomic on Y.
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(warps * 32);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
 #define SQNN_GEMV_LAUNCH(XSV, NQV)                                                                           \
     do {                                                                                                     \
         auto k = k_decode_gemv<N_OUT, N_IN, BT, XT, XSV, NQV>;                                               \
         if (prepare(k, smem)) return SQNN_E_CUDA;                                                            \
-        k<<<grid, warps * 32, smem, st>>>(A, (const uint32_t *)d_mask, d_alpha, (const XT *)d_x, ldx, batch, \
-                                           d_y, ldy, (uint32_t)n, wpt);                                      \
+        if (cudaLaunchKernelEx(&cfg, k, A, (const uint32_t *)d_mask, d_alpha, (const XT *)d_x, ldx, batch,   \
+                               d_y, ldy, (uint32_t)n, wpt) != cudaSuccess) return SQNN_E_CUDA;               \
     } while (0)
     if (!xs) SQNN_GEMV_LAUNCH(false, 0);
     else if (A.n_q == 1) SQNN_GEMV_LAUNCH(true, 1);
