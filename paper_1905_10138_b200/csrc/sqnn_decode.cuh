@@ -110,20 +110,49 @@ inline __host__ __device__ uint32_t table_words(uint32_t n_in, uint32_t nwp, uin
 // Builds the column words of M and the chunk tables.  All threads of the block take part.
 // An entry's value splits as (high << lo_bits) | low: entries with only low or only high bits
 // are XORed together from the columns directly, every other entry is the XOR of those two.
-SQNN_DEV void build_tables(const DecodeArgs &A, uint32_t *tab)
+// The build comes in two calls so that a kernel can request the rows of M first, start its other
+// fetches, and only then wait: build_tables_begin stores the rows in shared memory (block
+// barrier), build_tables_finish does the rest (ends with a block barrier).
+struct RowsAhead { uint32_t r0, r1; };              // rows threadIdx.x and threadIdx.x + blockDim.x
+
+SQNN_DEV uint32_t *rows_scratch()
 {
-    __shared__ uint32_t rows_s[256];                  // rows of M, fetched once with coalesced loads
+    __shared__ uint32_t rows_s[256];
+    return rows_s;
+}
+
+SQNN_DEV RowsAhead fetch_rows(const DecodeArgs &A)
+{
+    RowsAhead p{0u, 0u};
+    if (threadIdx.x < A.n_out) p.r0 = __ldg(A.rows + threadIdx.x);
+    if (threadIdx.x + blockDim.x < A.n_out) p.r1 = __ldg(A.rows + threadIdx.x + blockDim.x);
+    return p;
+}
+
+SQNN_DEV void build_tables_begin(const DecodeArgs &A, RowsAhead ahead)
+{
+    uint32_t *rows_s = rows_scratch();
+    const uint32_t n_out = A.n_out;
+    if (threadIdx.x < n_out) rows_s[threadIdx.x] = ahead.r0;
+    if (threadIdx.x + blockDim.x < n_out) rows_s[threadIdx.x + blockDim.x] = ahead.r1;
+    for (uint32_t j = threadIdx.x + 2 * blockDim.x; j < n_out; j += blockDim.x) rows_s[j] = __ldg(A.rows + j);
+    __syncthreads();
+}
+
+SQNN_DEV void build_tables_finish(const DecodeArgs &A, uint32_t *tab)
+{
+    const uint32_t *rows_s = rows_scratch();
     const uint32_t nwp = A.nwp, n_in = A.n_in, n_out = A.n_out, cb = A.cb;
     const uint32_t kshift = nwp == 1 ? 0 : nwp == 2 ? 1 : nwp == 4 ? 2 : 3;
     uint32_t *cols = tab + A.nchunks * (1u << cb) * nwp;
-    for (uint32_t j = threadIdx.x; j < n_out; j += blockDim.x) rows_s[j] = __ldg(A.rows + j);
-    __syncthreads();
-    for (uint32_t i = threadIdx.x; i < n_in * nwp; i += blockDim.x) {
+    // word k of column t: bit j of it is bit t of row 32 k + j -- one ballot over 32 rows
+    const uint32_t lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+    for (uint32_t i = threadIdx.x >> 5; i < n_in * nwp; i += nwarps) {
         const uint32_t t = i >> kshift, k = i & (nwp - 1);
-        uint32_t w = 0;
-        for (uint32_t j = 32 * k; j < n_out && j < 32 * k + 32; ++j)
-            w |= ((rows_s[j] >> t) & 1u) << (j - 32 * k);
-        cols[i] = w;
+        const uint32_t j = 32 * k + lane;
+        const uint32_t r = j < n_out ? rows_s[j] : 0u;
+        const uint32_t w = __ballot_sync(0xffffffffu, (r >> t) & 1u);
+        if (lane == 0) cols[i] = w;
     }
     __syncthreads();
     const uint32_t lo_bits = cb / 2, hi_bits = cb - lo_bits;
@@ -134,6 +163,7 @@ SQNN_DEV void build_tables(const DecodeArgs &A, uint32_t *tab)
         const uint32_t k = r & (nwp - 1), e = r >> kshift;
         const uint32_t v = e < n_lo ? e : (e - n_lo + 1) << lo_bits;
         uint32_t x = 0;
+#pragma unroll 4
         for (uint32_t b = 0; b < cb; ++b) {
             const uint32_t t = ch * cb + b;
             if (t < n_in && ((v >> b) & 1u)) x ^= cols[(t << kshift) + k];
@@ -152,6 +182,12 @@ SQNN_DEV void build_tables(const DecodeArgs &A, uint32_t *tab)
         }
     }
     __syncthreads();
+}
+
+SQNN_DEV void build_tables(const DecodeArgs &A, uint32_t *tab)
+{
+    build_tables_begin(A, fetch_rows(A));
+    build_tables_finish(A, tab);
 }
 
 template <int NWP>

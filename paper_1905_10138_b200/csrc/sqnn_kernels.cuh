@@ -119,6 +119,10 @@ SQNN_DEV void cp_async16(void *sdst, const void *gsrc)
 {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" :: "r"(smem_addr(sdst)), "l"(gsrc) : "memory");
 }
+SQNN_DEV void cp_async4(void *sdst, const void *gsrc)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;\n" :: "r"(smem_addr(sdst)), "l"(gsrc) : "memory");
+}
 SQNN_DEV void cp_async_wait_all() { asm volatile("cp.async.wait_all;\n" ::: "memory"); }
 
 // Starts the copy of a tile's 32 * W mask words (first word gw0) into shared memory: 16-byte
@@ -282,9 +286,11 @@ k_decode_gemv(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__
     const bool mask_vec = (reinterpret_cast<uintptr_t>(mask32) & 15) == 0;
     const uint64_t tile_first = (uint64_t)blockIdx.x * ngroups + group, tile_step = (uint64_t)gridDim.x * ngroups;
 
-    // What a tile needs from global memory besides the activations -- its mask words, the scales
-    // of its first rows and this warp's seeds / patch offsets -- is requested before the tables
-    // are built, so that the two latencies overlap; later tiles are requested one tile ahead.
+    // Whatever the first tile needs from global memory is requested up front with nothing waiting
+    // on it -- the rows of M and this warp's seeds / patch offsets into registers, the tile's mask
+    // words, the scales of its first rows and the activations by asynchronous copies -- so that
+    // one memory latency covers them all; the d_patch words follow once the offsets are here.
+    const RowsAhead rows_ahead = fetch_rows(A);
     auto request = [&](uint64_t tile) {
         const uint64_t gw0 = tile * 32 * W;
         if (gw0 * 32 >= A.mn) return;
@@ -293,7 +299,8 @@ k_decode_gemv(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__
             const uint64_t r_first = gw0 * 32 / n;
             for (uint32_t i = lane; i < GEMV_ALPHA_WORDS; i += 32) {
                 const uint64_t at = r_first * n_q + i;
-                alpha_s[i] = at < alpha_count ? __ldg(alpha + at) : 0.0f;
+                if (at < alpha_count) cp_async4(alpha_s + i, alpha + at);
+                else alpha_s[i] = 0.0f;
             }
         }
     };
@@ -302,6 +309,7 @@ k_decode_gemv(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__
         if (tile_first < A.tiles && sub < n_q) tile_fetch<N_OUT, N_IN>(A.pl[sub], tile_first, lane, pre);
     }
     if (tile_first < A.tiles) request(tile_first);
+    uint32_t st_pre[4] = {0u, 0u, 0u, 0u};
 
     for (uint32_t bc = 0; bc < batch; bc += BT) {
         if constexpr (XS) {
@@ -310,8 +318,7 @@ k_decode_gemv(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__
                 constexpr uint32_t PER = 16 / sizeof(XT);
                 const uint4 *src = reinterpret_cast<const uint4 *>(x + (int64_t)bc * ldx);
                 uint4 *dst = reinterpret_cast<uint4 *>(xs);
-#pragma unroll 4
-                for (uint32_t v = threadIdx.x; v < n / PER; v += blockDim.x) dst[v] = __ldg(src + v);
+                for (uint32_t v = threadIdx.x; v < n / PER; v += blockDim.x) cp_async16(dst + v, src + v);
                 for (uint32_t c = (n / PER) * PER + threadIdx.x; c < n; c += blockDim.x) xs[c] = x[(int64_t)bc * ldx + c];
             } else {
 #pragma unroll 4
@@ -324,8 +331,17 @@ k_decode_gemv(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__
                 }
             }
         }
-        if (bc == 0) build_tables(A, smem);              // ends with a block barrier
-        else __syncthreads();
+        if (bc == 0) {
+            build_tables_begin(A, rows_ahead);           // block barrier: the first requests are back
+            if constexpr (N_OUT != 0) {
+                if (tile_first < A.tiles && sub < n_q) stage_fetch<N_OUT, N_IN>(A, A.pl[sub], pre, lane, st_pre);
+            }
+            cp_async_wait_all();
+            build_tables_finish(A, smem);                // ends with a block barrier
+        } else {
+            cp_async_wait_all();
+            __syncthreads();
+        }
         for (uint64_t tile = tile_first; tile < A.tiles; tile += tile_step) {
             const uint64_t gw0 = tile * 32 * W;          // first 32-bit word of the tile
             const uint64_t P0 = gw0 * 32;
@@ -336,10 +352,15 @@ k_decode_gemv(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__
             if constexpr (N_OUT != 0) {
                 for (uint32_t i = sub; i < n_q; i += wpt) {
                     TileIn<N_OUT, N_IN> in;
-                    if (i == sub && bc == 0 && tile == tile_first) in = pre;
-                    else tile_fetch<N_OUT, N_IN>(A.pl[i], tile, lane, in);
                     uint32_t st[4];
-                    stage_fetch<N_OUT, N_IN>(A, A.pl[i], in, lane, st);
+                    if (i == sub && bc == 0 && tile == tile_first) {
+                        in = pre;
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) st[q] = st_pre[q];
+                    } else {
+                        tile_fetch<N_OUT, N_IN>(A.pl[i], tile, lane, in);
+                        stage_fetch<N_OUT, N_IN>(A, A.pl[i], in, lane, st);
+                    }
                     tile_decode<N_OUT, N_IN>(A, A.pl[i], in, st, region + i * 32 * W, smem, stage, lane);
                 }
             } else {
