@@ -139,12 +139,18 @@ SQNN_DEV void build_tables_begin(const DecodeArgs &A, RowsAhead ahead)
     __syncthreads();
 }
 
+// N_OUT, N_IN: the network shape when it is known at compile time (the index arithmetic then folds), 0 = read it from A.
+template <int N_OUT = 0, int N_IN = 0>
 SQNN_DEV void build_tables_finish(const DecodeArgs &A, uint32_t *tab)
 {
     const uint32_t *rows_s = rows_scratch();
-    const uint32_t nwp = A.nwp, n_in = A.n_in, n_out = A.n_out, cb = A.cb;
+    constexpr bool CT = N_OUT != 0;
+    constexpr uint32_t NWP_C = entry_words_padded(CT ? N_OUT : 32);
+    const uint32_t nwp = CT ? NWP_C : A.nwp, n_in = CT ? (uint32_t)N_IN : A.n_in, n_out = CT ? (uint32_t)N_OUT : A.n_out;
+    const uint32_t cb = CT ? chunk_bits(CT ? N_IN : 8, NWP_C) : A.cb;
+    const uint32_t nchunks = CT ? table_chunks(CT ? N_IN : 8, NWP_C) : A.nchunks;
     const uint32_t kshift = nwp == 1 ? 0 : nwp == 2 ? 1 : nwp == 4 ? 2 : 3;
-    uint32_t *cols = tab + A.nchunks * (1u << cb) * nwp;
+    uint32_t *cols = tab + nchunks * (1u << cb) * nwp;
     // word k of column t: bit j of it is bit t of row 32 k + j -- one ballot over 32 rows
     const uint32_t lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
     for (uint32_t i = threadIdx.x >> 5; i < n_in * nwp; i += nwarps) {
@@ -158,7 +164,7 @@ SQNN_DEV void build_tables_finish(const DecodeArgs &A, uint32_t *tab)
     const uint32_t lo_bits = cb / 2, hi_bits = cb - lo_bits;
     const uint32_t n_lo = 1u << lo_bits, n_hi = 1u << hi_bits;
     const uint32_t direct = (n_lo + n_hi - 1) * nwp;          // per chunk: low-only and high-only entries
-    for (uint32_t i = threadIdx.x; i < A.nchunks * direct; i += blockDim.x) {
+    for (uint32_t i = threadIdx.x; i < nchunks * direct; i += blockDim.x) {
         const uint32_t ch = i / direct, r = i - ch * direct;
         const uint32_t k = r & (nwp - 1), e = r >> kshift;
         const uint32_t v = e < n_lo ? e : (e - n_lo + 1) << lo_bits;
@@ -171,7 +177,7 @@ SQNN_DEV void build_tables_finish(const DecodeArgs &A, uint32_t *tab)
         tab[((((ch << cb) | v)) << kshift) + k] = x;
     }
     __syncthreads();
-    const uint32_t total = A.nchunks * (1u << cb) * nwp;
+    const uint32_t total = nchunks * (1u << cb) * nwp;
     for (uint32_t i = threadIdx.x; i < total; i += blockDim.x) {
         const uint32_t k = i & (nwp - 1), e = i >> kshift;
         const uint32_t v = e & ((1u << cb) - 1u);
@@ -184,10 +190,11 @@ SQNN_DEV void build_tables_finish(const DecodeArgs &A, uint32_t *tab)
     __syncthreads();
 }
 
+template <int N_OUT = 0, int N_IN = 0>
 SQNN_DEV void build_tables(const DecodeArgs &A, uint32_t *tab)
 {
     build_tables_begin(A, fetch_rows(A));
-    build_tables_finish(A, tab);
+    build_tables_finish<N_OUT, N_IN>(A, tab);
 }
 
 template <int NWP>

@@ -39,7 +39,7 @@ __global__ void __launch_bounds__(512, 2)
 k_decode_bits(DecodeArgs A, uint64_t *__restrict__ out)
 {
     extern __shared__ __align__(16) uint32_t smem[];
-    build_tables(A, smem);
+    build_tables<N_OUT, N_IN>(A, smem);
     const uint32_t W = words_per_lane<N_OUT>(A);
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     const uint32_t per_warp = 32 * W + STAGE_WORDS;
@@ -152,7 +152,7 @@ k_decode_bf16(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__
               uint64_t n, __nv_bfloat16 *__restrict__ out)
 {
     extern __shared__ __align__(16) uint32_t smem[];
-    build_tables(A, smem);
+    build_tables<N_OUT, N_IN>(A, smem);
     const uint32_t W = words_per_lane<N_OUT>(A);
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     const uint32_t n_q = A.n_q;
@@ -244,10 +244,195 @@ SQNN_DEV void load_x(const XT *p, float (&v)[BT])
     for (int q = 0; q < BT; ++q) v[q] = to_float(pk.e[q]);
 }
 
-// Words of a row segment a lane works on at the same time in the GEMV kernel (build-time tunable).
-#ifndef SQNN_GEMV_WORDS_PER_ROUND
-#define SQNN_GEMV_WORDS_PER_ROUND 2
-#endif
+// Shared-memory accesses by 32-bit shared address (no generic-address arithmetic in the hot loop).
+SQNN_DEV uint32_t lds_u32(uint32_t a)
+{
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a));
+    return v;
+}
+// v = [a] if `take` is non-zero, otherwise v keeps its value.
+SQNN_DEV void lds_u32_if(uint32_t &v, uint32_t a, uint32_t take)
+{
+    asm volatile("{ .reg .pred q; setp.ne.u32 q, %2, 0; @q ld.shared.u32 %0, [%1]; }" : "+r"(v) : "r"(a), "r"(take));
+}
+// acc = v * x + acc if `live` is non-zero (a skipped lane must not touch acc: its x may be anything).
+SQNN_DEV void fma_if(float &acc, float v, float x, uint32_t live)
+{
+    asm("{ .reg .pred q; setp.ne.u32 q, %3, 0; @q fma.rn.f32 %0, %1, %2, %0; }" : "+f"(acc) : "f"(v), "f"(x), "r"(live));
+}
+// BT activations of one column from shared address a (xs[c][BT]).
+template <int BT, typename XT>
+SQNN_DEV void lds_x(uint32_t a, float (&v)[BT])
+{
+    if constexpr (sizeof(XT) == 2) {
+        if constexpr (BT == 1) {
+            unsigned short h;
+            asm volatile("ld.shared.u16 %0, [%1];" : "=h"(h) : "r"(a));
+            v[0] = __uint_as_float((uint32_t)h << 16);
+        } else if constexpr (BT == 2) {
+            const uint32_t w = lds_u32(a);
+            v[0] = __uint_as_float(w << 16); v[1] = __uint_as_float(w & 0xffff0000u);
+        } else if constexpr (BT == 4) {
+            uint32_t w0, w1;
+            asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(w0), "=r"(w1) : "r"(a));
+            v[0] = __uint_as_float(w0 << 16); v[1] = __uint_as_float(w0 & 0xffff0000u);
+            v[2] = __uint_as_float(w1 << 16); v[3] = __uint_as_float(w1 & 0xffff0000u);
+        } else {
+            static_assert(BT == 8, "batch chunk of 1, 2, 4 or 8");
+            uint32_t w[4];
+            asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "r"(a));
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                v[2 * q] = __uint_as_float(w[q] << 16);
+                v[2 * q + 1] = __uint_as_float(w[q] & 0xffff0000u);
+            }
+        }
+    } else {
+        if constexpr (BT == 1) {
+            v[0] = __uint_as_float(lds_u32(a));
+        } else if constexpr (BT == 2) {
+            asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(v[0]), "=f"(v[1]) : "r"(a));
+        } else {
+#pragma unroll
+            for (int q = 0; q < BT; q += 4)
+                asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                             : "=f"(v[q]), "=f"(v[q + 1]), "=f"(v[q + 2]), "=f"(v[q + 3]) : "r"(a + 4 * q));
+        }
+    }
+}
+
+// Head of one step of the walk below, written out instruction by instruction: takes the highest care bit
+// k of `mk` out of it (k = 0 and mk unchanged when there is none), reports in `live` whether there was
+// one, and forms the weight value (+-alpha_1) + (+-alpha_2) + ... from bit k of the plane words.
+SQNN_DEV void walk_head(uint32_t &mk, uint32_t &k, uint32_t &live, float &v, const uint32_t (&wb)[1],
+                        const float (&al)[1], const float (&ng)[1])
+{
+    asm("{\n .reg .pred pl, ps;\n .reg .b32 t, u;\n"
+        " mov.u32 %2, %3;\n setp.ne.u32 pl, %3, 0;\n bfind.u32 %0, %3;\n selp.u32 %0, %0, 0, pl;\n"
+        " shl.b32 t, 1, %0;\n @pl xor.b32 %3, %3, t;\n"
+        " and.b32 u, %4, t;\n setp.ne.u32 ps, u, 0;\n selp.f32 %1, %5, %6, ps;\n}"
+        : "=&r"(k), "=&f"(v), "=&r"(live), "+r"(mk) : "r"(wb[0]), "f"(al[0]), "f"(ng[0]));
+}
+SQNN_DEV void walk_head(uint32_t &mk, uint32_t &k, uint32_t &live, float &v, const uint32_t (&wb)[2],
+                        const float (&al)[2], const float (&ng)[2])
+{
+    asm("{\n .reg .pred pl, ps;\n .reg .b32 t, u;\n .reg .f32 w;\n"
+        " mov.u32 %2, %3;\n setp.ne.u32 pl, %3, 0;\n bfind.u32 %0, %3;\n selp.u32 %0, %0, 0, pl;\n"
+        " shl.b32 t, 1, %0;\n @pl xor.b32 %3, %3, t;\n"
+        " and.b32 u, %4, t;\n setp.ne.u32 ps, u, 0;\n selp.f32 %1, %6, %8, ps;\n"
+        " and.b32 u, %5, t;\n setp.ne.u32 ps, u, 0;\n selp.f32 w, %7, %9, ps;\n add.rn.f32 %1, %1, w;\n}"
+        : "=&r"(k), "=&f"(v), "=&r"(live), "+r"(mk)
+        : "r"(wb[0]), "r"(wb[1]), "f"(al[0]), "f"(al[1]), "f"(ng[0]), "f"(ng[1]));
+}
+SQNN_DEV void walk_head(uint32_t &mk, uint32_t &k, uint32_t &live, float &v, const uint32_t (&wb)[3],
+                        const float (&al)[3], const float (&ng)[3])
+{
+    asm("{\n .reg .pred pl, ps;\n .reg .b32 t, u;\n .reg .f32 w;\n"
+        " mov.u32 %2, %3;\n setp.ne.u32 pl, %3, 0;\n bfind.u32 %0, %3;\n selp.u32 %0, %0, 0, pl;\n"
+        " shl.b32 t, 1, %0;\n @pl xor.b32 %3, %3, t;\n"
+        " and.b32 u, %4, t;\n setp.ne.u32 ps, u, 0;\n selp.f32 %1, %7, %10, ps;\n"
+        " and.b32 u, %5, t;\n setp.ne.u32 ps, u, 0;\n selp.f32 w, %8, %11, ps;\n add.rn.f32 %1, %1, w;\n"
+        " and.b32 u, %6, t;\n setp.ne.u32 ps, u, 0;\n selp.f32 w, %9, %12, ps;\n add.rn.f32 %1, %1, w;\n}"
+        : "=&r"(k), "=&f"(v), "=&r"(live), "+r"(mk)
+        : "r"(wb[0]), "r"(wb[1]), "r"(wb[2]), "f"(al[0]), "f"(al[1]), "f"(al[2]), "f"(ng[0]), "f"(ng[1]), "f"(ng[2]));
+}
+
+// Tail of one step of the walk: when the lane's word is used up (mk == 0) it moves to its next word at
+// shared address wa + step_a if that is still inside the segment (<= hi_a) -- mask word into mk (the
+// segment's last word trimmed by last_mask), plane words into wb, xa advanced by step_x -- and is done
+// otherwise (it then stays where it is).  Returns, the same in every lane, whether any lane is not done.
+// Plane i's word lies (NQ - i) * plane_bytes below the mask word.
+SQNN_DEV uint32_t walk_tail(uint32_t &mk, uint32_t &wa, uint32_t &xa, uint32_t (&wb)[1], uint32_t step_a,
+                            uint32_t hi_a, uint32_t step_x, uint32_t plane_bytes, uint32_t last_mask)
+{
+    uint32_t cont;
+    asm volatile("{\n .reg .pred pz, pt, pd, pa, pq;\n .reg .b32 na, a0;\n"
+        " setp.eq.u32 pz, %1, 0;\n add.u32 na, %2, %5;\n setp.le.and.u32 pt, na, %6, pz;\n"
+        " setp.gt.and.u32 pd, na, %6, pz;\n vote.sync.any.pred pa, !pd, 0xffffffff;\n selp.u32 %0, 1, 0, pa;\n"
+        " sub.u32 a0, na, %8;\n"
+        " @pt ld.shared.u32 %1, [na];\n @pt ld.shared.u32 %4, [a0];\n"
+        " @pt mov.u32 %2, na;\n @pt add.u32 %3, %3, %7;\n"
+        " setp.eq.and.u32 pq, na, %6, pt;\n @pq and.b32 %1, %1, %9;\n}"
+        : "=&r"(cont), "+r"(mk), "+r"(wa), "+r"(xa), "+r"(wb[0])
+        : "r"(step_a), "r"(hi_a), "r"(step_x), "r"(plane_bytes), "r"(last_mask));
+    return cont;
+}
+SQNN_DEV uint32_t walk_tail(uint32_t &mk, uint32_t &wa, uint32_t &xa, uint32_t (&wb)[2], uint32_t step_a,
+                            uint32_t hi_a, uint32_t step_x, uint32_t plane_bytes, uint32_t last_mask)
+{
+    uint32_t cont;
+    asm volatile("{\n .reg .pred pz, pt, pd, pa, pq;\n .reg .b32 na, a0, a1;\n"
+        " setp.eq.u32 pz, %1, 0;\n add.u32 na, %2, %6;\n setp.le.and.u32 pt, na, %7, pz;\n"
+        " setp.gt.and.u32 pd, na, %7, pz;\n vote.sync.any.pred pa, !pd, 0xffffffff;\n selp.u32 %0, 1, 0, pa;\n"
+        " sub.u32 a1, na, %9;\n sub.u32 a0, a1, %9;\n"
+        " @pt ld.shared.u32 %1, [na];\n @pt ld.shared.u32 %4, [a0];\n @pt ld.shared.u32 %5, [a1];\n"
+        " @pt mov.u32 %2, na;\n @pt add.u32 %3, %3, %8;\n"
+        " setp.eq.and.u32 pq, na, %7, pt;\n @pq and.b32 %1, %1, %10;\n}"
+        : "=&r"(cont), "+r"(mk), "+r"(wa), "+r"(xa), "+r"(wb[0]), "+r"(wb[1])
+        : "r"(step_a), "r"(hi_a), "r"(step_x), "r"(plane_bytes), "r"(last_mask));
+    return cont;
+}
+SQNN_DEV uint32_t walk_tail(uint32_t &mk, uint32_t &wa, uint32_t &xa, uint32_t (&wb)[3], uint32_t step_a,
+                            uint32_t hi_a, uint32_t step_x, uint32_t plane_bytes, uint32_t last_mask)
+{
+    uint32_t cont;
+    asm volatile("{\n .reg .pred pz, pt, pd, pa, pq;\n .reg .b32 na, a0, a1, a2;\n"
+        " setp.eq.u32 pz, %1, 0;\n add.u32 na, %2, %7;\n setp.le.and.u32 pt, na, %8, pz;\n"
+        " setp.gt.and.u32 pd, na, %8, pz;\n vote.sync.any.pred pa, !pd, 0xffffffff;\n selp.u32 %0, 1, 0, pa;\n"
+        " sub.u32 a2, na, %10;\n sub.u32 a1, a2, %10;\n sub.u32 a0, a1, %10;\n"
+        " @pt ld.shared.u32 %1, [na];\n @pt ld.shared.u32 %4, [a0];\n @pt ld.shared.u32 %5, [a1];\n @pt ld.shared.u32 %6, [a2];\n"
+        " @pt mov.u32 %2, na;\n @pt add.u32 %3, %3, %9;\n"
+        " setp.eq.and.u32 pq, na, %8, pt;\n @pq and.b32 %1, %1, %11;\n}"
+        : "=&r"(cont), "+r"(mk), "+r"(wa), "+r"(xa), "+r"(wb[0]), "+r"(wb[1]), "+r"(wb[2])
+        : "r"(step_a), "r"(hi_a), "r"(step_x), "r"(plane_bytes), "r"(last_mask));
+    return cont;
+}
+
+// The walk of one row segment of a decoded tile (GEMV kernel), activations in shared memory as xs[c][BT].
+// Each lane walks its own words of the segment -- word `lw`, then every `wstep`-th up to `lw_hi` -- from
+// the highest care bit down, and moves on to its next word as soon as the current one is used up: lanes
+// do not wait for one another between words, so the warp runs for as long as its busiest lane has care
+// bits.  The body is free of branches under a warp-uniform loop condition, so the lanes stay converged.
+// Only care positions contribute; an idle lane's load stays inside shared memory and its result is dropped.
+//   mask_sa      shared address of the tile's mask words; plane i's words lie (NQ - i) * plane_bytes below
+//   xs_sa        shared address of xs[0]
+//   c_tile       column (in this row) of bit 0 of the tile; may be negative
+template <int BT, typename XT, int NQ>
+SQNN_DEV void walk_segment(uint32_t mask_sa, uint32_t plane_bytes, uint32_t xs_sa, uint32_t lw, uint32_t lw_lo,
+                           uint32_t lw_hi, uint32_t wstep, uint32_t first_mask, uint32_t last_mask, int32_t c_tile,
+                           const float (&al)[NQ], float (&acc)[BT])
+{
+    constexpr uint32_t XB = BT * sizeof(XT);                 // bytes of one column of xs
+    const uint32_t hi_a = mask_sa + 4 * lw_hi;
+    const uint32_t step_a = 4 * wstep, step_x = 32 * XB * wstep;
+    uint32_t wa = mask_sa + 4 * lw;                          // shared address of the lane's current mask word
+    uint32_t xa = xs_sa + (uint32_t)(c_tile + (int32_t)(32 * lw)) * XB;    // ... of the column of its bit 0
+    const uint32_t more = lw <= lw_hi ? 1u : 0u;
+    uint32_t mk = 0, wb[NQ];
+#pragma unroll
+    for (int i = 0; i < NQ; ++i) wb[i] = 0;
+    lds_u32_if(mk, wa, more);
+#pragma unroll
+    for (int i = 0; i < NQ; ++i) lds_u32_if(wb[i], wa - (NQ - i) * plane_bytes, more);
+    if (lw == lw_lo) mk &= first_mask;
+    if (lw == lw_hi) mk &= last_mask;
+    // a lane without a word in this segment parks on the segment's last word with nothing to do
+    if (!more) { wa = hi_a; xa = xs_sa + (uint32_t)(c_tile + (int32_t)(32 * lw_hi)) * XB; }
+    float ng[NQ];
+#pragma unroll
+    for (int i = 0; i < NQ; ++i) ng[i] = -al[i];
+    uint32_t cont = __any_sync(0xffffffffu, more != 0) ? 1u : 0u;
+    while (cont) {
+        uint32_t k, live;
+        float v, xv[BT];
+        walk_head(mk, k, live, v, wb, al, ng);
+        lds_x<BT, XT>(xa + k * XB, xv);
+#pragma unroll
+        for (int q = 0; q < BT; ++q) fma_if(acc[q], v, xv[q], live);
+        cont = walk_tail(mk, wa, xa, wb, step_a, hi_a, step_x, plane_bytes, last_mask);
+    }
+}
 
 // Words of per-warp scratch the GEMV kernel keeps for the scales of the rows a tile touches.
 constexpr uint32_t GEMV_ALPHA_WORDS = 64;
@@ -337,7 +522,7 @@ k_decode_gemv(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__
                 if (tile_first < A.tiles && sub < n_q) stage_fetch<N_OUT, N_IN>(A, A.pl[sub], pre, lane, st_pre);
             }
             cp_async_wait_all();
-            build_tables_finish(A, smem);                // ends with a block barrier
+            build_tables_finish<N_OUT, N_IN>(A, smem);   // ends with a block barrier
         } else {
             cp_async_wait_all();
             __syncthreads();
@@ -373,95 +558,91 @@ k_decode_gemv(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__
             // Y is cleared by the kernel before this one in the stream; under a programmatic dependent
             // launch this is where its results are awaited (a no-op otherwise)
             asm volatile("griddepcontrol.wait;" ::: "memory");
-            for (uint64_t r = r_first; r * n < P1; ++r) {
-                const uint64_t a = r * n > P0 ? r * n : P0;
-                const uint64_t b = (r + 1) * n < P1 ? (r + 1) * n : P1;
+            // row segments of the tile, in tile-local bit coordinates [a_loc, b_loc); c_tile is the column
+            // (in the segment's row) of tile bit 0 and goes negative from the second row on
+            const uint32_t T = (uint32_t)(P1 - P0);
+            uint32_t a_loc = 0, ai = 0;
+            int32_t c_tile = (int32_t)(P0 - r_first * n);
+            for (uint64_t r = r_first; a_loc < T; ++r, ai += n_q, c_tile -= (int32_t)n) {
+                uint32_t b_loc = (uint32_t)((int32_t)n - c_tile);
+                b_loc = b_loc < T ? b_loc : T;
                 constexpr int NR = NQ > 0 ? NQ : 1;
                 float al[NR];
-                const uint32_t ai = (uint32_t)(r - r_first) * n_q;
                 if constexpr (NQ > 0) {
 #pragma unroll
                     for (int i = 0; i < NQ; ++i)
                         al[i] = ai + i < GEMV_ALPHA_WORDS ? alpha_s[ai + i] : __ldg(alpha + r * n_q + i);
                 }
-                const uint32_t lw_lo = (uint32_t)((a >> 5) - gw0), lw_hi = (uint32_t)(((b - 1) >> 5) - gw0);
-                const int32_t c_tile = (int32_t)((int64_t)P0 - (int64_t)(r * n));   // column of tile bit 0
-                const uint32_t a_loc = (uint32_t)(a - P0), b_loc = (uint32_t)(b - P0);
+                const uint32_t lw_lo = a_loc >> 5, lw_hi = (b_loc - 1) >> 5;
                 float acc[BT];
 #pragma unroll
                 for (int q = 0; q < BT; ++q) acc[q] = 0.0f;
-                // a lane takes up to four of the segment's words at a time and visits one set mask
-                // bit of each per round: four independent chains of shared-memory reads
-                constexpr uint32_t K = SQNN_GEMV_WORDS_PER_ROUND;
                 const uint32_t wstep = 32 * wpt;
-                for (uint32_t lw0 = lw_lo + sub * 32 + lane; lw0 <= lw_hi; lw0 += wstep * K) {
-                    uint32_t mk[K], wb[K][NR], k_idle[K];
-                    int32_t cb[K];
-                    uint32_t any = 0;
+                const uint32_t first_mask = 0xffffffffu << (a_loc & 31u);
+                const uint32_t last_mask = 0xffffffffu >> (31u - ((b_loc - 1u) & 31u));
+                uint32_t lw = lw_lo + sub * 32 + lane;
+                if constexpr (XS && NQ > 0) {
+                    walk_segment<BT, XT, NQ>(smem_addr(mask_s), 128 * W, smem_addr(xs), lw, lw_lo, lw_hi, wstep,
+                                             first_mask, last_mask, c_tile, al, acc);
+                } else {
+                // the same walk in plain C++ for any number of planes and for activations left in global memory
+                uint32_t mk = 0, wb[NR];
+                int32_t cbase = 0;
 #pragma unroll
-                    for (uint32_t j = 0; j < K; ++j) {
-                        const uint32_t lw = lw0 + j * wstep;
-                        mk[j] = 0;
-                        cb[j] = c_tile + (int32_t)a_loc;    // a valid column for the idle slots
-                        k_idle[j] = 0;
+                for (int i = 0; i < NR; ++i) wb[i] = 0;
+                auto take_word = [&]() {
+                    uint32_t m = mask_s[lw];
+                    if (lw == lw_lo) m &= first_mask;
+                    if (lw == lw_hi) m &= last_mask;
+                    mk = m;
+                    cbase = c_tile + (int32_t)(lw * 32);
+                    if constexpr (NQ > 0) {
 #pragma unroll
-                        for (int i = 0; i < NR; ++i) wb[j][i] = 0;
-                        if (lw <= lw_hi) {
-                            uint32_t m = mask_s[lw];
-                            const uint32_t lo = lw * 32;
-                            if (lo < a_loc) {
-                                m &= 0xffffffffu << (a_loc - lo);
-                                k_idle[j] = a_loc - lo;     // bit 0 of this word belongs to the row before
-                            }
-                            if (lo + 32 > b_loc) m &= 0xffffffffu >> (lo + 32 - b_loc);
-                            mk[j] = m;
-                            cb[j] = c_tile + (int32_t)lo;
-                            if constexpr (NQ > 0) {
-#pragma unroll
-                                for (int i = 0; i < NQ; ++i) wb[j][i] = region[i * 32 * W + lw];
-                            } else {
-                                wb[j][0] = lw;
-                            }
-                        }
-                        any |= mk[j];
+                        for (int i = 0; i < NQ; ++i) wb[i] = region[i * 32 * W + lw];
+                    } else {
+                        wb[0] = lw;
                     }
-                    while (any) {
-                        any = 0;
-                        // branch-free: an exhausted word contributes value 0 at a column of this row
-                        // (0 * x must not meet an x read from outside the row: it could be Inf or NaN)
+                };
+                bool more = lw <= lw_hi;
+                if (more) take_word();
+                const int32_t c_safe = c_tile + (int32_t)a_loc;     // a column of this row, for idle lanes
+                // branch-free body under a warp-uniform loop condition: the lanes stay converged
+                while (__any_sync(0xffffffffu, more)) {
+                    const bool live = mk != 0;
+                    const uint32_t k = live ? 31u - (uint32_t)__clz((int)mk) : 0u;
+                    const uint32_t bit = live ? 1u << k : 0u;
+                    mk ^= bit;
+                    float v = 0.0f;
+                    if constexpr (NQ > 0) {
 #pragma unroll
-                        for (uint32_t j = 0; j < K; ++j) {
-                            const bool live = mk[j] != 0;
-                            const uint32_t k = live ? 31u - (uint32_t)__clz((int)mk[j]) : k_idle[j];
-                            mk[j] &= ~(1u << k);
-                            float v = 0.0f;
-                            if constexpr (NQ > 0) {
-#pragma unroll
-                                for (int i = 0; i < NQ; ++i) {
-                                    const float t = ((wb[j][i] >> k) & 1u) ? al[i] : -al[i];
-                                    v = i == 0 ? t : v + t;
-                                }
-                            } else {
-                                for (uint32_t i = 0; i < n_q; ++i) {
-                                    const float a1 = __ldg(alpha + r * n_q + i);
-                                    v += ((region[i * 32 * W + wb[j][0]] >> k) & 1u) ? a1 : -a1;
-                                }
-                            }
-                            v = live ? v : 0.0f;
-                            const int32_t c = cb[j] + (int32_t)k;
-                            if constexpr (XS) {
-                                float xv[BT];
-                                load_x<BT, XT>(xs + (uint32_t)c * BT, xv);
-#pragma unroll
-                                for (int q = 0; q < BT; ++q) acc[q] = fmaf(v, xv[q], acc[q]);
-                            } else {
-#pragma unroll
-                                for (int q = 0; q < BT; ++q)
-                                    if (bc + q < batch) acc[q] = fmaf(v, to_float(x[(int64_t)(bc + q) * ldx + c]), acc[q]);
-                            }
-                            any |= mk[j];
+                        for (int i = 0; i < NQ; ++i) {
+                            const float t = (wb[i] & bit) ? al[i] : -al[i];
+                            v = i == 0 ? t : v + t;
+                        }
+                    } else {
+                        for (uint32_t i = 0; i < n_q; ++i) {
+                            const float a1 = __ldg(alpha + r * n_q + i);
+                            v += (region[i * 32 * W + wb[0]] & bit) ? a1 : -a1;
                         }
                     }
+                    v = live ? v : 0.0f;
+                    const int32_t c = live ? cbase + (int32_t)k : c_safe;
+                    if constexpr (XS) {
+                        float xv[BT];
+                        load_x<BT, XT>(xs + (uint32_t)c * BT, xv);
+#pragma unroll
+                        for (int q = 0; q < BT; ++q) acc[q] = fmaf(v, xv[q], acc[q]);
+                    } else {
+#pragma unroll
+                        for (int q = 0; q < BT; ++q)
+                            if (bc + q < batch) acc[q] = fmaf(v, to_float(x[(int64_t)(bc + q) * ldx + c]), acc[q]);
+                    }
+                    if (mk == 0 && more) {
+                        lw += wstep;
+                        more = lw <= lw_hi;
+                        if (more) take_word();
+                    }
+                }
                 }
 #pragma unroll
                 for (int q = 0; q < BT; ++q) {
@@ -470,6 +651,7 @@ k_decode_gemv(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__
                     for (uint32_t d = 16; d >= 1; d >>= 1) s += __shfl_xor_sync(0xffffffffu, s, d);
                     if (lane == 0 && bc + q < batch) atomicAdd(y + (int64_t)(bc + q) * ldy + r, s);
                 }
+                a_loc = b_loc;
             }
             if (wpt == 1) __syncwarp();                  // the group is done with its regions
             else asm volatile("bar.sync %0, %1;\n" :: "r"(1 + group), "r"(32 * wpt) : "memory");
@@ -553,16 +735,17 @@ template <int N_OUT, int N_IN, int BT, typename XT>
 inline int launch_gemv_bt(const DecodeArgs &A, const uint64_t *d_mask, const float *d_alpha, const void *d_x,
                           int64_t ldx, uint32_t batch, float *d_y, int64_t ldy, uint64_t n, cudaStream_t st)
 {
-    // Aim at ~32 warps per SM: with few tiles, up to 4 warps share a tile; a block holds up to
-    // 15 tile groups (named barriers) and 20 warps.
+    // One tile group per tile an SM gets (up to 15, the named barriers), and as many warps per group
+    // (up to 4) as fit a block of 20 warps -- as long as a row still gives every lane of the group a word.
+    // (More warps per block at fewer registers were slower: every warp repeats the per-tile bookkeeping.)
     const uint64_t live = (A.words64 * 2 + 32ull * A.W - 1) / (32ull * A.W);
     const uint32_t sms = (uint32_t)sm_count();
-    uint32_t wpt = 1;
-    // (only while a row still gives every lane of the group at least two words)
-    while (wpt < 4 && live * wpt * 2 <= 32ull * sms && n >= 2048ull * wpt * 2) wpt *= 2;
+    constexpr uint32_t max_warps = 20;
     uint32_t groups = (uint32_t)((live + sms - 1) / sms);
-    const uint32_t max_groups = 20 / wpt < 15 ? 20 / wpt : 15;
-    groups = groups < 1 ? 1 : groups > max_groups ? max_groups : groups;
+    groups = groups < 1 ? 1 : groups > 15 ? 15 : groups;
+    uint32_t wpt = max_warps / groups;
+    wpt = wpt < 1 ? 1 : wpt > 4 ? 4 : wpt;
+    while (wpt > 1 && n < 1024ull * wpt) --wpt;
     if (wpt == 1 && groups < 4) groups = 4;
     const size_t tab = (size_t)table_words(A.n_in, A.nwp, A.nchunks, A.cb) * 4;
     const size_t per_group = ((size_t)(A.n_q + 1) * 32 * A.W + GEMV_ALPHA_WORDS + (size_t)wpt * STAGE_WORDS) * 4;
