@@ -303,38 +303,46 @@ SQNN_DEV void lds_x(uint32_t a, float (&v)[BT])
 }
 
 // Head of one step of the walk below, written out instruction by instruction: takes the highest care bit
-// k of `mk` out of it (k = 0 and mk unchanged when there is none), reports in `live` whether there was
-// one, and forms the weight value (+-alpha_1) + (+-alpha_2) + ... from bit k of the plane words.
-SQNN_DEV void walk_head(uint32_t &mk, uint32_t &k, uint32_t &live, float &v, const uint32_t (&wb)[1],
-                        const float (&al)[1], const float (&ng)[1])
-{
-    asm("{\n .reg .pred pl, ps;\n .reg .b32 t, u;\n"
-        " mov.u32 %2, %3;\n setp.ne.u32 pl, %3, 0;\n bfind.u32 %0, %3;\n selp.u32 %0, %0, 0, pl;\n"
-        " shl.b32 t, 1, %0;\n @pl xor.b32 %3, %3, t;\n"
-        " and.b32 u, %4, t;\n setp.ne.u32 ps, u, 0;\n selp.f32 %1, %5, %6, ps;\n}"
-        : "=&r"(k), "=&f"(v), "=&r"(live), "+r"(mk) : "r"(wb[0]), "f"(al[0]), "f"(ng[0]));
-}
-SQNN_DEV void walk_head(uint32_t &mk, uint32_t &k, uint32_t &live, float &v, const uint32_t (&wb)[2],
-                        const float (&al)[2], const float (&ng)[2])
+// k1 and then the lowest care bit k2 out of `mk` (k = 0 where there is none), reports in live1 / live2
+// whether there was one, and forms the weight values (+-alpha_1) + (+-alpha_2) + ... from bits k1 and k2
+// of the plane words.
+SQNN_DEV void walk_head(uint32_t &mk, uint32_t &k1, uint32_t &live1, float &v1, uint32_t &k2, uint32_t &live2,
+                        float &v2, const uint32_t (&wb)[1], const float (&al)[1], const float (&ng)[1])
 {
     asm("{\n .reg .pred pl, ps;\n .reg .b32 t, u;\n .reg .f32 w;\n"
-        " mov.u32 %2, %3;\n setp.ne.u32 pl, %3, 0;\n bfind.u32 %0, %3;\n selp.u32 %0, %0, 0, pl;\n"
-        " shl.b32 t, 1, %0;\n @pl xor.b32 %3, %3, t;\n"
-        " and.b32 u, %4, t;\n setp.ne.u32 ps, u, 0;\n selp.f32 %1, %6, %8, ps;\n"
-        " and.b32 u, %5, t;\n setp.ne.u32 ps, u, 0;\n selp.f32 w, %7, %9, ps;\n add.rn.f32 %1, %1, w;\n}"
-        : "=&r"(k), "=&f"(v), "=&r"(live), "+r"(mk)
+        " mov.u32 %2, %6;\n setp.ne.u32 pl, %6, 0;\n bfind.u32 %0, %6;\n selp.u32 %0, %0, 0, pl;\n"
+        " shl.b32 t, 1, %0;\n @pl xor.b32 %6, %6, t;\n"
+        " and.b32 u, %7, t;\n setp.ne.u32 ps, u, 0;\n selp.f32 %1, %8, %9, ps;\n"
+        " neg.s32 t, %6;\n and.b32 t, t, %6;\n mov.u32 %5, t;\n bfind.u32 %3, t;\n setp.ne.u32 pl, t, 0;\n"
+        " selp.u32 %3, %3, 0, pl;\n xor.b32 %6, %6, t;\n"
+        " and.b32 u, %7, t;\n setp.ne.u32 ps, u, 0;\n selp.f32 %4, %8, %9, ps;\n}"
+        : "=&r"(k1), "=&f"(v1), "=&r"(live1), "=&r"(k2), "=&f"(v2), "=&r"(live2), "+r"(mk)
+        : "r"(wb[0]), "f"(al[0]), "f"(ng[0]));
+}
+SQNN_DEV void walk_head(uint32_t &mk, uint32_t &k1, uint32_t &live1, float &v1, uint32_t &k2, uint32_t &live2,
+                        float &v2, const uint32_t (&wb)[2], const float (&al)[2], const float (&ng)[2])
+{
+    asm("{\n .reg .pred pl, ps;\n .reg .b32 t, u;\n .reg .f32 w;\n"
+        " mov.u32 %2, %6;\n setp.ne.u32 pl, %6, 0;\n bfind.u32 %0, %6;\n selp.u32 %0, %0, 0, pl;\n"
+        " shl.b32 t, 1, %0;\n @pl xor.b32 %6, %6, t;\n"
+        " and.b32 u, %7, t;\n setp.ne.u32 ps, u, 0;\n selp.f32 %1, %9, %11, ps;\n and.b32 u, %8, t;\n setp.ne.u32 ps, u, 0;\n selp.f32 w, %10, %12, ps;\n add.rn.f32 %1, %1, w;\n"
+        " neg.s32 t, %6;\n and.b32 t, t, %6;\n mov.u32 %5, t;\n bfind.u32 %3, t;\n setp.ne.u32 pl, t, 0;\n"
+        " selp.u32 %3, %3, 0, pl;\n xor.b32 %6, %6, t;\n"
+        " and.b32 u, %7, t;\n setp.ne.u32 ps, u, 0;\n selp.f32 %4, %9, %11, ps;\n and.b32 u, %8, t;\n setp.ne.u32 ps, u, 0;\n selp.f32 w, %10, %12, ps;\n add.rn.f32 %4, %4, w;\n}"
+        : "=&r"(k1), "=&f"(v1), "=&r"(live1), "=&r"(k2), "=&f"(v2), "=&r"(live2), "+r"(mk)
         : "r"(wb[0]), "r"(wb[1]), "f"(al[0]), "f"(al[1]), "f"(ng[0]), "f"(ng[1]));
 }
-SQNN_DEV void walk_head(uint32_t &mk, uint32_t &k, uint32_t &live, float &v, const uint32_t (&wb)[3],
-                        const float (&al)[3], const float (&ng)[3])
+SQNN_DEV void walk_head(uint32_t &mk, uint32_t &k1, uint32_t &live1, float &v1, uint32_t &k2, uint32_t &live2,
+                        float &v2, const uint32_t (&wb)[3], const float (&al)[3], const float (&ng)[3])
 {
     asm("{\n .reg .pred pl, ps;\n .reg .b32 t, u;\n .reg .f32 w;\n"
-        " mov.u32 %2, %3;\n setp.ne.u32 pl, %3, 0;\n bfind.u32 %0, %3;\n selp.u32 %0, %0, 0, pl;\n"
-        " shl.b32 t, 1, %0;\n @pl xor.b32 %3, %3, t;\n"
-        " and.b32 u, %4, t;\n setp.ne.u32 ps, u, 0;\n selp.f32 %1, %7, %10, ps;\n"
-        " and.b32 u, %5, t;\n setp.ne.u32 ps, u, 0;\n selp.f32 w, %8, %11, ps;\n add.rn.f32 %1, %1, w;\n"
-        " and.b32 u, %6, t;\n setp.ne.u32 ps, u, 0;\n selp.f32 w, %9, %12, ps;\n add.rn.f32 %1, %1, w;\n}"
-        : "=&r"(k), "=&f"(v), "=&r"(live), "+r"(mk)
+        " mov.u32 %2, %6;\n setp.ne.u32 pl, %6, 0;\n bfind.u32 %0, %6;\n selp.u32 %0, %0, 0, pl;\n"
+        " shl.b32 t, 1, %0;\n @pl xor.b32 %6, %6, t;\n"
+        " and.b32 u, %7, t;\n setp.ne.u32 ps, u, 0;\n selp.f32 %1, %10, %13, ps;\n and.b32 u, %8, t;\n setp.ne.u32 ps, u, 0;\n selp.f32 w, %11, %14, ps;\n add.rn.f32 %1, %1, w;\n and.b32 u, %9, t;\n setp.ne.u32 ps, u, 0;\n selp.f32 w, %12, %15, ps;\n add.rn.f32 %1, %1, w;\n"
+        " neg.s32 t, %6;\n and.b32 t, t, %6;\n mov.u32 %5, t;\n bfind.u32 %3, t;\n setp.ne.u32 pl, t, 0;\n"
+        " selp.u32 %3, %3, 0, pl;\n xor.b32 %6, %6, t;\n"
+        " and.b32 u, %7, t;\n setp.ne.u32 ps, u, 0;\n selp.f32 %4, %10, %13, ps;\n and.b32 u, %8, t;\n setp.ne.u32 ps, u, 0;\n selp.f32 w, %11, %14, ps;\n add.rn.f32 %4, %4, w;\n and.b32 u, %9, t;\n setp.ne.u32 ps, u, 0;\n selp.f32 w, %12, %15, ps;\n add.rn.f32 %4, %4, w;\n}"
+        : "=&r"(k1), "=&f"(v1), "=&r"(live1), "=&r"(k2), "=&f"(v2), "=&r"(live2), "+r"(mk)
         : "r"(wb[0]), "r"(wb[1]), "r"(wb[2]), "f"(al[0]), "f"(al[1]), "f"(al[2]), "f"(ng[0]), "f"(ng[1]), "f"(ng[2]));
 }
 
@@ -391,7 +399,7 @@ SQNN_DEV uint32_t walk_tail(uint32_t &mk, uint32_t &wa, uint32_t &xa, uint32_t (
 
 // The walk of one row segment of a decoded tile (GEMV kernel), activations in shared memory as xs[c][BT].
 // Each lane walks its own words of the segment -- word `lw`, then every `wstep`-th up to `lw_hi` -- from
-// the highest care bit down, and moves on to its next word as soon as the current one is used up: lanes
+// both ends (two care bits a step), and moves on to its next word as soon as the current one is used up: lanes
 // do not wait for one another between words, so the warp runs for as long as its busiest lane has care
 // bits.  The body is free of branches under a warp-uniform loop condition, so the lanes stay converged.
 // Only care positions contribute; an idle lane's load stays inside shared memory and its result is dropped.
@@ -424,12 +432,15 @@ SQNN_DEV void walk_segment(uint32_t mask_sa, uint32_t plane_bytes, uint32_t xs_s
     for (int i = 0; i < NQ; ++i) ng[i] = -al[i];
     uint32_t cont = __any_sync(0xffffffffu, more != 0) ? 1u : 0u;
     while (cont) {
-        uint32_t k, live;
-        float v, xv[BT];
-        walk_head(mk, k, live, v, wb, al, ng);
-        lds_x<BT, XT>(xa + k * XB, xv);
+        uint32_t k1, k2, live1, live2;
+        float v1, v2, xv1[BT], xv2[BT];
+        walk_head(mk, k1, live1, v1, k2, live2, v2, wb, al, ng);
+        lds_x<BT, XT>(xa + k1 * XB, xv1);
+        lds_x<BT, XT>(xa + k2 * XB, xv2);
 #pragma unroll
-        for (int q = 0; q < BT; ++q) fma_if(acc[q], v, xv[q], live);
+        for (int q = 0; q < BT; ++q) fma_if(acc[q], v1, xv1[q], live1);
+#pragma unroll
+        for (int q = 0; q < BT; ++q) fma_if(acc[q], v2, xv2[q], live2);
         cont = walk_tail(mk, wa, xa, wb, step_a, hi_a, step_x, plane_bytes, last_mask);
     }
 }
