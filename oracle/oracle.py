@@ -59,6 +59,10 @@ def _L():
         lib.orc_reconstruct.argtypes = [i64, i64, i32, vp, vp, vp, vp, vp]
         lib.orc_matmul.argtypes = [i64, i64, i32, vp, vp, vp, vp, i64, vp]
         lib.orc_eq1.argtypes = [i64, i32, i32, vp, vp]
+        lib.orc_eq1_blocked.argtypes = [i64, i32, i32, vp, i64, vp]
+        lib.orc_fifo_model.argtypes = [i64, vp, i32, i32, i32, vp]
+        lib.orc_csr_relative_time.argtypes = [i64, vp, i32]
+        lib.orc_csr_relative_time.restype = ctypes.c_double
         _lib = lib
     return _lib
 
@@ -202,3 +206,30 @@ def eq1(mn: int, n_out: int, n_in: int, np_) -> dict:
     _L().orc_eq1(mn, n_out, n_in, _p(np_), _p(out))
     return {"r": out[0], "bits_wc": out[1], "bits_npatch": out[2], "bits_dpatch": out[3],
             "max_p": int(out[4]), "sum_p": int(out[5]), "bits_per_weight": 1.0 / out[0]}
+
+
+def eq1_blocked(mn: int, n_out: int, n_in: int, np_, block: int) -> dict:
+    """Eq. 1 with the n_patch width chosen per block of `block` slices (Section 5.2)."""
+    np_ = np.ascontiguousarray(np_, dtype=np.uint16)
+    assert np_.size == (mn + n_out - 1) // n_out and block >= 1
+    out = np.zeros(4, dtype=np.float64)
+    _L().orc_eq1_blocked(mn, n_out, n_in, _p(np_), block, _p(out))
+    return {"r": out[0], "bits_npatch": out[1], "blocks": int(out[2]), "bits_widths": out[3],
+            "bits_per_weight": 1.0 / out[0]}
+
+
+def fifo_model(np_, n_fifo: int, rate: int, depth: int) -> dict:
+    """Cycle-by-cycle model of the patch-data FIFO of one XOR-gate network (Section 5.1)."""
+    np_ = np.ascontiguousarray(np_, dtype=np.uint16)
+    assert n_fifo >= 1 and rate >= 1 and depth >= 1
+    out = np.zeros(5, dtype=np.float64)
+    _L().orc_fifo_model(np_.size, _p(np_), n_fifo, rate, depth, _p(out))
+    return {"cycles": int(out[0]), "stall_bandwidth": int(out[1]), "stall_empty": int(out[2]),
+            "stall_full": int(out[3]), "peak": int(out[4]),
+            "relative_time": out[0] / max(np_.size, 1)}
+
+
+def csr_relative_time(nnz_per_row, lanes: int) -> float:
+    """Lock-step CSR rows, `lanes` at a time: cycles / (sum nnz / lanes) (Section 5.1)."""
+    nnz = np.ascontiguousarray(nnz_per_row, dtype=np.int64)
+    return float(_L().orc_csr_relative_time(nnz.size, _p(nnz), lanes))

@@ -404,3 +404,118 @@ void orc_eq1(int64_t mn, int n_out, int n_in, const uint16_t *np, double *out)
     out[4] = (double)maxp;
     out[5] = (double)sump;
 }
+
+/* ------------------------------------------------------------------------- */
+/* Blocked n_patch assignment (Section 5.2): the plane's l slices are cut     */
+/* into blocks of `block` consecutive slices and the width of the n_patch     */
+/* field is chosen per block from that block's own max p, so Eq. 1's middle   */
+/* term l * ceil(lg max p) becomes  sum over blocks of                        */
+/*   (slices in the block) * ceil(lg max p of the block).                     */
+/* The paper does not say how a block's width is made known to the decoder;   */
+/* out[3] reports one byte per block for it, separately.                      */
+/* out[0] = r with blocked widths (width bytes not counted), out[1] = bits of */
+/* n_patch with blocked widths, out[2] = number of blocks, out[3] = bits of   */
+/* the per-block width bytes.                                                 */
+/* ------------------------------------------------------------------------- */
+void orc_eq1_blocked(int64_t mn, int n_out, int n_in, const uint16_t *np, int64_t block, double *out)
+{
+    const int64_t l = (mn + n_out - 1) / n_out;
+    int64_t sump = 0, blocks = 0;
+    double b_np = 0.0;
+    for (int64_t s0 = 0; s0 < l; s0 += block) {
+        int64_t s1 = s0 + block < l ? s0 + block : l;
+        int64_t maxp = 0;
+        for (int64_t s = s0; s < s1; ++s) {
+            if (np[s] > maxp) maxp = np[s];
+            sump += np[s];
+        }
+        b_np += (double)(s1 - s0) * (double)ceil_lg(maxp);
+        blocks += 1;
+    }
+    double b_wc = (double)n_in / (double)n_out * (double)mn;
+    double b_dp = (double)sump * (double)ceil_lg(n_out);
+    out[0] = (double)mn / (b_wc + b_np + b_dp);
+    out[1] = b_np;
+    out[2] = (double)blocks;
+    out[3] = 8.0 * (double)blocks;
+}
+
+/* ------------------------------------------------------------------------- */
+/* Patch-data FIFO of one XOR-gate network (Section 5.1), cycle by cycle.     */
+/* Reading of the section (it gives no equations):                            */
+/*  - the network decrypts one slice per cycle when nothing holds it up;      */
+/*  - d_patch arrives as its own stream, `rate` entries per cycle, into a     */
+/*    FIFO of `depth` entries; the stream waits while the FIFO is full;       */
+/*  - the FIFO has n_fifo banks and hands at most n_fifo entries per cycle to */
+/*    the patch logic; a slice leaves the decoder in the cycle in which the   */
+/*    last of its n_patch entries has been handed over (a slice without       */
+/*    patches takes one cycle);                                               */
+/*  - within a cycle the stream writes first, then the patch logic reads.     */
+/* out[0] = cycles, out[1] = cycles in which the decoder held a slice over    */
+/* because more than n_fifo entries were still due (bandwidth stall),         */
+/* out[2] = cycles in which it held a slice over because the FIFO ran empty,  */
+/* out[3] = cycles in which the stream waited on a full FIFO, out[4] = peak   */
+/* occupancy after the write phase.  Relative execution time = cycles / l.    */
+/* ------------------------------------------------------------------------- */
+void orc_fifo_model(int64_t l, const uint16_t *np, int n_fifo, int rate, int depth, double *out)
+{
+    int64_t total = 0;
+    for (int64_t s = 0; s < l; ++s) total += np[s];
+    int64_t cycles = 0, stall_bw = 0, stall_empty = 0, stall_full = 0, peak = 0;
+    int64_t fifo = 0, produced = 0;
+    int64_t s = 0;
+    int64_t need = l > 0 ? np[0] : 0;
+    while (s < l) {
+        cycles += 1;
+        /* the stream writes */
+        int64_t w = rate;
+        if (w > total - produced) w = total - produced;
+        if (w > depth - fifo) {
+            w = depth - fifo;
+            stall_full += 1;
+        }
+        fifo += w;
+        produced += w;
+        if (fifo > peak) peak = fifo;
+        /* the patch logic reads */
+        int64_t r = need;
+        if (r > n_fifo) r = n_fifo;
+        if (r > fifo) r = fifo;
+        fifo -= r;
+        need -= r;
+        if (need == 0) {
+            s += 1;
+            if (s < l) need = np[s];
+        } else if (r == n_fifo) {
+            stall_bw += 1;
+        } else {
+            stall_empty += 1;
+        }
+    }
+    out[0] = (double)cycles;
+    out[1] = (double)stall_bw;
+    out[2] = (double)stall_empty;
+    out[3] = (double)stall_full;
+    out[4] = (double)peak;
+}
+
+/* ------------------------------------------------------------------------- */
+/* The CSR side of the same comparison (Section 5.1, Section 1): `lanes` rows */
+/* are worked on side by side, one non-zero per lane and cycle, and a group   */
+/* of rows is done when its longest row is, so a group costs max nnz cycles.  */
+/* Returns cycles / (sum nnz / lanes): 1.0 when every row has the same count. */
+/* ------------------------------------------------------------------------- */
+double orc_csr_relative_time(int64_t rows, const int64_t *nnz, int lanes)
+{
+    int64_t cycles = 0, sum = 0;
+    for (int64_t r0 = 0; r0 < rows; r0 += lanes) {
+        int64_t mx = 0;
+        for (int64_t r = r0; r < rows && r < r0 + lanes; ++r) {
+            if (nnz[r] > mx) mx = nnz[r];
+            sum += nnz[r];
+        }
+        cycles += mx;
+    }
+    if (sum == 0) return 1.0;
+    return (double)cycles / ((double)sum / (double)lanes);
+}

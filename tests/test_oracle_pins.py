@@ -448,3 +448,104 @@ def test_matmul_general_case_against_numpy():
     # dropping the mask changes the result (the mask really is applied)
     W_unmasked = ((planes.astype(np.float64) * 2 - 1) * alpha.astype(np.float64).T[:, :, None]).sum(axis=0)
     assert not np.allclose(Y, X @ W_unmasked.T)
+
+
+# ---------------------------------------------------------------------------------------------
+# Section 5.2, blocked n_patch assignment
+# ---------------------------------------------------------------------------------------------
+def _ceil_lg(v):
+    v = np.asarray(v, dtype=np.float64)
+    return np.where(v <= 1, 0.0, np.ceil(np.log2(np.maximum(v, 1))))
+
+
+def test_blocked_npatch_hand_computed_and_limits():
+    # six slices of 100 weights, n_in = 10: blocks of two have max p 1, 5, 3 -> widths 0, 3, 2 bits
+    p = np.array([0, 1, 2, 5, 0, 3], dtype=np.uint16)
+    b = orc.eq1_blocked(600, 100, 10, p, 2)
+    assert b["bits_npatch"] == 2 * 0 + 2 * 3 + 2 * 2 and b["blocks"] == 3
+    assert b["r"] == pytest.approx(600 / (60 + 10 + 11 * 7))
+    # one block covering the plane is Eq. 1 itself
+    whole = orc.eq1_blocked(600, 100, 10, p, 6)
+    plain = orc.eq1(600, 100, 10, p)
+    assert whole["bits_npatch"] == plain["bits_npatch"] == 6 * 3 and whole["r"] == pytest.approx(plain["r"])
+    # blocks of one slice: every slice pays for its own count only
+    rng = np.random.default_rng(11)
+    q = rng.integers(0, 40, 997).astype(np.uint16)
+    mn = 997 * 80 - 13                                   # ragged last slice, still 997 slices
+    one = orc.eq1_blocked(mn, 80, 16, q, 1)
+    assert one["bits_npatch"] == float(_ceil_lg(q).sum()) and one["blocks"] == 997
+    # a finer blocking never needs more n_patch bits than a coarser one that it refines
+    sizes = [997, 256, 64, 16, 4, 1]
+    bits = [orc.eq1_blocked(mn, 80, 16, q, s)["bits_npatch"] for s in sizes]
+    assert bits[0] == orc.eq1(mn, 80, 16, q)["bits_npatch"]
+    assert all(bits[i + 1] <= bits[i] for i in range(1, len(bits) - 1))   # 256 | 64 | 16 | 4 | 1 refine one another
+    assert max(bits[1:]) <= bits[0]
+
+
+def test_blocked_npatch_helps_when_one_region_is_dense():
+    # Section 5.2's case: a few slices with many care bits force a wide field on every slice
+    p = np.zeros(1024, dtype=np.uint16)
+    p[:8] = 37
+    plain = orc.eq1(1024 * 100, 100, 10, p)
+    blocked = orc.eq1_blocked(1024 * 100, 100, 10, p, 128)
+    assert plain["bits_npatch"] == 1024 * 6
+    assert blocked["bits_npatch"] == 128 * 6            # only the first block pays
+    assert blocked["r"] > plain["r"]
+
+
+# ---------------------------------------------------------------------------------------------
+# Section 5.1, patch-data FIFO of one XOR-gate network
+# ---------------------------------------------------------------------------------------------
+def test_fifo_model_worked_example():
+    # n_fifo = 2 banks, two entries arrive per cycle: slices with 0,1,2 patches take one cycle,
+    # 5 patches take three, 3 patches take two; the FIFO never runs dry
+    f = orc.fifo_model(np.array([0, 1, 2, 5, 0, 3], dtype=np.uint16), n_fifo=2, rate=2, depth=256)
+    assert f["cycles"] == 1 + 1 + 1 + 3 + 1 + 2
+    assert f["stall_bandwidth"] == 2 + 1 and f["stall_empty"] == 0 and f["stall_full"] == 0
+    assert f["relative_time"] == pytest.approx(9 / 6)
+
+
+def test_fifo_model_closed_forms():
+    rng = np.random.default_rng(12)
+    p = rng.poisson(0.8, 5000).astype(np.uint16)
+    l = p.size
+    # no patches at all: one slice per cycle
+    z = orc.fifo_model(np.zeros(100, np.uint16), 1, 1, 4)
+    assert z["cycles"] == 100 and z["stall_bandwidth"] == z["stall_empty"] == z["stall_full"] == 0
+    # enough banks for the largest count and a stream that keeps up: no stall (relative time 1.0)
+    big = orc.fifo_model(p, n_fifo=int(p.max()), rate=int(p.max()), depth=256)
+    assert big["cycles"] == l and big["relative_time"] == 1.0
+    # bank-limited only (stream as fast as the banks, FIFO deep enough): each slice costs
+    # max(1, ceil(p / n_fifo)) cycles
+    for banks in (1, 2, 3):
+        f = orc.fifo_model(p, n_fifo=banks, rate=banks, depth=256)
+        expect = int(np.maximum(1, -(-p.astype(np.int64) // banks)).sum())
+        assert f["cycles"] == expect and f["stall_empty"] == 0
+        assert f["stall_bandwidth"] == expect - l
+    # more banks never cost cycles
+    c = [orc.fifo_model(p, n_fifo=b, rate=b, depth=256)["cycles"] for b in (1, 2, 4, 8)]
+    assert c == sorted(c, reverse=True) and c[-1] == l
+    # stream-limited: two patches per slice but one entry per cycle arrives -> two cycles per slice
+    s = orc.fifo_model(np.full(50, 2, np.uint16), n_fifo=4, rate=1, depth=256)
+    assert s["cycles"] == 100 and s["stall_empty"] == 50 and s["stall_bandwidth"] == 0
+    # lower bounds that hold for any setting
+    for banks, rate, depth in ((1, 1, 2), (2, 1, 8), (3, 5, 4), (4, 2, 256)):
+        f = orc.fifo_model(p, banks, rate, depth)
+        total = int(p.sum())
+        assert f["cycles"] >= max(l, -(-total // banks), -(-total // rate))
+        assert f["peak"] <= depth
+    # a stream faster than the patch logic fills a shallow FIFO and then waits
+    full = orc.fifo_model(np.full(200, 1, np.uint16), n_fifo=1, rate=4, depth=8)
+    assert full["cycles"] == 200 and full["stall_full"] > 0 and full["peak"] == 8
+
+
+def test_csr_relative_time():
+    assert orc.csr_relative_time([3, 3, 3, 3], 2) == 1.0              # no variation between rows
+    assert orc.csr_relative_time([1, 5, 2, 2], 2) == pytest.approx((5 + 2) / (10 / 2))
+    assert orc.csr_relative_time([1, 5, 2, 2], 1) == 1.0              # one row at a time: nothing waits
+    rng = np.random.default_rng(13)
+    nnz = rng.binomial(1000, 0.1, 512)
+    t = orc.csr_relative_time(nnz, 32)
+    groups = nnz.reshape(-1, 32)
+    assert t == pytest.approx(groups.max(axis=1).sum() / (nnz.sum() / 32))
+    assert t > 1.05                                                   # Section 5.1: CSR rows vary
