@@ -150,6 +150,35 @@ int sqnn_describe_host(const void *blob, size_t blob_bytes, sqnn_desc *desc);
 /* Size accounting of a host blob (Eq. 1, Section 3.2, and stored bytes). */
 int sqnn_stats_host(const void *blob, size_t blob_bytes, sqnn_stats *stats);
 
+/* Blocked n_patch assignment (Section 5.2): what Eq. 1 gives when the n_patch field width is
+ * chosen per block of `block_slices` consecutive slices (from that block's own largest count)
+ * instead of once per plane.  Accounting only: the stored format keeps one width per plane.
+ * *bits_npatch = sum over planes and blocks of (slices in the block) * ceil(lg max p of the block),
+ * *bpw_eq1 = Eq. 1's bits per weight with that middle term (the block widths themselves, which the
+ * paper does not count, are not counted).  Either output may be NULL.  Errors: INVALID_ARG
+ * (block_slices = 0), BAD_BLOB. */
+int sqnn_stats_blocked_host(const void *blob, size_t blob_bytes, uint64_t block_slices,
+                            double *bpw_eq1, uint64_t *bits_npatch);
+
+/* Result of sqnn_fifo_model_host. */
+typedef struct sqnn_fifo_result {
+    uint64_t cycles;            /* cycles to pass all slices; relative execution time = cycles / l */
+    uint64_t stall_bandwidth;   /* cycles a slice was held because more than n_fifo entries were due */
+    uint64_t stall_empty;       /* cycles a slice was held because the FIFO had run dry              */
+    uint64_t stall_full;        /* cycles the d_patch stream waited on a full FIFO                   */
+    uint64_t peak;              /* largest occupancy reached                                          */
+} sqnn_fifo_result;
+
+/* Cycle model of the patch-data FIFO that Section 5.1 puts beside each XOR-gate network, run over
+ * the n_patch counts of one plane (np[l], host): the network passes one slice per cycle unless it
+ * has to wait for patch data; d_patch arrives as a stream of `rate` entries per cycle into a FIFO
+ * of `depth` entries (the stream waits while it is full; it writes before the patch logic reads in
+ * the same cycle); the FIFO's n_fifo banks hand over at most n_fifo entries per cycle, and a slice
+ * leaves in the cycle its last entry is handed over.  The section gives no equations; these are
+ * the readings taken.  Errors: INVALID_ARG (NULL, or a zero parameter). */
+int sqnn_fifo_model_host(const uint16_t *np, uint64_t l, uint32_t n_fifo, uint32_t rate, uint32_t depth,
+                         sqnn_fifo_result *result);
+
 /* Releases memory returned by the functions above.  NULL is allowed. */
 void sqnn_free(void *p);
 

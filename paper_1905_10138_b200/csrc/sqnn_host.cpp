@@ -498,4 +498,58 @@ int sqnn_stats_host(const void *blob, size_t blob_bytes, sqnn_stats *stats)
     return SQNN_OK;
 }
 
+int sqnn_stats_blocked_host(const void *blob, size_t blob_bytes, uint64_t block_slices,
+                            double *bpw_eq1, uint64_t *bits_npatch)
+{
+    if (block_slices == 0) return SQNN_E_INVALID_ARG;
+    sqnn_desc d;
+    int rc = sqnn_describe_host(blob, blob_bytes, &d);
+    if (rc != SQNN_OK) return rc;
+    const uint8_t *b = (const uint8_t *)blob;
+    const uint64_t mn = d.m * d.n, l = d.slices;
+    uint64_t np_bits = 0, dp_entries = 0;
+    for (uint32_t i = 0; i < d.n_q; ++i) {
+        const uint32_t *nps = (const uint32_t *)(b + d.off_np[i]);
+        for (uint64_t s0 = 0; s0 < l; s0 += block_slices) {
+            const uint64_t s1 = std::min(l, s0 + block_slices);
+            uint32_t maxp = 0;
+            for (uint64_t s = s0; s < s1; ++s) maxp = std::max(maxp, read_field(nps, s, d.w_np[i]));
+            np_bits += (s1 - s0) * ceil_lg_u64(maxp);
+        }
+        dp_entries += d.n_dp[i];
+    }
+    if (bits_npatch) *bits_npatch = np_bits;
+    if (bpw_eq1)
+        *bpw_eq1 = ((double)d.n_q * (double)d.n_in / (double)d.n_out * (double)mn + (double)np_bits +
+                    (double)dp_entries * ceil_lg_u64(d.n_out)) / (double)mn;
+    return SQNN_OK;
+}
+
+int sqnn_fifo_model_host(const uint16_t *np, uint64_t l, uint32_t n_fifo, uint32_t rate, uint32_t depth,
+                         sqnn_fifo_result *result)
+{
+    if (!result || (!np && l) || n_fifo == 0 || rate == 0 || depth == 0) return SQNN_E_INVALID_ARG;
+    std::memset(result, 0, sizeof *result);
+    uint64_t left = 0;                                   // entries the stream has not delivered yet
+    for (uint64_t s = 0; s < l; ++s) left += np[s];
+    uint64_t held = 0;                                   // entries in the FIFO
+    for (uint64_t s = 0; s < l; ++s) {
+        uint64_t due = np[s];
+        for (;;) {                                       // one pass = one cycle spent on slice s
+            ++result->cycles;
+            uint64_t in = std::min<uint64_t>(rate, left);
+            if (in > depth - held) { in = depth - held; ++result->stall_full; }
+            held += in;
+            left -= in;
+            result->peak = std::max(result->peak, held);
+            const uint64_t out = std::min(std::min<uint64_t>(due, n_fifo), held);
+            held -= out;
+            due -= out;
+            if (due == 0) break;
+            if (out == n_fifo) ++result->stall_bandwidth; else ++result->stall_empty;
+        }
+    }
+    return SQNN_OK;
+}
+
 }  // extern "C"

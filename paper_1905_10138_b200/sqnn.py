@@ -54,6 +54,11 @@ class Stats(ctypes.Structure):
                 "bpw_eq1": float(self.bpw_eq1), "bpw_actual": float(self.bpw_actual)}
 
 
+class FifoResult(ctypes.Structure):
+    _fields_ = [("cycles", ctypes.c_uint64), ("stall_bandwidth", ctypes.c_uint64),
+                ("stall_empty", ctypes.c_uint64), ("stall_full", ctypes.c_uint64), ("peak", ctypes.c_uint64)]
+
+
 class Desc(ctypes.Structure):
     _fields_ = [("m", ctypes.c_uint64), ("n", ctypes.c_uint64), ("slices", ctypes.c_uint64),
                 ("slices_padded", ctypes.c_uint64),
@@ -89,6 +94,10 @@ def lib():
         L.sqnn_unpack_host.argtypes = [vp, sz, u32, P(vp), P(vp), P(vp), P(u64)]
         L.sqnn_describe_host.argtypes = [vp, sz, P(Desc)]
         L.sqnn_stats_host.argtypes = [vp, sz, P(Stats)]
+        L.sqnn_stats_blocked_host.argtypes = [vp, sz, u64, P(ctypes.c_double), P(u64)]
+        L.sqnn_stats_blocked_host.restype = i32
+        L.sqnn_fifo_model_host.argtypes = [vp, u64, u32, u32, u32, P(FifoResult)]
+        L.sqnn_fifo_model_host.restype = i32
         L.sqnn_free.argtypes = [vp]
         L.sqnn_free.restype = None
         L.sqnn_decode.argtypes = [P(Desc), vp, vp, vp, i32, vp, sz, vp, vp]
@@ -200,6 +209,26 @@ def sqnn_stats_host(blob: np.ndarray) -> dict:
     _check(lib().sqnn_stats_host(_np_ptr(blob), blob.size, ctypes.byref(st)), "sqnn_stats_host")
     d = sqnn_describe_host(blob)
     return st.as_dict(d.n_q)
+
+
+def sqnn_stats_blocked_host(blob: np.ndarray, block_slices: int) -> dict:
+    """Eq. 1 with the n_patch width chosen per block of `block_slices` slices (Section 5.2)."""
+    blob = np.ascontiguousarray(blob, dtype=np.uint8)
+    bpw, bits = ctypes.c_double(), ctypes.c_uint64()
+    _check(lib().sqnn_stats_blocked_host(_np_ptr(blob), blob.size, int(block_slices), ctypes.byref(bpw),
+                                         ctypes.byref(bits)), "sqnn_stats_blocked_host")
+    return {"bpw_eq1": bpw.value, "bits_npatch": int(bits.value)}
+
+
+def sqnn_fifo_model_host(n_patch: np.ndarray, n_fifo: int, rate: int, depth: int) -> dict:
+    """Cycle model of the patch-data FIFO of Section 5.1 over the n_patch counts of one plane."""
+    n_patch = np.ascontiguousarray(n_patch, dtype=np.uint16)
+    res = FifoResult()
+    _check(lib().sqnn_fifo_model_host(_np_ptr(n_patch), n_patch.size, int(n_fifo), int(rate), int(depth),
+                                      ctypes.byref(res)), "sqnn_fifo_model_host")
+    out = {k: int(getattr(res, k)) for k, _ in FifoResult._fields_}
+    out["relative_time"] = out["cycles"] / max(n_patch.size, 1)
+    return out
 
 
 def sqnn_unpack_host(blob: np.ndarray, plane: int):

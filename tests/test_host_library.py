@@ -185,3 +185,37 @@ def test_device_entry_points_reject_bad_arguments_without_a_gpu():
                                 None, 0, None, None) == sqnn.E_INVALID_ARG
     assert sqnn.sqnn_workspace_bytes(d, 1) == 0
     assert sqnn.sqnn_workspace_bytes(d, 16) >= (16 * 80 + 63) // 64 * 8
+
+
+@pytest.mark.parametrize("name,make", LAYERS[:5], ids=[n for n, _ in LAYERS[:5]])
+def test_blocked_npatch_accounting_matches_the_oracle(name, make):
+    """Section 5.2: per-block n_patch widths, library (from the blob) against the oracle (from its own arrays)."""
+    layer = make()
+    blob, stats = library_blob(layer)
+    ref = oracle_arrays(layer)
+    l = (layer.mn + layer.n_out - 1) // layer.n_out
+    for block in (1, 7, 128, l, 10 * l):
+        got = sqnn.sqnn_stats_blocked_host(blob, block)
+        per_plane = [orc.eq1_blocked(layer.mn, layer.n_out, layer.n_in, a[1], block) for a in ref]
+        assert got["bits_npatch"] == sum(int(p["bits_npatch"]) for p in per_plane)
+        assert got["bpw_eq1"] == pytest.approx(sum(p["bits_per_weight"] for p in per_plane), rel=1e-12)
+    # one block per plane is the plain Eq. 1 figure
+    assert sqnn.sqnn_stats_blocked_host(blob, l)["bpw_eq1"] == pytest.approx(stats["bpw_eq1"], rel=1e-12)
+    with pytest.raises(sqnn.SqnnError):
+        sqnn.sqnn_stats_blocked_host(blob, 0)
+
+
+def test_fifo_model_matches_the_oracle():
+    """Section 5.1: the library's cycle model against the oracle's on encoder output and on random counts."""
+    rng = np.random.default_rng(77)
+    cases = [oracle_arrays(wl.make_sweep_layer(0, 3, m=64, n=1000))[0][1],      # heavy patch load
+             oracle_arrays(wl.make_layer(2, m=96, n=1000))[0][1],
+             rng.poisson(3.0, 4000).astype(np.uint16), np.zeros(17, np.uint16), np.zeros(0, np.uint16)]
+    for counts in cases:
+        for n_fifo, rate, depth in ((1, 1, 4), (2, 2, 256), (4, 1, 16), (3, 7, 5), (8, 8, 256)):
+            got = sqnn.sqnn_fifo_model_host(counts, n_fifo, rate, depth)
+            ref = orc.fifo_model(counts, n_fifo, rate, depth)
+            for key in ("cycles", "stall_bandwidth", "stall_empty", "stall_full", "peak"):
+                assert got[key] == ref[key], (key, n_fifo, rate, depth)
+    with pytest.raises(sqnn.SqnnError):
+        sqnn.sqnn_fifo_model_host(cases[0], 0, 1, 1)
