@@ -449,10 +449,12 @@ SQNN_DEV void walk_segment(uint32_t mask_sa, uint32_t plane_bytes, uint32_t xs_s
 constexpr uint32_t GEMV_ALPHA_WORDS = 64;
 
 // K3: decryption fused with Y[b][r] = sum_c W[r][c] X[b][c] for small batch, fp32 accumulate.
-// A warp decodes its tile of every plane into shared memory, then walks the row segments the
-// tile covers: lanes take the tile's 32-bit words in turn, visit the set bits of the mask word,
-// rebuild the weight value (+-alpha_1) + (+-alpha_2) + ... and accumulate value * x.  Partial
-// sums of a row segment are reduced over the warp and added to Y with one atomic per (row, b).
+// A group of 1 to 4 warps shares a tile: its warps decode the tile's planes into shared memory (one
+// plane per warp), then all of them walk the row segments the tile covers.  In a segment each lane
+// owns every (32 * warps)-th 32-bit word; it takes two care bits of its word a step, rebuilds the
+// weight values (+-alpha_1) + (+-alpha_2) + ... from the plane words and accumulates value * x, and
+// moves to its next word as soon as this one is used up (walk_segment).  Partial sums of a row
+// segment are reduced over the warp and added to Y with one atomic per (row, b).
 // Everything the walk reads is on chip by then: the tile's mask words arrive by cp.async while
 // the tile is decoded, the scales of its rows are fetched up front, and (XS = true) the
 // activations of the current batch chunk sit in shared memory as xs[c][BT].

@@ -42,6 +42,9 @@ constexpr uint32_t KC = 64;               // columns per pipeline step
 constexpr uint32_t MACRO = 512;           // columns decoded to bits at a time
 constexpr uint32_t STEPS_PER_MACRO = MACRO / KC;
 constexpr uint32_t RB_WORDS = MACRO / 32 + 1;   // words per row of the bit buffer (odd stride)
+// Copies of the 256-entry sign table, interleaved entry by entry: lane l reads copy l % LUT_COPIES, so two lanes
+// can only collide on a bank when they agree in l % LUT_COPIES.
+constexpr uint32_t LUT_COPIES = 8;
 constexpr uint32_t DEC_WARPS = 16;
 constexpr uint32_t DEC_THREADS = DEC_WARPS * 32;
 constexpr uint32_t THREADS = DEC_THREADS + 64;  // + TMA warp + MMA warp
@@ -291,8 +294,8 @@ k_decode_mma(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ C
     uint32_t *rb = reinterpret_cast<uint32_t *>(b_stages + (size_t)M.stages * M.b_stage_bytes);   // [buf][item][row][rbp]
     const uint32_t rb_buf_words = n_items * ROWS * rbp;
     uint32_t *tab = rb + M.rb_bufs * rb_buf_words;
-    uint2 *lut256 = reinterpret_cast<uint2 *>(tab + table_words(A.n_in, A.nwp, A.nchunks, A.cb));   // [256]
-    __nv_bfloat16 *lut = reinterpret_cast<__nv_bfloat16 *>(lut256 + 256);                             // [row][16]
+    uint2 *lut256 = reinterpret_cast<uint2 *>(tab + table_words(A.n_in, A.nwp, A.nchunks, A.cb));   // [256][LUT_COPIES]
+    __nv_bfloat16 *lut = reinterpret_cast<__nv_bfloat16 *>(lut256 + 256 * LUT_COPIES);                             // [row][16]
     float *alpha_s = reinterpret_cast<float *>(lut + ROWS * 16);         // [row][8]
     uint64_t *bars = reinterpret_cast<uint64_t *>(alpha_s + ROWS * 8);
     uint64_t *full_a = bars, *full_b = bars + MAX_STAGES, *empty = bars + 2 * MAX_STAGES;
@@ -311,14 +314,14 @@ k_decode_mma(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ C
 
     if (tid == 0) {
         for (uint32_t s = 0; s < MAX_STAGES; ++s) {
-            mbar_init(full_a + s, DEC_THREADS);
+            mbar_init(full_a + s, DEC_WARPS);        // one arrival per decode warp
             mbar_init(full_b + s, 1);
             mbar_init(empty + s, 1);
         }
         mbar_init(accum, 1);
         for (uint32_t s = 0; s < 2; ++s) {
             mbar_init(bits_full + s, 1);
-            mbar_init(bits_empty + s, DEC_THREADS);
+            mbar_init(bits_empty + s, DEC_WARPS);
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
@@ -331,7 +334,9 @@ k_decode_mma(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ C
 #pragma unroll
         for (uint32_t k = 0; k < 4; ++k)
             h[k] = ((tid >> (4 + k)) & 1u) ? (((tid >> k) & 1u) ? 0x3f80u : 0xbf80u) : 0u;
-        lut256[tid] = make_uint2(h[0] | (h[1] << 16), h[2] | (h[3] << 16));
+#pragma unroll
+        for (uint32_t c = 0; c < LUT_COPIES; ++c)
+            lut256[tid * LUT_COPIES + c] = make_uint2(h[0] | (h[1] << 16), h[2] | (h[3] << 16));
     }
     if (tid < ROWS) {
         // per-row scales and the table of all 2^n_q weight values (index bit i = plane i, bit 3 = mask)
@@ -436,9 +441,15 @@ k_decode_mma(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ C
                 // phase 2: steps of 64 columns; one thread per (row, 16 columns)
                 const uint32_t steps_here = stop ? 0u : (cnt + KC - 1) / KC;
                 const uint32_t row = tid >> 2, quarter = tid & 3, sw = row & 7;
+                const uint2 *lut_mine = lut256 + (lane & (LUT_COPIES - 1));
                 for (uint32_t ks = 0; ks < steps_here; ++ks, ++it) {
                     const uint32_t stage = it % M.stages, use = it / M.stages;
-                    if (use > 0 && !mbar_wait(empty + stage, (use - 1) & 1u, abort_flag, A.status)) break;
+                    // one lane per warp watches the barrier that frees the stage; the warp follows it
+                    if (use > 0) {
+                        uint32_t freed = 1;
+                        if (lane == 0) freed = mbar_wait(empty + stage, (use - 1) & 1u, abort_flag, A.status) ? 1u : 0u;
+                        if (!__shfl_sync(0xffffffffu, freed, 0)) break;
+                    }
                     uint8_t *a_stage = a_stages + stage * a_stage_bytes;
                     const uint32_t wi = ks * 2 + (quarter >> 1), sh16 = (quarter & 1) * 16;
                     uint32_t mw = (rbb[(A.n_q * ROWS + row) * rbp + wi] >> sh16) & 0xffffu;
@@ -450,7 +461,7 @@ k_decode_mma(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ C
                             uint2 e[4];
 #pragma unroll
                             for (uint32_t q = 0; q < 4; ++q)
-                                e[q] = lut256[(((mw >> (4 * q)) & 15u) << 4) | ((bw >> (4 * q)) & 15u)];
+                                e[q] = lut_mine[((((mw >> (4 * q)) & 15u) << 4) | ((bw >> (4 * q)) & 15u)) * LUT_COPIES];
                             uint8_t *arow = a_stage + i * A_STAGE_BYTES + row * 128;
                             *reinterpret_cast<uint4 *>(arow + (((quarter * 2) ^ sw) << 4)) = make_uint4(e[0].x, e[0].y, e[1].x, e[1].y);
                             *reinterpret_cast<uint4 *>(arow + (((quarter * 2 + 1) ^ sw) << 4)) = make_uint4(e[2].x, e[2].y, e[3].x, e[3].y);
@@ -490,9 +501,11 @@ k_decode_mma(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ C
                         }
                     }
                     fence_async_smem();                 // generic-proxy writes -> visible to the tensor core
-                    mbar_arrive(full_a + stage);
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(full_a + stage);     // the warp's 32 row segments are in place
                 }
-                if (M.tma_bits) mbar_arrive(bits_empty + buf);     // this thread is done with the buffer
+                __syncwarp();
+                if (M.tma_bits && lane == 0) mbar_arrive(bits_empty + buf);   // this warp is done with the buffer
                 if (decode_barrier_any(*abort_flag)) break;       // same decision in every decode thread
             }
         } else if (warp == DEC_WARPS) {
@@ -680,7 +693,7 @@ int mma_dispatch(const sqnn_desc *desc, const DecodeArgs &A0, const uint64_t *d_
     M.per_plane = (uint64_t)M.A.n_q * M.nbt <= 512 ? 1u : 0u;
     // The bit buffer is filled by TMA when the rows of the packed planes start on 16-byte boundaries.
     M.tma_bits = (d_workspace && desc->n % 128 == 0 && ((uintptr_t)d_mask & 15) == 0) ? 1u : 0u;
-    const size_t budget = 220 * 1024;
+    const size_t budget = 225 * 1024;        // + 1 KB of static shared memory stays within the 227 KB a block may have
     size_t fixed = 0, per_stage = 0;
     for (;;) {
         M.rbp = M.tma_bits ? 16 : RB_WORDS;
@@ -689,7 +702,7 @@ int mma_dispatch(const sqnn_desc *desc, const DecodeArgs &A0, const uint64_t *d_
         M.tmem_cols = 32;
         while (M.tmem_cols < a_tiles * M.nbt) M.tmem_cols *= 2;
         fixed = (size_t)M.rb_bufs * (M.A.n_q + 1) * ROWS * M.rbp * 4 +
-                (size_t)table_words(M.A.n_in, M.A.nwp, M.A.nchunks, M.A.cb) * 4 + 256 * 8 + ROWS * 16 * 2 +
+                (size_t)table_words(M.A.n_in, M.A.nwp, M.A.nchunks, M.A.cb) * 4 + 256 * 8 * LUT_COPIES + ROWS * 16 * 2 +
                 ROWS * 8 * 4 + (3 * MAX_STAGES + 5) * 8 + 16 + 1024;
         per_stage = (size_t)a_tiles * A_STAGE_BYTES + M.b_stage_bytes;
         if (fixed + 2 * per_stage <= budget) break;
