@@ -451,10 +451,11 @@ constexpr uint32_t GEMV_ALPHA_WORDS = 64;
 // K3: decryption fused with Y[b][r] = sum_c W[r][c] X[b][c] for small batch, fp32 accumulate.
 // A group of 1 to 4 warps shares a tile: its warps decode the tile's planes into shared memory (one
 // plane per warp), then all of them walk the row segments the tile covers.  In a segment each lane
-// owns every (32 * warps)-th 32-bit word; it takes two care bits of its word a step, rebuilds the
-// weight values (+-alpha_1) + (+-alpha_2) + ... from the plane words and accumulates value * x, and
-// moves to its next word as soon as this one is used up (walk_segment).  Partial sums of a row
-// segment are reduced over the warp and added to Y with one atomic per (row, b).
+// owns every (32 * warps)-th 32-bit word (with short rows every 32nd word of the segments that are its
+// warp's turn); it takes two care bits of its word a step, rebuilds the weight values
+// (+-alpha_1) + (+-alpha_2) + ... from the plane words and accumulates value * x, and moves to its next
+// word as soon as this one is used up (walk_segment).  Partial sums of a row segment are reduced over
+// the warp and added to Y with one atomic per (row, b).
 // Everything the walk reads is on chip by then: the tile's mask words arrive by cp.async while
 // the tile is decoded, the scales of its rows are fetched up front, and (XS = true) the
 // activations of the current batch chunk sit in shared memory as xs[c][BT].
@@ -463,7 +464,7 @@ template <int N_OUT, int N_IN, int BT, typename XT, bool XS, int NQ>
 __global__ void __launch_bounds__(640)
 k_decode_gemv(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__restrict__ alpha,
               const XT *__restrict__ x, int64_t ldx, uint32_t batch, float *__restrict__ y,
-              int64_t ldy, uint32_t n, uint32_t wpt)
+              int64_t ldy, uint32_t n, uint32_t wpt, uint32_t seg_par)
 {
     extern __shared__ __align__(16) uint32_t smem[];
     const uint32_t W = words_per_lane<N_OUT>(A);
@@ -574,11 +575,15 @@ k_decode_gemv(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__
             // row segments of the tile, in tile-local bit coordinates [a_loc, b_loc); c_tile is the column
             // (in the segment's row) of tile bit 0 and goes negative from the second row on
             const uint32_t T = (uint32_t)(P1 - P0);
-            uint32_t a_loc = 0, ai = 0;
+            // Short rows (seg_par): the group's warps take whole segments in turn instead of sharing the
+            // words of each, so that a lane still gets more than one word of a row.
+            uint32_t a_loc = 0, b_loc = 0, ai = 0, turn = 0;
             int32_t c_tile = (int32_t)(P0 - r_first * n);
-            for (uint64_t r = r_first; a_loc < T; ++r, ai += n_q, c_tile -= (int32_t)n) {
-                uint32_t b_loc = (uint32_t)((int32_t)n - c_tile);
+            for (uint64_t r = r_first; a_loc < T;
+                 ++r, ai += n_q, c_tile -= (int32_t)n, a_loc = b_loc, turn = turn + 1 == wpt ? 0 : turn + 1) {
+                b_loc = (uint32_t)((int32_t)n - c_tile);
                 b_loc = b_loc < T ? b_loc : T;
+                if (seg_par && turn != sub) continue;
                 constexpr int NR = NQ > 0 ? NQ : 1;
                 float al[NR];
                 if constexpr (NQ > 0) {
@@ -590,10 +595,10 @@ k_decode_gemv(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__
                 float acc[BT];
 #pragma unroll
                 for (int q = 0; q < BT; ++q) acc[q] = 0.0f;
-                const uint32_t wstep = 32 * wpt;
+                const uint32_t wstep = seg_par ? 32 : 32 * wpt;
                 const uint32_t first_mask = 0xffffffffu << (a_loc & 31u);
                 const uint32_t last_mask = 0xffffffffu >> (31u - ((b_loc - 1u) & 31u));
-                uint32_t lw = lw_lo + sub * 32 + lane;
+                uint32_t lw = lw_lo + (seg_par ? 0 : sub * 32) + lane;
                 if constexpr (XS && NQ > 0) {
                     walk_segment<BT, XT, NQ>(smem_addr(mask_s), 128 * W, smem_addr(xs), lw, lw_lo, lw_hi, wstep,
                                              first_mask, last_mask, c_tile, al, acc);
@@ -664,7 +669,6 @@ k_decode_gemv(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__
                     for (uint32_t d = 16; d >= 1; d >>= 1) s += __shfl_xor_sync(0xffffffffu, s, d);
                     if (lane == 0 && bc + q < batch) atomicAdd(y + (int64_t)(bc + q) * ldy + r, s);
                 }
-                a_loc = b_loc;
             }
             if (wpt == 1) __syncwarp();                  // the group is done with its regions
             else asm volatile("bar.sync %0, %1;\n" :: "r"(1 + group), "r"(32 * wpt) : "memory");
@@ -749,7 +753,7 @@ inline int launch_gemv_bt(const DecodeArgs &A, const uint64_t *d_mask, const flo
                           int64_t ldx, uint32_t batch, float *d_y, int64_t ldy, uint64_t n, cudaStream_t st)
 {
     // One tile group per tile an SM gets (up to 15, the named barriers), and as many warps per group
-    // (up to 4) as fit a block of 20 warps -- as long as a row still gives every lane of the group a word.
+    // (up to 4) as fit a block of 20 warps.
     // (More warps per block at fewer registers were slower: every warp repeats the per-tile bookkeeping.)
     const uint64_t live = (A.words64 * 2 + 32ull * A.W - 1) / (32ull * A.W);
     const uint32_t sms = (uint32_t)sm_count();
@@ -758,7 +762,8 @@ inline int launch_gemv_bt(const DecodeArgs &A, const uint64_t *d_mask, const flo
     groups = groups < 1 ? 1 : groups > 15 ? 15 : groups;
     uint32_t wpt = max_warps / groups;
     wpt = wpt < 1 ? 1 : wpt > 4 ? 4 : wpt;
-    while (wpt > 1 && n < 1024ull * wpt) --wpt;
+    // rows too short to give every lane of the group two words: the warps take whole row segments in turn
+    const uint32_t seg_par = (wpt > 1 && n < 2048ull * wpt) ? 1u : 0u;
     if (wpt == 1 && groups < 4) groups = 4;
     const size_t tab = (size_t)table_words(A.n_in, A.nwp, A.nchunks, A.cb) * 4;
     const size_t per_group = ((size_t)(A.n_q + 1) * 32 * A.W + GEMV_ALPHA_WORDS + (size_t)wpt * STAGE_WORDS) * 4;
@@ -791,7 +796,7 @@ inline int launch_gemv_bt(const DecodeArgs &A, const uint64_t *d_mask, const flo
         auto k = k_decode_gemv<N_OUT, N_IN, BT, XT, XSV, NQV>;                                               \
         if (prepare(k, smem)) return SQNN_E_CUDA;                                                            \
         if (cudaLaunchKernelEx(&cfg, k, A, (const uint32_t *)d_mask, d_alpha, (const XT *)d_x, ldx, batch,   \
-                               d_y, ldy, (uint32_t)n, wpt) != cudaSuccess) return SQNN_E_CUDA;               \
+                               d_y, ldy, (uint32_t)n, wpt, seg_par) != cudaSuccess) return SQNN_E_CUDA;               \
     } while (0)
     if (!xs) SQNN_GEMV_LAUNCH(false, 0);
     else if (A.n_q == 1) SQNN_GEMV_LAUNCH(true, 1);
