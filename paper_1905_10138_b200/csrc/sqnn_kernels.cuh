@@ -231,6 +231,12 @@ k_decode_bf16(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__
     }
 }
 
+// a / b with the short 32-bit division whenever a fits 32 bits (it does for layers below 2^32 weights).
+SQNN_DEV uint64_t div_u64_u32(uint64_t a, uint32_t b)
+{
+    return (a >> 32) == 0 ? (uint64_t)((uint32_t)a / b) : a / b;
+}
+
 SQNN_DEV float to_float(float v) { return v; }
 SQNN_DEV float to_float(__nv_bfloat16 v) { return __bfloat162float(v); }
 
@@ -481,7 +487,7 @@ k_decode_gemv(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__
     uint32_t *stage = warp0 + ngroups * per_group + warp * STAGE_WORDS;
     XT *xs = reinterpret_cast<XT *>(warp0 + ngroups * per_group + nwarps * STAGE_WORDS);
     const uint64_t mask_words = A.words64 * 2;
-    const uint64_t alpha_count = (A.mn / n) * n_q;
+    const uint64_t alpha_count = div_u64_u32(A.mn, n) * n_q;
     const bool mask_vec = (reinterpret_cast<uintptr_t>(mask32) & 15) == 0;
     const uint64_t tile_first = (uint64_t)blockIdx.x * ngroups + group, tile_step = (uint64_t)gridDim.x * ngroups;
 
@@ -495,7 +501,7 @@ k_decode_gemv(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__
         if (gw0 * 32 >= A.mn) return;
         if (sub == n_q % wpt) {
             stage_mask_tile(mask_s, mask32, gw0, mask_words, W, lane, mask_vec);
-            const uint64_t r_first = gw0 * 32 / n;
+            const uint64_t r_first = div_u64_u32(gw0 * 32, n);
             for (uint32_t i = lane; i < GEMV_ALPHA_WORDS; i += 32) {
                 const uint64_t at = r_first * n_q + i;
                 if (at < alpha_count) cp_async4(alpha_s + i, alpha + at);
@@ -546,7 +552,7 @@ k_decode_gemv(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__
             const uint64_t P0 = gw0 * 32;
             if (P0 >= A.mn) continue;
             const uint64_t P1 = (P0 + 1024ull * W < A.mn) ? P0 + 1024ull * W : A.mn;
-            const uint64_t r_first = P0 / n;
+            const uint64_t r_first = div_u64_u32(P0, n);
             if (bc != 0 || tile != tile_first) request(tile);       // not requested ahead of time
             if constexpr (N_OUT != 0) {
                 for (uint32_t i = sub; i < n_q; i += wpt) {
