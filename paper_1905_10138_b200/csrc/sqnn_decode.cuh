@@ -373,6 +373,92 @@ SQNN_DEV void patch_tile(const DecodeArgs &A, const PlanePtrs &P, uint32_t *regi
     if (bad) flag(A.status, 1u);
 }
 
+// The same patch step for runs that fit one window (alignment bytes + entries <= 512), which is nearly
+// every tile at the patch densities the format is meant for.  Differences from patch_tile: a lane handles
+// the four entries of one staged d_patch word a round, straight from the register it was fetched into
+// (nothing but the marks goes through shared memory); marks are indexed by byte position in the staged
+// words and, since they grow along the run, "nearest mark at or before" is a running maximum -- three
+// maxima inside the lane, one ballot and one shuffle across lanes, one shuffle to carry it into the next
+// round.
+template <uint32_t G, uint32_t N_OUT, typename WT>
+SQNN_DEV void patch_tile_fast(const DecodeArgs &A, const PlanePtrs &P, uint32_t *region, uint32_t *stage,
+                              const uint32_t (&st)[4], uint32_t base, uint32_t total, WT win, uint32_t lane)
+{
+    const uint32_t w_np = P.w_np;
+    const uint32_t fm = (1u << w_np) - 1u;
+    uint32_t f[G];
+    uint32_t cnt = 0;
+#pragma unroll
+    for (uint32_t i = 0; i < G; ++i) {
+        f[i] = (uint32_t)win & fm;
+        win >>= w_np;
+        cnt += f[i];
+    }
+    uint32_t incl = cnt;
+#pragma unroll
+    for (uint32_t d = 1; d < 32; d <<= 1) {
+        const uint32_t v = __shfl_up_sync(0xffffffffu, incl, d);
+        if (lane >= d) incl += v;
+    }
+    if (__shfl_sync(0xffffffffu, incl, 31) != total) {      // counts disagree with the offsets
+        flag(A.status, 2u);
+        return;
+    }
+    const uint32_t ob = base & 3u;                           // entry 0 sits at byte `ob` of the staged words
+    const uint32_t rounds = (ob + total + 127u) >> 7;        // 128 byte positions a round, at most 4 rounds
+    uint32_t *marks32 = stage + STAGE_DP_WORDS;
+    uint2 *marks64 = reinterpret_cast<uint2 *>(marks32);
+    uint16_t *marks = reinterpret_cast<uint16_t *>(marks32);
+    for (uint32_t j = 0; j < rounds; ++j) marks64[32 * j + lane] = make_uint2(0u, 0u);
+    __syncwarp();
+    // mark = first tile bit of the slice + 1, dropped at the byte position of the slice's first entry
+    uint32_t run = ob + incl - cnt, mark = lane * G * N_OUT + 1u;
+#pragma unroll
+    for (uint32_t i = 0; i < G; ++i) {
+        if (f[i] != 0) marks[run] = (uint16_t)mark;
+        run += f[i];
+        mark += N_OUT;
+    }
+    __syncwarp();
+    const uint32_t lower = (1u << lane) - 1u;                // lanes below this one
+    uint32_t carry = 0, bad = 0;
+#pragma unroll
+    for (uint32_t j = 0; j < 4; ++j) {
+        if (j < rounds) {                                    // the same in every lane
+            const uint2 mm = marks64[32 * j + lane];
+            const uint32_t m0 = mm.x & 0xffffu, m1 = mm.x >> 16, m2 = mm.y & 0xffffu, m3 = mm.y >> 16;
+            const uint32_t last = max(max(m0, m1), max(m2, m3));
+            const uint32_t have = __ballot_sync(0xffffffffu, last != 0) & lower;
+            const uint32_t got = __shfl_sync(0xffffffffu, last, (31 - __clz((int)have)) & 31);
+            const uint32_t prev = have ? got : carry;
+            uint32_t v[4];
+            v[0] = max(m0, prev);
+            v[1] = max(m1, v[0]);
+            v[2] = max(m2, v[1]);
+            v[3] = max(m3, v[2]);
+            carry = __shfl_sync(0xffffffffu, v[3], 31);
+            const uint32_t w = st[j];
+            // byte q of this word is entry 4 * (32 j + lane) + q - ob: inside the run iff lo <= q < hi
+            const int32_t lo = (int32_t)ob - (int32_t)(4u * (32u * j + lane));
+            const int32_t hi = lo + (int32_t)total;
+#pragma unroll
+            for (int32_t q = 0; q < 4; ++q) {
+                if (q >= lo && q < hi) {
+                    const uint32_t pos = (w >> (8 * q)) & 0xffu;
+                    if (v[q] != 0 && pos < N_OUT) {
+                        const uint32_t bit = v[q] - 1u + pos;
+                        atomicXor(region + (bit >> 5), 1u << (bit & 31u));
+                    } else {
+                        bad = 1u;
+                    }
+                }
+            }
+        }
+    }
+    __syncwarp();
+    if (bad) flag(A.status, 1u);
+}
+
 // Expands and patches the lane's G slices of one tile (already fetched into `in`, staged d_patch
 // words in `st`) into region[lane * W .. lane * W + W); the patch step then works on the whole
 // tile.  `stage` is the warp's STAGE_WORDS words of shared scratch.  WAIT_BULK: lane 0 first waits for its pending bulk copy out of
@@ -432,15 +518,18 @@ SQNN_DEV void tile_decode(const DecodeArgs &A, const PlanePtrs &P, const TileIn<
     if (in.total != 0) {
         __syncwarp();                                   // every lane's words are in place
         const uint32_t nb = lane * G * P.w_np, sh = nb & 31u;
+        const bool one_window = (in.base & 3u) + in.total <= 512u;      // the same in every lane
         if (G * P.w_np <= 32) {
             const uint32_t win = __funnelshift_r(in.np0, in.np1, sh) &
                                  (G * P.w_np == 32 ? 0xffffffffu : (1u << (G * P.w_np)) - 1u);
-            patch_tile<G, n_out, uint32_t>(A, P, region, stage, st, in.base, in.total, win, lane);
+            if (one_window) patch_tile_fast<G, n_out, uint32_t>(A, P, region, stage, st, in.base, in.total, win, lane);
+            else patch_tile<G, n_out, uint32_t>(A, P, region, stage, st, in.base, in.total, win, lane);
         } else {
             uint64_t win = (uint64_t)__funnelshift_r(in.np0, in.np1, sh) |
                            ((uint64_t)__funnelshift_r(in.np1, in.np2, sh) << 32);
             if (G * P.w_np < 64) win &= (1ull << (G * P.w_np)) - 1ull;
-            patch_tile<G, n_out, uint64_t>(A, P, region, stage, st, in.base, in.total, win, lane);
+            if (one_window) patch_tile_fast<G, n_out, uint64_t>(A, P, region, stage, st, in.base, in.total, win, lane);
+            else patch_tile<G, n_out, uint64_t>(A, P, region, stage, st, in.base, in.total, win, lane);
         }
     }
     __syncwarp();
