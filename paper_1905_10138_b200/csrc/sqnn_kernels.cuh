@@ -768,8 +768,9 @@ inline int launch_gemv_bt(const DecodeArgs &A, const uint64_t *d_mask, const flo
     groups = groups < 1 ? 1 : groups > 15 ? 15 : groups;
     uint32_t wpt = max_warps / groups;
     wpt = wpt < 1 ? 1 : wpt > 4 ? 4 : wpt;
-    // rows too short to give every lane of the group two words: the warps take whole row segments in turn
-    const uint32_t seg_par = (wpt > 1 && n < 2048ull * wpt) ? 1u : 0u;
+    // a tile that spans more rows than the group has warps: the warps take whole row segments in turn, which
+    // gives a lane more words of a row (a steadier load per lane) than sharing the words of every segment
+    const uint32_t seg_par = (wpt > 1 && 4ull * 1024 * A.W >= 5ull * n * wpt) ? 1u : 0u;
     if (wpt == 1 && groups < 4) groups = 4;
     const size_t tab = (size_t)table_words(A.n_in, A.nwp, A.nchunks, A.cb) * 4;
     const size_t per_group = ((size_t)(A.n_q + 1) * 32 * A.W + GEMV_ALPHA_WORDS + (size_t)wpt * STAGE_WORDS) * 4;
