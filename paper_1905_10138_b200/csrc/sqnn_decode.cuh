@@ -373,7 +373,7 @@ SQNN_DEV void patch_tile(const DecodeArgs &A, const PlanePtrs &P, uint32_t *regi
     if (bad) flag(A.status, 1u);
 }
 
-// The same patch step for runs that fit one window (alignment bytes + entries <= 512), which is nearly
+// The same patch step for runs that fit one window (at most PATCH_WIN entries), which is nearly
 // every tile at the patch densities the format is meant for.  Differences from patch_tile: a lane handles
 // the four entries of one staged d_patch word a round, straight from the register it was fetched into
 // (nothing but the marks goes through shared memory); marks are indexed by byte position in the staged
@@ -518,7 +518,8 @@ SQNN_DEV void tile_decode(const DecodeArgs &A, const PlanePtrs &P, const TileIn<
     if (in.total != 0) {
         __syncwarp();                                   // every lane's words are in place
         const uint32_t nb = lane * G * P.w_np, sh = nb & 31u;
-        const bool one_window = (in.base & 3u) + in.total <= 512u;      // the same in every lane
+        // the words fetched ahead hold at most PATCH_WIN entries (then alignment bytes + entries <= 511)
+        const bool one_window = in.total <= PATCH_WIN;                   // the same in every lane
         if (G * P.w_np <= 32) {
             const uint32_t win = __funnelshift_r(in.np0, in.np1, sh) &
                                  (G * P.w_np == 32 ? 0xffffffffu : (1u << (G * P.w_np)) - 1u);

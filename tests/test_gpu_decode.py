@@ -43,6 +43,11 @@ GENERIC = [
     ("gen-1x1", lambda: generic_layer(1, 1, 5, 77, 0.5, 15)),
     ("gen-96x9-q8", lambda: generic_layer(96, 9, 20, 999, 0.1, 16, n_q=8)),
     ("gen-tiny", lambda: generic_layer(100, 10, 1, 3, 1.0, 17)),
+    # patch runs of 300-600 entries per tile: three and four rounds of the single-window patch step, and tiles on
+    # either side of its 512-byte limit in the same layer (the longer ones take the windowed form)
+    ("gen-100x10-keep12", lambda: generic_layer(100, 10, 129, 4001, 0.12, 31)),
+    ("gen-100x10-keep135", lambda: generic_layer(100, 10, 129, 4001, 0.135, 32)),
+    ("gen-60x12-keep255-q2", lambda: generic_layer(60, 12, 77, 3000, 0.255, 33, n_q=2)),
 ]
 
 
