@@ -34,6 +34,10 @@ GEMV = [
     ("gen-33x20-q2-b5", lambda: generic_layer(33, 20, 31, 2049, 0.5, 13, n_q=2), "bf16", 5),
     ("gen-narrow-n", lambda: generic_layer(40, 12, 300, 17, 0.4, 21), "f32", 4),        # rows shorter than a word
     ("gen-empty-rows", lambda: generic_layer(100, 10, 64, 500, 0.0, 22), "f32", 1),     # everything pruned
+    # patch runs on both sides of the single-window limit of the patch step
+    ("gen-100x10-keep135", lambda: generic_layer(100, 10, 129, 4001, 0.135, 32), "f32", 2),
+    # 828 warp tiles: five to six per SM, three warps share a tile and take its row segments in turn
+    ("cfg2-2300rows-b1", lambda: wl.make_layer(2, m=2300, n=9216), "bf16", 1),
 ]
 
 
