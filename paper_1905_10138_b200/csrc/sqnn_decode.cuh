@@ -140,7 +140,9 @@ SQNN_DEV void build_tables_begin(const DecodeArgs &A, RowsAhead ahead)
 }
 
 // N_OUT, N_IN: the network shape when it is known at compile time (the index arithmetic then folds), 0 = read it from A.
-template <int N_OUT = 0, int N_IN = 0>
+// WAIT_ASYNC: the thread's pending cp.async copies are awaited just before the closing barrier, so that what they
+// bring in is visible to the whole block after it while the build itself runs under their latency.
+template <int N_OUT = 0, int N_IN = 0, bool WAIT_ASYNC = false>
 SQNN_DEV void build_tables_finish(const DecodeArgs &A, uint32_t *tab)
 {
     const uint32_t *rows_s = rows_scratch();
@@ -187,6 +189,7 @@ SQNN_DEV void build_tables_finish(const DecodeArgs &A, uint32_t *tab)
             tab[i] = tab[((chbase | l) << kshift) + k] ^ tab[((chbase | h) << kshift) + k];
         }
     }
+    if constexpr (WAIT_ASYNC) asm volatile("cp.async.wait_all;\n" ::: "memory");
     __syncthreads();
 }
 

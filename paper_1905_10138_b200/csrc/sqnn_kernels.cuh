@@ -541,8 +541,8 @@ k_decode_gemv(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__
             if constexpr (N_OUT != 0) {
                 if (tile_first < A.tiles && sub < n_q) stage_fetch<N_OUT, N_IN>(A, A.pl[sub], pre, lane, st_pre);
             }
-            cp_async_wait_all();
-            build_tables_finish<N_OUT, N_IN>(A, smem);   // ends with a block barrier
+            // the asynchronous copies (activations, mask, scales) are awaited inside, before the closing barrier
+            build_tables_finish<N_OUT, N_IN, true>(A, smem);
         } else {
             cp_async_wait_all();
             __syncthreads();
@@ -581,15 +581,29 @@ k_decode_gemv(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__
             // row segments of the tile, in tile-local bit coordinates [a_loc, b_loc); c_tile is the column
             // (in the segment's row) of tile bit 0 and goes negative from the second row on
             const uint32_t T = (uint32_t)(P1 - P0);
-            // Short rows (seg_par): the group's warps take whole segments in turn instead of sharing the
-            // words of each, so that a lane still gets more than one word of a row.
+            // seg_par: the group's warps take whole segments instead of sharing the words of each, so that a
+            // lane gets more words of a row.  Each segment goes to the warp that has been given the fewest
+            // weights so far (every warp keeps the same books, so they agree without talking).
+            // (With many short segments per tile, seg_par == 1, they simply take turns.)
             uint32_t a_loc = 0, b_loc = 0, ai = 0, turn = 0;
+            uint32_t given[4] = {0u, 0u, 0u, 0u};
             int32_t c_tile = (int32_t)(P0 - r_first * n);
             for (uint64_t r = r_first; a_loc < T;
                  ++r, ai += n_q, c_tile -= (int32_t)n, a_loc = b_loc, turn = turn + 1 == wpt ? 0 : turn + 1) {
                 b_loc = (uint32_t)((int32_t)n - c_tile);
                 b_loc = b_loc < T ? b_loc : T;
-                if (seg_par && turn != sub) continue;
+                if (seg_par == 1) {
+                    if (turn != sub) continue;
+                } else if (seg_par == 2) {
+                    uint32_t pick = 0;
+#pragma unroll
+                    for (uint32_t w = 1; w < 4; ++w)
+                        if (w < wpt && given[w] < given[pick]) pick = w;
+#pragma unroll
+                    for (uint32_t w = 0; w < 4; ++w)
+                        if (w == pick) given[w] += b_loc - a_loc;
+                    if (pick != sub) continue;
+                }
                 constexpr int NR = NQ > 0 ? NQ : 1;
                 float al[NR];
                 if constexpr (NQ > 0) {
@@ -770,7 +784,8 @@ inline int launch_gemv_bt(const DecodeArgs &A, const uint64_t *d_mask, const flo
     wpt = wpt < 1 ? 1 : wpt > 4 ? 4 : wpt;
     // a tile that spans more rows than the group has warps: the warps take whole row segments in turn, which
     // gives a lane more words of a row (a steadier load per lane) than sharing the words of every segment
-    const uint32_t seg_par = (wpt > 1 && 4ull * 1024 * A.W >= 5ull * n * wpt) ? 1u : 0u;
+    // (2 = by load, for tiles of fewer than 8 rows; 1 = in turn)
+    const uint32_t seg_par = (wpt > 1 && 4ull * 1024 * A.W >= 5ull * n * wpt) ? (1024ull * A.W < 8ull * n ? 2u : 1u) : 0u;
     if (wpt == 1 && groups < 4) groups = 4;
     const size_t tab = (size_t)table_words(A.n_in, A.nwp, A.nchunks, A.cb) * 4;
     const size_t per_group = ((size_t)(A.n_q + 1) * 32 * A.W + GEMV_ALPHA_WORDS + (size_t)wpt * STAGE_WORDS) * 4;
