@@ -34,6 +34,11 @@ GEMV = [
     ("gen-33x20-q2-b5", lambda: generic_layer(33, 20, 31, 2049, 0.5, 13, n_q=2), "bf16", 5),
     ("gen-narrow-n", lambda: generic_layer(40, 12, 300, 17, 0.4, 21), "f32", 4),        # rows shorter than a word
     ("gen-empty-rows", lambda: generic_layer(100, 10, 64, 500, 0.0, 22), "f32", 1),     # everything pruned
+    # four and more planes (scales and plane words not held in registers) and rows too long for the
+    # activations to be staged on chip: the plain C++ form of the walk
+    ("gen-60x12-q5-b3", lambda: generic_layer(60, 12, 40, 3000, 0.2, 41, n_q=5), "bf16", 3),
+    ("gen-long-rows-b2", lambda: generic_layer(40, 12, 5, 100003, 0.1, 42), "bf16", 2),
+    ("gen-long-rows-f32-b1", lambda: generic_layer(100, 10, 3, 50001, 0.1, 43), "f32", 1),
     # patch runs on both sides of the single-window limit of the patch step
     ("gen-100x10-keep135", lambda: generic_layer(100, 10, 129, 4001, 0.135, 32), "f32", 2),
     # 828 warp tiles: five to six per SM, three warps share a tile and take its row segments in turn
