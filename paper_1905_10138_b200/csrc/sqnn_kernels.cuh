@@ -586,7 +586,7 @@ k_decode_gemv(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__
             // weights so far (every warp keeps the same books, so they agree without talking).
             // (With many short segments per tile, seg_par == 1, they simply take turns.)
             uint32_t a_loc = 0, b_loc = 0, ai = 0, turn = 0;
-            uint32_t given[4] = {0u, 0u, 0u, 0u};
+            uint32_t g0 = 0, g1 = 0, g2 = 0, g3 = 0;     // weights given to each warp of the group so far
             int32_t c_tile = (int32_t)(P0 - r_first * n);
             for (uint64_t r = r_first; a_loc < T;
                  ++r, ai += n_q, c_tile -= (int32_t)n, a_loc = b_loc, turn = turn + 1 == wpt ? 0 : turn + 1) {
@@ -595,13 +595,15 @@ k_decode_gemv(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__
                 if (seg_par == 1) {
                     if (turn != sub) continue;
                 } else if (seg_par == 2) {
-                    uint32_t pick = 0;
-#pragma unroll
-                    for (uint32_t w = 1; w < 4; ++w)
-                        if (w < wpt && given[w] < given[pick]) pick = w;
-#pragma unroll
-                    for (uint32_t w = 0; w < 4; ++w)
-                        if (w == pick) given[w] += b_loc - a_loc;
+                    uint32_t pick = 0, least = g0;
+                    if (wpt > 1 && g1 < least) { pick = 1; least = g1; }
+                    if (wpt > 2 && g2 < least) { pick = 2; least = g2; }
+                    if (wpt > 3 && g3 < least) { pick = 3; least = g3; }
+                    const uint32_t len = b_loc - a_loc;
+                    g0 += pick == 0 ? len : 0u;
+                    g1 += pick == 1 ? len : 0u;
+                    g2 += pick == 2 ? len : 0u;
+                    g3 += pick == 3 ? len : 0u;
                     if (pick != sub) continue;
                 }
                 constexpr int NR = NQ > 0 ? NQ : 1;
