@@ -369,9 +369,18 @@ def cpu_baseline(layer, rows=4096):
     for _ in range(reps):
         oracle_step(layer, rows, sub_mask, arrays, x64)
     dt = (time.perf_counter() - t0) / reps
-    return {"value": rows * layer.n * layer.n_q / dt, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle",
+    # the same passes on one thread, for the per-core figure
+    threads = orc.num_threads()
+    orc.set_num_threads(1)
+    t0 = time.perf_counter()
+    for _ in range(2):
+        oracle_step(layer, rows, sub_mask, arrays, x64)
+    dt1 = (time.perf_counter() - t0) / 2
+    orc.set_num_threads(threads)
+    return {"value": rows * layer.n * layer.n_q / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
             "sample": f"first {rows} of {layer.m} rows of the same layer, decode + fp64 product, batch 1, "
-                      f"{reps} repetitions", "seconds_per_pass": dt}
+                      f"{reps} repetitions", "seconds_per_pass": dt,
+            "value_one_thread": rows * layer.n * layer.n_q / dt1}
 
 
 def run_reference(args):
