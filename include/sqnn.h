@@ -13,6 +13,15 @@
  * a plane) and d_patch (positions inside the slice) and are flipped after the expansion
  * (Section 3.2).  Positions past mn in the last slice are don't-cares.
  *
+ * Two byte layouts carry the same three parts (w^c, n_patch, d_patch).  The *device blob* is what
+ * the kernels read: the seed stream, the network's lookup tables, and the patches regrouped per
+ * tile of 256 slices as 16-bit bit positions inside the tile (position = slice-in-tile * n_out +
+ * d_patch), so that the decoder needs no n_patch stream and no prefix sum to find a slice's
+ * patches.  The *storage form* (sqnn_store_host / sqnn_load_host) is the compact layout of
+ * Section 3.2 for files: n_patch fields whose width is chosen per block of slices (Section 5.2)
+ * and d_patch entries of ceil(lg n_out) bits.  sqnn_unpack_host returns the same logical arrays
+ * from a device blob whichever way it was made.
+ *
  * General rules
  *  - Plain C.  Every function returns an int status (SQNN_OK = 0, negative = error) unless
  *    noted; nothing aborts, throws or prints.
@@ -24,8 +33,9 @@
  *    device memory and create no streams.
  *  - Host buffers the library returns (blob, unpacked arrays) are released with sqnn_free.
  *  - d_status (device, one uint32, may be NULL) receives a sticky non-zero code when a
- *    kernel had to skip a malformed patch entry (position >= n_out, or a patch index past
- *    the end of the d_patch section); the caller zeroes it.  Kernels never trap.
+ *    kernel had to skip a malformed patch entry (1: position outside its tile, 2: a tile's
+ *    offsets point past the end of the patch section) or gave up a bounded wait
+ *    (6 = -SQNN_E_TIMEOUT); the caller zeroes it.  Kernels never trap.
  */
 #ifndef SQNN_H_
 #define SQNN_H_
@@ -40,9 +50,10 @@ extern "C" {
 #define SQNN_MAX_PLANES   8      /* n_q <= 8                                            */
 #define SQNN_MAX_N_OUT    256    /* n_out <= 256: a d_patch position fits one byte      */
 #define SQNN_MAX_N_IN     32     /* n_in <= 32: a seed fits one uint32                  */
-#define SQNN_BLOCK_SLICES 128    /* one d_patch offset is stored per 128 slices         */
+#define SQNN_TILE_SLICES  256    /* patches are indexed per tile of 256 slices          */
 #define SQNN_PAD_SLICES   1024   /* streams are zero-padded to a multiple of 1024 slices*/
 #define SQNN_MAX_BATCH    1024
+#define SQNN_PATCH_HIST_BINS 16  /* n_patch = 0 .. 14, last bin: 15 and more            */
 #define SQNN_STATIC_SCRATCH_BYTES (8u << 20)   /* built-in scratch of sqnn_decode_matmul_static */
 
 enum {
@@ -81,34 +92,41 @@ typedef struct sqnn_planes {
 
 /* Size accounting.  bpw_eq1 = sum over planes of 1 / r with r from Eq. 1 taken literally
  * (ceil(lg max p) bits per n_patch, ceil(lg n_out) bits per d_patch entry).  bpw_actual counts
- * the bytes of the blob sections as stored (padding and the per-128-slice offsets included,
- * header and the network excluded), per weight.  The pruning mask (1 bit / weight, kept
- * outside the blob) is not part of either. */
+ * the bytes of the device blob's sections as stored (padding included; header and the rows of M
+ * excluded), per weight: bits_wc the seed streams, bits_dpatch the 16-bit patch positions,
+ * bits_index the per-tile patch offsets plus the lookup tables (bits_tables of it), bits_npatch 0
+ * (the device blob has no n_patch stream; counts follow from the positions).  The pruning mask
+ * (1 bit / weight, kept outside the blob) is not part of either.  patch_hist[k] = number of
+ * slices (all planes) with n_patch = k, the last bin collecting 15 and more (Section 5.2 looks
+ * at this distribution). */
 typedef struct sqnn_stats {
     uint64_t slices;                          /* l per plane                              */
     uint64_t patches[SQNN_MAX_PLANES];        /* sum of n_patch per plane                 */
     uint32_t max_patch[SQNN_MAX_PLANES];      /* max n_patch per plane                    */
     uint64_t bits_wc, bits_npatch, bits_dpatch, bits_index;   /* stored sizes, all planes */
+    uint64_t bits_tables;                     /* part of bits_index                       */
+    uint64_t patch_hist[SQNN_PATCH_HIST_BINS];
     double   bpw_eq1, bpw_actual;
 } sqnn_stats;
 
-/* Parsed blob header.  Offsets are bytes from the start of the blob, each a multiple of 16.
- * Per plane i: the w^c stream (slice s occupies bits [s*n_in, (s+1)*n_in), least significant
- * bit first inside little-endian 32-bit words); the n_patch stream (w_np[i] bits per slice,
- * same packing; absent when w_np[i] = 0); the offsets (uint32 per block of 128 slices: number
- * of d_patch entries before the block, plus one closing entry = n_dp[i]); the d_patch entries
- * (one byte each, slice order, ascending inside a slice).  Streams cover slices_padded slices
+/* Parsed header of a device blob.  Offsets are bytes from the start of the blob, each a multiple
+ * of 16.  Tables: the lookup tables of the network -- the seed is cut into tab_chunks chunks of
+ * tab_chunk_bits bits, entry (chunk, value) = XOR of the columns of M the value selects, as
+ * tab_entry_words 32-bit words (bits >= n_out zero) at word ((chunk << tab_chunk_bits) | value) *
+ * tab_entry_words; the geometry is a fixed function of (n_out, n_in).  Per plane i: the w^c
+ * stream (slice s occupies bits [s*n_in, (s+1)*n_in), least significant bit first inside
+ * little-endian 32-bit words); the tile index (uint32 per tile of 256 slices: number of patch
+ * entries before the tile, plus one closing entry = n_pp[i]); the patch entries (uint16 each:
+ * bit position inside the tile, ascending inside a tile).  Streams cover slices_padded slices
  * (padding slices have seed 0 and no patch) and every section ends with >= 16 zero bytes. */
 typedef struct sqnn_desc {
     uint64_t m, n, slices, slices_padded;
-    uint32_t n_q, n_out, n_in, block_slices;
-    uint32_t w_np[SQNN_MAX_PLANES];
-    uint32_t w_dp;                            /* bits per stored d_patch entry (8)        */
-    uint32_t reserved;
+    uint32_t n_q, n_out, n_in, tile_slices;
+    uint32_t tab_chunks, tab_chunk_bits, tab_entry_words, reserved;
     uint64_t off_xornet;                      /* n_out uint32 rows                        */
-    uint64_t off_wc[SQNN_MAX_PLANES], off_np[SQNN_MAX_PLANES];
-    uint64_t off_idx[SQNN_MAX_PLANES], off_dp[SQNN_MAX_PLANES];
-    uint64_t n_dp[SQNN_MAX_PLANES];
+    uint64_t off_tables, tables_bytes;
+    uint64_t off_wc[SQNN_MAX_PLANES], off_idx[SQNN_MAX_PLANES], off_pp[SQNN_MAX_PLANES];
+    uint64_t n_pp[SQNN_MAX_PLANES];           /* patch entries per plane = sum of n_patch */
     uint64_t total_bytes;
 } sqnn_desc;
 
@@ -142,9 +160,10 @@ int sqnn_pack_host(const sqnn_xornet *net, uint64_t m, uint64_t n, uint32_t n_q,
 int sqnn_unpack_host(const void *blob, size_t blob_bytes, uint32_t plane,
                      uint32_t **wc, uint16_t **np, uint16_t **dp, uint64_t *n_dp);
 
-/* Validates a host blob and fills *desc: magic / version, section bounds and alignment, field
- * widths, offsets non-decreasing and consistent with the n_patch stream, sum(n_patch) = n_dp,
- * every d_patch entry < n_out, padding slices empty.  BAD_BLOB on any violation. */
+/* Validates a host blob and fills *desc: magic / version, section bounds and alignment, the table
+ * geometry and the tables themselves (recomputed from the rows of M), tile offsets non-decreasing
+ * and closing at n_pp, every patch position inside its tile and not past the last real slice,
+ * positions strictly ascending inside a tile, padding slices empty.  BAD_BLOB on any violation. */
 int sqnn_describe_host(const void *blob, size_t blob_bytes, sqnn_desc *desc);
 
 /* Size accounting of a host blob (Eq. 1, Section 3.2, and stored bytes). */
@@ -205,20 +224,25 @@ int sqnn_decode(const sqnn_desc *desc, const void *d_blob, const uint64_t *d_mas
 
 /* Decryption fused with the product the layer exists for: Y[b][r] = sum_c W[r][c] * X[b][c],
  * W[r][c] = mask[r][c] * sum_i alpha[r][i] * (2 b_i[r][c] - 1) with b_i the decoded planes
- * (Sections 3.1, 3.2; the sparse quantized product of Section 1).  The decoded weights never
+ * (Sections 3.1, 3.2; the sparse quantized product of Section 1).  The rescaled weights never
  * reach global memory.  d_x: device, batch rows of n elements (x_dtype SQNN_X_F32 or
  * SQNN_X_BF16), row stride ldx elements.  d_y: device fp32, batch rows of m, row stride ldy;
- * fully overwritten.  batch <= 15 runs the fp32-accumulate GEMV kernel (weights exact);
- * batch >= 16 runs the tcgen05 kernel (weights rounded to bf16, activations must be BF16 with a
- * 16-byte aligned base and a row pitch that is a multiple of 16 bytes, fp32 accumulation in
- * tensor memory).  d_workspace: device scratch of at least sqnn_workspace_bytes(desc, batch)
- * bytes, 256-byte aligned, contents undefined before and after.  For batch >= 16 it receives the
- * decoded planes as packed bits (1 bit per weight and plane; the rescaled weights themselves
- * exist only in shared memory), which the tensor-core kernel then reads; it may be NULL, in
- * which case that kernel decodes the slices itself (same results, slower).  For batch <= 15 it
- * is not used.  Errors: INVALID_ARG, UNSUPPORTED (F32 activations with batch >= 16, unaligned
- * activations with batch >= 16, batch > SQNN_MAX_BATCH), WORKSPACE (workspace given but too
- * small or misaligned), CUDA. */
+ * fully overwritten.
+ *  - batch <= 15: one kernel; every block decodes the slices that cover its own rows into shared
+ *    memory and accumulates in fp32 on the plain ALUs (weights exact).  Each Y[b][r] is summed in
+ *    a fixed order, so results are bit-identical from run to run.  No workspace is used.  A row
+ *    must fit shared memory as bits: n * (n_q + 1) <= 1 400 000, else UNSUPPORTED.
+ *  - batch >= 16: two kernels.  The decode kernel writes the planes as packed bits (1 bit per
+ *    weight and plane) into d_workspace; the tcgen05 kernel reads boxes of them, expands them to
+ *    bf16 tiles in shared memory and multiplies with fp32 accumulation in tensor memory.
+ *    Activations must be BF16 with a 16-byte aligned base and a row pitch that is a multiple of
+ *    16 bytes.  d_workspace: device scratch of at least sqnn_workspace_bytes(desc, batch) bytes,
+ *    256-byte aligned, contents undefined before and after; required.  Column ranges handled by
+ *    different blocks are combined with fp32 atomics on Y, so results can differ from run to run
+ *    in the last bits (well inside the 1e-2 tolerance of this path).
+ * Errors: INVALID_ARG, UNSUPPORTED (F32 activations with batch >= 16, unaligned activations with
+ * batch >= 16, batch > SQNN_MAX_BATCH, rows too long for batch <= 15), WORKSPACE (batch >= 16 and
+ * the workspace is missing, too small or misaligned), CUDA. */
 int sqnn_decode_matmul(const sqnn_desc *desc, const void *d_blob, const uint64_t *d_mask,
                        const float *d_alpha, const void *d_x, int x_dtype, uint32_t batch,
                        int64_t ldx, float *d_y, int64_t ldy, void *d_workspace,
@@ -257,7 +281,7 @@ int sqnn_search_seeds(const sqnn_xornet *net, uint64_t m, uint64_t n, uint32_t n
                       const uint64_t *d_planes, const uint64_t *d_mask, uint32_t *d_wc, uint16_t *d_np,
                       void *cuda_stream);
 
-/* Scratch bytes sqnn_decode_matmul can use for this layer and batch (0 if none). */
+/* Scratch bytes sqnn_decode_matmul needs for this layer and batch (0 for batch <= 15). */
 size_t sqnn_workspace_bytes(const sqnn_desc *desc, uint32_t batch);
 
 /* Human-readable name of a status code; never NULL. */

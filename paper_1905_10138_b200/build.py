@@ -13,7 +13,7 @@ SOURCES = ["sqnn_host.cpp", "sqnn_api.cu", "sqnn_mma.cu", "sqnn_search.cu"]
 SHAPE_SOURCE = "sqnn_shape.cu"
 # (n_out, n_in) with compile-time kernels -- the list in csrc/sqnn_shapes.h -- plus the run-time shape (0, 0)
 SHAPES = [(40, 12), (40, 16), (60, 12), (80, 8), (80, 16), (100, 10), (200, 10), (0, 0)]
-HEADERS = ["sqnn_blob.h", "sqnn_decode.cuh", "sqnn_launch.h", "sqnn_kernels.cuh", "sqnn_shapes.h", SHAPE_SOURCE]
+HEADERS = ["sqnn_blob.h", "sqnn_layout.h", "sqnn_decode.cuh", "sqnn_launch.h", "sqnn_kernels.cuh", "sqnn_gemv.cuh", "sqnn_shapes.h", SHAPE_SOURCE]
 
 
 def _nvcc() -> str:

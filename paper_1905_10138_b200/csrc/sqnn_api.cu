@@ -17,12 +17,12 @@ int decode_shape(const DecodeArgs &A, sqnn_out_mode mode, const uint64_t *d_mask
                  uint64_t n, void *d_out, cudaStream_t st);
 template <int N_OUT, int N_IN>
 int gemv_shape(const DecodeArgs &A, const uint64_t *d_mask, const float *d_alpha, const void *d_x, int x_dtype,
-               int64_t ldx, uint32_t batch, float *d_y, int64_t ldy, uint64_t n, cudaStream_t st);
+               int64_t ldx, uint32_t batch, float *d_y, int64_t ldy, uint64_t m, uint64_t n, cudaStream_t st);
 #define SQNN_DECLARE(NO, NI)                                                                                  \
     template <> int decode_shape<NO, NI>(const DecodeArgs &, sqnn_out_mode, const uint64_t *, const float *,  \
                                          uint64_t, void *, cudaStream_t);                                     \
     template <> int gemv_shape<NO, NI>(const DecodeArgs &, const uint64_t *, const float *, const void *, int, \
-                                       int64_t, uint32_t, float *, int64_t, uint64_t, cudaStream_t);
+                                       int64_t, uint32_t, float *, int64_t, uint64_t, uint64_t, cudaStream_t);
 SQNN_FOR_SHAPES(SQNN_DECLARE)
 SQNN_DECLARE(0, 0)
 #undef SQNN_DECLARE
@@ -33,31 +33,34 @@ int fill_decode_args(const sqnn_desc *d, const void *d_blob, uint32_t *d_status,
     if (((uintptr_t)d_blob & 15) != 0) return SQNN_E_INVALID_ARG;
     if (d->n_out < 1 || d->n_out > SQNN_MAX_N_OUT || d->n_in < 1 || d->n_in > SQNN_MAX_N_IN ||
         d->n_q < 1 || d->n_q > SQNN_MAX_PLANES || d->m == 0 || d->n == 0 ||
-        d->block_slices != SQNN_BLOCK_SLICES || d->slices_padded % SQNN_PAD_SLICES != 0)
+        d->tile_slices != SQNN_TILE_SLICES || d->slices_padded % SQNN_PAD_SLICES != 0)
         return SQNN_E_INVALID_ARG;
     const uint8_t *b = (const uint8_t *)d_blob;
     A->mn = d->m * d->n;
     A->words64 = (A->mn + 63) / 64;
     A->n_out = d->n_out; A->n_in = d->n_in; A->n_q = d->n_q;
-    A->G = slices_per_lane(d->n_out);
+    A->KT = format_tiles_per_kernel_tile(d->n_out);
+    A->G = 8 * A->KT;
     A->W = A->G * d->n_out / 32;
-    A->tiles = d->slices_padded / (32ull * A->G);
+    A->ktiles = d->slices_padded / (32ull * A->G);
     A->nw = entry_words(d->n_out);
     A->nwp = entry_words_padded(d->n_out);
     A->nchunks = table_chunks(d->n_in, A->nwp);
     A->cb = chunk_bits(d->n_in, A->nwp);
-    A->rows = (const uint32_t *)(b + d->off_xornet);
+    A->tab_words = table_words(d->n_out, d->n_in);
+    // the table geometry is a fixed function of the shape; a descriptor that says otherwise is not ours
+    if (d->tab_entry_words != A->nwp || d->tab_chunks != A->nchunks || d->tab_chunk_bits != A->cb ||
+        d->tables_bytes != (uint64_t)A->tab_words * 4 || d->off_tables % 16 != 0)
+        return SQNN_E_INVALID_ARG;
+    A->tab = (const uint32_t *)(b + d->off_tables);
     A->status = d_status;
     for (uint32_t i = 0; i < d->n_q; ++i) {
-        if (d->off_wc[i] % 16 || d->off_np[i] % 16 || d->off_idx[i] % 16 || d->off_dp[i] % 16 ||
-            d->n_dp[i] > 0xffffffffull || d->w_np[i] > 9)
+        if (d->off_wc[i] % 16 || d->off_idx[i] % 16 || d->off_pp[i] % 16 || d->n_pp[i] > 0xffffffffull)
             return SQNN_E_INVALID_ARG;
         A->pl[i].wc = (const uint32_t *)(b + d->off_wc[i]);
-        A->pl[i].np = (const uint32_t *)(b + d->off_np[i]);
         A->pl[i].idx = (const uint32_t *)(b + d->off_idx[i]);
-        A->pl[i].dp = b + d->off_dp[i];
-        A->pl[i].n_dp = (uint32_t)d->n_dp[i];
-        A->pl[i].w_np = d->w_np[i];
+        A->pl[i].pp = (const uint16_t *)(b + d->off_pp[i]);
+        A->pl[i].n_pp = (uint32_t)d->n_pp[i];
     }
     for (uint32_t i = d->n_q; i < 8; ++i) A->pl[i] = A->pl[0];
     return SQNN_OK;
@@ -93,33 +96,15 @@ int sm_count()
 }
 
 
-// Clears Y[b][r] (row stride ldy); dependents may be launched as soon as every block has started.
-__global__ void k_clear_y(float *__restrict__ y, int64_t ldy, uint64_t m, uint64_t cells)
-{
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < cells; i += (uint64_t)gridDim.x * blockDim.x) {
-        const uint64_t b = i / m;
-        y[(int64_t)b * ldy + (int64_t)(i - b * m)] = 0.0f;
-    }
-}
-
 static int gemv_dispatch(const DecodeArgs &A, const uint64_t *d_mask, const float *d_alpha, const void *d_x,
                          int x_dtype, int64_t ldx, uint32_t batch, float *d_y, int64_t ldy, uint64_t m, uint64_t n,
                          cudaStream_t st)
 {
-    // Y is accumulated with atomics: clear it first.  The clearing kernel lets the product kernel
-    // start at once (programmatic dependent launch); that one waits for the cleared Y only before
-    // its first atomic, so its launch and its first fetches overlap the clearing.
-    const uint64_t cells = (uint64_t)batch * m;
-    uint64_t blocks = (cells + 1023) / 1024;
-    if (blocks > (uint64_t)sm_count()) blocks = (uint64_t)sm_count();
-    k_clear_y<<<(uint32_t)blocks, 256, 0, st>>>(d_y, ldy, m, cells);
-    if (cudaGetLastError() != cudaSuccess) return SQNN_E_CUDA;
 #define SQNN_GEMV_CASE(NO, NI) \
-    if (A.n_out == NO && A.n_in == NI) return gemv_shape<NO, NI>(A, d_mask, d_alpha, d_x, x_dtype, ldx, batch, d_y, ldy, n, st);
+    if (A.n_out == NO && A.n_in == NI) return gemv_shape<NO, NI>(A, d_mask, d_alpha, d_x, x_dtype, ldx, batch, d_y, ldy, m, n, st);
     SQNN_FOR_SHAPES(SQNN_GEMV_CASE)
 #undef SQNN_GEMV_CASE
-    return gemv_shape<0, 0>(A, d_mask, d_alpha, d_x, x_dtype, ldx, batch, d_y, ldy, n, st);
+    return gemv_shape<0, 0>(A, d_mask, d_alpha, d_x, x_dtype, ldx, batch, d_y, ldy, m, n, st);
 }
 
 int decode_bits_dispatch(const DecodeArgs &A, void *d_out, cudaStream_t st)
@@ -184,10 +169,9 @@ extern "C" int sqnn_decode_matmul(const sqnn_desc *desc, const void *d_blob, con
     if (batch <= 15)
         return gemv_dispatch(A, d_mask, d_alpha, d_x, x_dtype, ldx, batch, d_y, ldy, desc->m, desc->n, st);
     if (x_dtype != SQNN_X_BF16) return SQNN_E_UNSUPPORTED;
-    // With a workspace the planes are decoded to packed bits first (fast tiled decoder) and the
-    // tensor-core kernel reads them from there; without one it decodes inside the kernel (slower).
-    if (d_workspace) {
-        if (workspace_bytes < mma_workspace_bytes(desc, batch) || ((uintptr_t)d_workspace & 255)) return SQNN_E_WORKSPACE;
-    }
+    // The planes are decoded to packed bits in the workspace first; the tensor-core kernel reads
+    // them from there.
+    if (!d_workspace || workspace_bytes < mma_workspace_bytes(desc, batch) || ((uintptr_t)d_workspace & 255))
+        return SQNN_E_WORKSPACE;
     return mma_dispatch(desc, A, d_mask, d_alpha, d_x, ldx, batch, d_y, ldy, d_workspace, st);
 }

@@ -1,10 +1,10 @@
-// On-disk / in-memory header of a packed blob (internal to the library).
+// Header of a device blob (internal to the library).
 #ifndef SQNN_BLOB_H_
 #define SQNN_BLOB_H_
 #include "sqnn.h"
 
-#define SQNN_BLOB_MAGIC        "SQNNBLB1"
-#define SQNN_BLOB_VERSION      1u
+#define SQNN_BLOB_MAGIC        "SQNNBLB2"
+#define SQNN_BLOB_VERSION      2u
 #define SQNN_BLOB_HEADER_BYTES 512u
 
 typedef struct sqnn_blob_header {

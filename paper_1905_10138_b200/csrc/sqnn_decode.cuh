@@ -1,19 +1,24 @@
 // Device-side decryption of one warp tile: seeds -> XOR-gate network (table lookup) ->
 // patch flips, producing a run of consecutive output words in shared memory.
 //
-// Work split.  A lane owns G consecutive slices, G a multiple of 4 chosen so that G * n_out is
-// a multiple of 32 bits; its W = G * n_out / 32 output words are private to it while it expands
-// and patches.  A warp tile is therefore 32 * G consecutive slices = 32 * W consecutive 32-bit
-// words of the flattened plane, and it starts on a boundary of the per-128-slice d_patch
-// offsets.  In the packed streams a tile is G * n_in words of seeds and G * w_np words of
-// n_patch counts.
+// Work split.  A lane owns G consecutive slices, G = 8 * KT with KT the number of format tiles
+// (256 slices) per kernel tile, chosen so that G * n_out is a multiple of 32 bits; its
+// W = G * n_out / 32 output words are private to it while it expands.  A kernel tile is therefore
+// 32 * G consecutive slices = 32 * W consecutive 32-bit words of the flattened plane.  In the
+// seed stream a lane's 8 slices of one format tile are n_in consecutive bytes.
 //
-// The network (Section 3.1, w~ = M . w^c) is evaluated with tables: the seed is cut into
-// chunks of cb bits and table[chunk][value] holds the XOR of the columns of M selected by
-// the value, as an n_out-bit word padded to nwp 32-bit words.
+// The network (Section 3.1, w~ = M . w^c) is evaluated with the lookup tables stored in the
+// blob (geometry in sqnn_layout.h), copied to shared memory once per block.
+//
+// Patches (Section 3.2) come per format tile as 16-bit bit positions inside the tile; the warp
+// flips them in the shared-memory copy of the tile with one shared-memory reduction each, lanes
+// taking entries in turn -- no counts, no prefix sum.
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
+
+#include "sqnn.h"
+#include "sqnn_layout.h"
 
 #define SQNN_DEV __device__ __forceinline__
 
@@ -21,54 +26,24 @@ namespace sqnn {
 
 struct PlanePtrs {
     const uint32_t *wc;    // seed stream
-    const uint32_t *np;    // n_patch stream (unused when w_np == 0)
-    const uint32_t *idx;   // d_patch entries before each block of 128 slices
-    const uint8_t *dp;     // d_patch entries
-    uint32_t n_dp;
-    uint32_t w_np;
+    const uint32_t *idx;   // patch entries before each format tile (+ closing entry)
+    const uint16_t *pp;    // patch entries: bit position inside the format tile
+    uint32_t n_pp;
 };
 
 struct DecodeArgs {
     uint64_t mn;           // weights per plane
     uint64_t words64;      // ceil(mn / 64)
-    uint64_t tiles;        // warp tiles per plane
+    uint64_t ktiles;       // kernel tiles per plane (padded stream)
     uint32_t n_out, n_in, n_q;
-    uint32_t G, W;         // slices and words per lane
+    uint32_t KT, G, W;     // format tiles per kernel tile, slices and words per lane
     uint32_t nw, nwp;      // words per table entry: used, padded (1, 2, 4, 8)
     uint32_t nchunks, cb;  // table chunks, bits per chunk
-    const uint32_t *rows;  // rows of M
+    uint32_t tab_words;    // words of all tables (multiple of 4)
+    const uint32_t *tab;   // tables in the blob
     uint32_t *status;      // sticky error word or NULL
     PlanePtrs pl[8];
 };
-
-__host__ __device__ constexpr uint32_t gcd_u32(uint32_t a, uint32_t b) { return b == 0 ? a : gcd_u32(b, a % b); }
-// Smallest multiple of 4 slices whose bits fill whole words, doubled (up to 8) while the lane
-// would own fewer than 16 words, so that small networks still get tiles worth their overhead.
-__host__ __device__ constexpr uint32_t slices_per_lane(uint32_t n_out)
-{
-    uint32_t g = 32 / gcd_u32(n_out, 32);
-    if (g < 4) g = 4;
-    while (g < 8 && g * n_out / 32 < 16) g *= 2;
-    return g;
-}
-__host__ __device__ constexpr uint32_t entry_words(uint32_t n_out) { return (n_out + 31) / 32; }
-__host__ __device__ constexpr uint32_t entry_words_padded(uint32_t n_out)
-{
-    return entry_words(n_out) <= 1 ? 1 : entry_words(n_out) <= 2 ? 2 : entry_words(n_out) <= 4 ? 4 : 8;
-}
-// Fewest chunks whose tables stay within 48 KB.
-__host__ __device__ constexpr uint32_t table_chunks(uint32_t n_in, uint32_t nwp)
-{
-    for (uint32_t c = 1; c <= 8; ++c) {
-        uint32_t cb = (n_in + c - 1) / c;
-        if (cb <= 14 && (uint64_t)c * (1ull << cb) * nwp * 4 <= 48 * 1024) return c;
-    }
-    return 8;
-}
-__host__ __device__ constexpr uint32_t chunk_bits(uint32_t n_in, uint32_t nwp)
-{
-    return (n_in + table_chunks(n_in, nwp) - 1) / table_chunks(n_in, nwp);
-}
 
 SQNN_DEV uint32_t extract_bits(const uint32_t *__restrict__ base, uint64_t bitpos, uint32_t width)
 {
@@ -101,375 +76,242 @@ SQNN_DEV void bulk_wait_read()
 }
 SQNN_DEV void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory"); }
 
-// Shared-memory words the tables need, rounded so that what follows stays 16-byte aligned.
-inline __host__ __device__ uint32_t table_words(uint32_t n_in, uint32_t nwp, uint32_t nchunks, uint32_t cb)
+SQNN_DEV void cp_async16(void *sdst, const void *gsrc)
 {
-    return (nchunks * (1u << cb) * nwp + n_in * nwp + 3u) & ~3u;
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" :: "r"(smem_addr(sdst)), "l"(gsrc) : "memory");
+}
+SQNN_DEV void cp_async4(void *sdst, const void *gsrc)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;\n" :: "r"(smem_addr(sdst)), "l"(gsrc) : "memory");
+}
+SQNN_DEV void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int PENDING>
+SQNN_DEV void cp_async_wait_group() { asm volatile("cp.async.wait_group %0;\n" :: "n"(PENDING) : "memory"); }
+SQNN_DEV void cp_async_wait_all() { asm volatile("cp.async.wait_all;\n" ::: "memory"); }
+
+// Flips one bit of a shared-memory word (address given as a 32-bit shared address).
+SQNN_DEV void smem_flip(uint32_t region_sa, uint32_t bit)
+{
+    asm volatile("red.shared.xor.b32 [%0], %1;\n" :: "r"(region_sa + ((bit >> 5) << 2)), "r"(1u << (bit & 31u)) : "memory");
 }
 
-// Builds the column words of M and the chunk tables.  All threads of the block take part.
-// An entry's value splits as (high << lo_bits) | low: entries with only low or only high bits
-// are XORed together from the columns directly, every other entry is the XOR of those two.
-// The build comes in two calls so that a kernel can request the rows of M first, start its other
-// fetches, and only then wait: build_tables_begin stores the rows in shared memory (block
-// barrier), build_tables_finish does the rest (ends with a block barrier).
-struct RowsAhead { uint32_t r0, r1; };              // rows threadIdx.x and threadIdx.x + blockDim.x
-
-SQNN_DEV uint32_t *rows_scratch()
+// Starts the copy of the lookup tables from the blob into shared memory (all threads of the
+// block; one commit group).  Wait for the group and pass a block barrier before the first lookup.
+SQNN_DEV void tables_request(const DecodeArgs &A, uint32_t *tab_s)
 {
-    __shared__ uint32_t rows_s[256];
-    return rows_s;
+    for (uint32_t v = threadIdx.x; v < A.tab_words / 4; v += blockDim.x) cp_async16(tab_s + 4 * v, A.tab + 4 * v);
+    cp_async_commit();
 }
 
-SQNN_DEV RowsAhead fetch_rows(const DecodeArgs &A)
-{
-    RowsAhead p{0u, 0u};
-    if (threadIdx.x < A.n_out) p.r0 = __ldg(A.rows + threadIdx.x);
-    if (threadIdx.x + blockDim.x < A.n_out) p.r1 = __ldg(A.rows + threadIdx.x + blockDim.x);
-    return p;
-}
-
-SQNN_DEV void build_tables_begin(const DecodeArgs &A, RowsAhead ahead)
-{
-    uint32_t *rows_s = rows_scratch();
-    const uint32_t n_out = A.n_out;
-    if (threadIdx.x < n_out) rows_s[threadIdx.x] = ahead.r0;
-    if (threadIdx.x + blockDim.x < n_out) rows_s[threadIdx.x + blockDim.x] = ahead.r1;
-    for (uint32_t j = threadIdx.x + 2 * blockDim.x; j < n_out; j += blockDim.x) rows_s[j] = __ldg(A.rows + j);
-    __syncthreads();
-}
-
-// N_OUT, N_IN: the network shape when it is known at compile time (the index arithmetic then folds), 0 = read it from A.
-// WAIT_ASYNC: the thread's pending cp.async copies are awaited just before the closing barrier, so that what they
-// bring in is visible to the whole block after it while the build itself runs under their latency.
-template <int N_OUT = 0, int N_IN = 0, bool WAIT_ASYNC = false>
-SQNN_DEV void build_tables_finish(const DecodeArgs &A, uint32_t *tab)
-{
-    const uint32_t *rows_s = rows_scratch();
-    constexpr bool CT = N_OUT != 0;
-    constexpr uint32_t NWP_C = entry_words_padded(CT ? N_OUT : 32);
-    const uint32_t nwp = CT ? NWP_C : A.nwp, n_in = CT ? (uint32_t)N_IN : A.n_in, n_out = CT ? (uint32_t)N_OUT : A.n_out;
-    const uint32_t cb = CT ? chunk_bits(CT ? N_IN : 8, NWP_C) : A.cb;
-    const uint32_t nchunks = CT ? table_chunks(CT ? N_IN : 8, NWP_C) : A.nchunks;
-    const uint32_t kshift = nwp == 1 ? 0 : nwp == 2 ? 1 : nwp == 4 ? 2 : 3;
-    uint32_t *cols = tab + nchunks * (1u << cb) * nwp;
-    // word k of column t: bit j of it is bit t of row 32 k + j -- one ballot over 32 rows
-    const uint32_t lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
-    for (uint32_t i = threadIdx.x >> 5; i < n_in * nwp; i += nwarps) {
-        const uint32_t t = i >> kshift, k = i & (nwp - 1);
-        const uint32_t j = 32 * k + lane;
-        const uint32_t r = j < n_out ? rows_s[j] : 0u;
-        const uint32_t w = __ballot_sync(0xffffffffu, (r >> t) & 1u);
-        if (lane == 0) cols[i] = w;
-    }
-    __syncthreads();
-    const uint32_t lo_bits = cb / 2, hi_bits = cb - lo_bits;
-    const uint32_t n_lo = 1u << lo_bits, n_hi = 1u << hi_bits;
-    const uint32_t direct = (n_lo + n_hi - 1) * nwp;          // per chunk: low-only and high-only entries
-    for (uint32_t i = threadIdx.x; i < nchunks * direct; i += blockDim.x) {
-        const uint32_t ch = i / direct, r = i - ch * direct;
-        const uint32_t k = r & (nwp - 1), e = r >> kshift;
-        const uint32_t v = e < n_lo ? e : (e - n_lo + 1) << lo_bits;
-        uint32_t x = 0;
-#pragma unroll 4
-        for (uint32_t b = 0; b < cb; ++b) {
-            const uint32_t t = ch * cb + b;
-            if (t < n_in && ((v >> b) & 1u)) x ^= cols[(t << kshift) + k];
-        }
-        tab[((((ch << cb) | v)) << kshift) + k] = x;
-    }
-    __syncthreads();
-    const uint32_t total = nchunks * (1u << cb) * nwp;
-    for (uint32_t i = threadIdx.x; i < total; i += blockDim.x) {
-        const uint32_t k = i & (nwp - 1), e = i >> kshift;
-        const uint32_t v = e & ((1u << cb) - 1u);
-        const uint32_t l = v & (n_lo - 1), h = v & ~(n_lo - 1);
-        if (l != 0 && h != 0) {
-            const uint32_t chbase = e - v;
-            tab[i] = tab[((chbase | l) << kshift) + k] ^ tab[((chbase | h) << kshift) + k];
-        }
-    }
-    if constexpr (WAIT_ASYNC) asm volatile("cp.async.wait_all;\n" ::: "memory");
-    __syncthreads();
-}
-
-template <int N_OUT = 0, int N_IN = 0>
-SQNN_DEV void build_tables(const DecodeArgs &A, uint32_t *tab)
-{
-    build_tables_begin(A, fetch_rows(A));
-    build_tables_finish<N_OUT, N_IN>(A, tab);
-}
-
+// The same tables, replicated for conflict-free lookups (sqnn_layout.h): element (entry e, copy j)
+// -- for 32-byte entries (entry e, half h, copy j) -- is stored at consecutive 16-byte (or smaller)
+// slots in the order of its linear index, so the fill is a coalesced copy in which 32 / NWP
+// consecutive threads store the same entry.  All threads of the block; ends without a barrier.
 template <int NWP>
-SQNN_DEV void load_entry(const uint32_t *tab, uint32_t e, uint32_t (&x)[NWP])
+SQNN_DEV void tables_replicate(const DecodeArgs &A, uint32_t *tab_s)
 {
+    constexpr uint32_t R = table_copies(NWP);
+    constexpr uint32_t VW = NWP >= 4 ? 4 : NWP;                  // words per stored element (16, 8 or 4 bytes)
+    constexpr uint32_t PER = 32 / R;                             // source elements one warp store covers
+    const uint32_t elems = (A.nchunks << A.cb) * (NWP / VW);     // source elements (halves count separately)
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    // a warp takes 32 source elements at a time: one coalesced load, then R stores of 32 consecutive
+    // replicated elements each, the values handed round by shuffles
+    for (uint32_t e0 = warp * 32; e0 < elems; e0 += nwarps * 32) {
+        uint32_t v[VW];
+#pragma unroll
+        for (uint32_t k = 0; k < VW; ++k) v[k] = 0;
+        if (e0 + lane < elems) {
+            if constexpr (VW == 4) {
+                const uint4 t = __ldg(reinterpret_cast<const uint4 *>(A.tab + 4 * (e0 + lane)));
+                v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+            } else if constexpr (VW == 2) {
+                const uint2 t = __ldg(reinterpret_cast<const uint2 *>(A.tab + 2 * (e0 + lane)));
+                v[0] = t.x; v[1] = t.y;
+            } else {
+                v[0] = __ldg(A.tab + e0 + lane);
+            }
+        }
+#pragma unroll
+        for (uint32_t j = 0; j < R; ++j) {
+            const uint32_t src = j * PER + lane / R;             // source element (within the 32) of this lane's store
+            uint32_t o[VW];
+#pragma unroll
+            for (uint32_t k = 0; k < VW; ++k) o[k] = __shfl_sync(0xffffffffu, v[k], src);
+            const uint32_t i = (e0 + j * PER) * R + lane;        // replicated element index
+            if (e0 + src < elems) {
+                if constexpr (VW == 4) *reinterpret_cast<uint4 *>(tab_s + 4 * i) = make_uint4(o[0], o[1], o[2], o[3]);
+                else if constexpr (VW == 2) *reinterpret_cast<uint2 *>(tab_s + 2 * i) = make_uint2(o[0], o[1]);
+                else tab_s[i] = o[0];
+            }
+        }
+    }
+}
+
+// Entry e of the tables in shared memory.  REP: from the replicated tables, through the copy of this lane.
+template <int NWP, bool REP>
+SQNN_DEV void load_entry(const uint32_t *tab, uint32_t e, uint32_t lane, uint32_t (&x)[NWP])
+{
+    constexpr uint32_t R = table_copies(NWP);
     if constexpr (NWP == 1) {
-        x[0] = tab[e];
+        x[0] = REP ? tab[e * R + lane] : tab[e];
     } else if constexpr (NWP == 2) {
-        const uint2 v = *reinterpret_cast<const uint2 *>(tab + 2 * e);
+        const uint2 v = *reinterpret_cast<const uint2 *>(tab + 2 * (REP ? e * R + (lane & (R - 1)) : e));
         x[0] = v.x; x[1] = v.y;
     } else if constexpr (NWP == 4) {
-        const uint4 v = *reinterpret_cast<const uint4 *>(tab + 4 * e);
+        const uint4 v = *reinterpret_cast<const uint4 *>(tab + 4 * (REP ? e * R + (lane & (R - 1)) : e));
         x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
     } else {
-        const uint4 v = *reinterpret_cast<const uint4 *>(tab + 8 * e);
-        const uint4 u = *reinterpret_cast<const uint4 *>(tab + 8 * e + 4);
+        const uint32_t i0 = REP ? (2 * e) * R + (lane & (R - 1)) : 2 * e;
+        const uint32_t i1 = REP ? (2 * e + 1) * R + (lane & (R - 1)) : 2 * e + 1;
+        const uint4 v = *reinterpret_cast<const uint4 *>(tab + 4 * i0);
+        const uint4 u = *reinterpret_cast<const uint4 *>(tab + 4 * i1);
         x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
         x[4] = u.x; x[5] = u.y; x[6] = u.z; x[7] = u.w;
     }
 }
 
-// Per-warp scratch of the patch step: 128 words of staged d_patch bytes (one window of up to
-// PATCH_WIN entries, after up to 3 bytes of alignment) and one 16-bit mark per entry of the window.
-constexpr uint32_t PATCH_WIN = 508;
-constexpr uint32_t STAGE_DP_WORDS = 128;
-constexpr uint32_t STAGE_WORDS = STAGE_DP_WORDS + 256;
-
-// Compile-time facts of a network shape.
+// Compile-time facts of a network shape (n_out a multiple of 4: one format tile per kernel tile).
 template <int N_OUT, int N_IN>
 struct Shape {
+    static_assert(N_OUT % 4 == 0, "compile-time shapes have n_out a multiple of 4");
     static constexpr uint32_t n_out = N_OUT, n_in = N_IN;
-    static constexpr uint32_t G = slices_per_lane(N_OUT), W = G * N_OUT / 32;
+    static constexpr uint32_t G = 8, W = N_OUT / 4;
     static constexpr uint32_t NW = entry_words(N_OUT), NWP = entry_words_padded(N_OUT);
     static constexpr uint32_t NCH = table_chunks(N_IN, NWP), CB = chunk_bits(N_IN, NWP);
-    static constexpr uint32_t SPAN = G * N_IN, NSW = (SPAN + 31) / 32;
-    static_assert(G <= 8, "compile-time shapes keep at most 8 slices per lane");
+    static constexpr uint32_t SPAN = 8 * N_IN;                       // seed bits of one lane
+    static constexpr bool ALIGNED = SPAN % 32 == 0;                   // a lane's seeds start on a word
+    static constexpr uint32_t NSW = (SPAN + 31) / 32;                 // words holding them
+    static constexpr uint32_t NRAW = ALIGNED ? NSW : NSW + 1;
+    static constexpr uint32_t TILE_BITS = SQNN_TILE_SLICES * N_OUT;
 };
 
-// What one lane reads from global memory for one tile of one plane.
+// The words holding a lane's 8 seeds of one tile.
 template <int N_OUT, int N_IN>
-struct TileIn {
-    uint32_t raw[Shape<N_OUT, N_IN>::NSW + 1];   // words holding the lane's G seeds
-    uint32_t np0, np1, np2;                      // words holding the lane's G n_patch fields
-    uint32_t base, total;                        // the tile's run of d_patch entries
+struct TileSeeds {
+    uint32_t raw[Shape<N_OUT, N_IN>::NRAW];
 };
+// A tile's run of patch entries [base, end) and the first words of it, fetched ahead of time:
+// lane l holds 32-bit words (base >> 1) + l + 32 k, k < 4, of the entry array (two entries each).
+struct TileRun {
+    uint32_t base, end;
+};
+constexpr uint32_t PATCH_AHEAD = 4;
 
 template <int N_OUT, int N_IN>
-SQNN_DEV void tile_fetch(const PlanePtrs &P, uint64_t tile, uint32_t lane, TileIn<N_OUT, N_IN> &in)
+SQNN_DEV void fetch_seeds(const PlanePtrs &P, uint64_t tile, uint32_t lane, TileSeeds<N_OUT, N_IN> &s)
 {
     using S = Shape<N_OUT, N_IN>;
-    const uint32_t *w = P.wc + tile * (S::G * S::n_in) + ((lane * S::SPAN) >> 5);
+    const uint32_t *w = P.wc + tile * (8 * S::n_in) + ((lane * S::SPAN) >> 5);
+    if constexpr (S::ALIGNED && S::NSW == 4) {
+        const uint4 v = __ldg(reinterpret_cast<const uint4 *>(w));
+        s.raw[0] = v.x; s.raw[1] = v.y; s.raw[2] = v.z; s.raw[3] = v.w;
+    } else if constexpr (S::ALIGNED && S::NSW == 2) {
+        const uint2 v = __ldg(reinterpret_cast<const uint2 *>(w));
+        s.raw[0] = v.x; s.raw[1] = v.y;
+    } else {
 #pragma unroll
-    for (uint32_t k = 0; k <= S::NSW; ++k) in.raw[k] = __ldg(w + k);
-    in.base = in.total = in.np0 = in.np1 = in.np2 = 0;
-    if (P.w_np != 0) {
-        const uint32_t *ix = P.idx + tile * (S::G / 4);
-        in.base = __ldg(ix);
-        in.total = __ldg(ix + S::G / 4) - in.base;
-        const uint32_t *q = P.np + tile * (S::G * P.w_np) + ((lane * S::G * P.w_np) >> 5);
-        in.np0 = __ldg(q);
-        in.np1 = __ldg(q + 1);
-        in.np2 = __ldg(q + 2);
+        for (uint32_t k = 0; k < S::NRAW; ++k) s.raw[k] = __ldg(w + k);     // sections end with slack
     }
 }
 
-// The tile's staged d_patch words: lane l fetches words l, l + 32, l + 64, l + 96 of the run.
-template <int N_OUT, int N_IN>
-SQNN_DEV void stage_fetch(const DecodeArgs &A, const PlanePtrs &P, TileIn<N_OUT, N_IN> &in, uint32_t lane,
-                          uint32_t (&st)[4])
+SQNN_DEV TileRun fetch_run(const PlanePtrs &P, uint64_t tile)
 {
-    st[0] = st[1] = st[2] = st[3] = 0;
-    if (in.total == 0) return;
-    if (in.base > P.n_dp || in.total > P.n_dp - in.base) {       // offsets point outside the section
-        flag(A.status, 2u);
-        in.total = 0;
-        return;
-    }
-    const uint32_t nbytes = in.total < PATCH_WIN ? in.total : PATCH_WIN;
-    const uint32_t nwords = ((in.base & 3u) + nbytes + 3) >> 2;
-    const uint32_t *src = reinterpret_cast<const uint32_t *>(P.dp) + (in.base >> 2);
-#pragma unroll
-    for (uint32_t j = 0; j < 4; ++j)
-        if (lane + 32 * j < nwords) st[j] = __ldg(src + lane + 32 * j);
+    TileRun r;
+    r.base = __ldg(P.idx + tile);
+    r.end = __ldg(P.idx + tile + 1);
+    return r;
 }
 
-// Flips the patched positions of a tile (Section 3.2), the warp working through the tile's run of
-// d_patch entries 32 at a time.  An entry does not say which slice it belongs to; that follows
-// from the n_patch counts.  Each lane knows where the entries of its own G slices start (a warp
-// scan of the per-lane counts), so it drops a mark (the slice's first bit + 1) at the index of each of its
-// slices' first entry; every entry then takes the nearest mark at or before it (a ballot and one
-// shuffle per 32 entries), and the lane holding the entry flips bit slice * n_out + position of
-// the tile with a shared-memory atomic.  Runs longer than PATCH_WIN entries are handled in
-// windows, the last mark carrying over.  `win` holds the lane's n_patch fields (G fields of w_np bits, lowest first),
-// `st` the first window's d_patch words fetched ahead of time.
-template <uint32_t G, uint32_t N_OUT, typename WT>
-SQNN_DEV void patch_tile(const DecodeArgs &A, const PlanePtrs &P, uint32_t *region, uint32_t *stage,
-                         const uint32_t (&st)[4], uint32_t base, uint32_t total, WT win, uint32_t lane)
+// Checks the run against the section and requests its first words.
+SQNN_DEV void fetch_patches(const DecodeArgs &A, const PlanePtrs &P, TileRun &run, uint32_t lane,
+                            uint32_t (&pw)[PATCH_AHEAD])
 {
-    const uint32_t w_np = P.w_np;
-    const uint32_t fm = (1u << w_np) - 1u;
-    uint32_t f[G];
-    uint32_t cnt = 0;
-#pragma unroll
-    for (uint32_t i = 0; i < G; ++i) {
-        f[i] = (uint32_t)(win >> (i * w_np)) & fm;
-        cnt += f[i];
-    }
-    uint32_t incl = cnt;
-#pragma unroll
-    for (uint32_t d = 1; d < 32; d <<= 1) {
-        const uint32_t v = __shfl_up_sync(0xffffffffu, incl, d);
-        if (lane >= d) incl += v;
-    }
-    const uint32_t first = incl - cnt;
-    if (__shfl_sync(0xffffffffu, incl, 31) != total) {      // counts disagree with the offsets
+    if (run.end < run.base || run.end > P.n_pp) {                // offsets point outside the section
         flag(A.status, 2u);
-        return;
+        run.end = run.base = 0;
     }
-    uint32_t *marks32 = stage + STAGE_DP_WORDS;
-    uint16_t *marks = reinterpret_cast<uint16_t *>(marks32);
-    const uint32_t below_me = 0xffffffffu >> (31 - lane);   // lanes 0 .. lane
-    uint32_t carry = 0, bad = 0;
-    for (uint32_t w0 = 0; w0 < total; w0 += PATCH_WIN) {
-        const uint32_t wn = total - w0 < PATCH_WIN ? total - w0 : PATCH_WIN;
-        const uint32_t ob = (base + w0) & 3u;
-        if (w0 == 0) {
+    const uint32_t *pp32 = reinterpret_cast<const uint32_t *>(P.pp);
+    const uint32_t w0 = run.base >> 1, wend = (run.end + 1) >> 1;
 #pragma unroll
-            for (uint32_t j = 0; j < 4; ++j) stage[lane + 32 * j] = st[j];
-        } else {
-            const uint32_t nwords = (ob + wn + 3) >> 2;
-            const uint32_t *src = reinterpret_cast<const uint32_t *>(P.dp) + ((base + w0) >> 2);
-#pragma unroll
-            for (uint32_t j = 0; j < 4; ++j)
-                if (lane + 32 * j < nwords) stage[lane + 32 * j] = __ldg(src + lane + 32 * j);
-        }
-        // marks of whole 64-entry groups are cleared, so the last group reads zeros past wn
-        for (uint32_t q = lane; q < ((wn + 63) >> 6) * 32; q += 32) marks32[q] = 0;
-        __syncwarp();
-        // mark = first tile bit of the slice + 1, dropped at the slice's first entry
-        uint32_t run = first - w0;
-#pragma unroll
-        for (uint32_t i = 0; i < G; ++i) {
-            if (f[i] != 0 && run < wn) marks[run] = (uint16_t)((lane * G + i) * N_OUT + 1);
-            run += f[i];
-        }
-        __syncwarp();
-        const uint8_t *bytes = reinterpret_cast<const uint8_t *>(stage) + ob;
-        // two groups of 32 entries per round (two independent chains of shared-memory reads and
-        // shuffles); every entry takes the nearest mark at or before it, else the carry
-        for (uint32_t e0 = 0; e0 < wn; e0 += 64) {
-            const uint32_t ea = e0 + lane, eb = ea + 32;
-            uint32_t va = marks[ea], vb = marks[eb];
-            const uint32_t pa = bytes[ea], pb = bytes[eb];
-            const uint32_t sa = __ballot_sync(0xffffffffu, va != 0) & below_me;
-            const uint32_t sb = __ballot_sync(0xffffffffu, vb != 0) & below_me;
-            const uint32_t ga = __shfl_sync(0xffffffffu, va, (31 - __clz((int)sa)) & 31);
-            const uint32_t gb = __shfl_sync(0xffffffffu, vb, (31 - __clz((int)sb)) & 31);
-            va = sa ? ga : carry;
-            const uint32_t ca = __shfl_sync(0xffffffffu, va, 31);
-            vb = sb ? gb : ca;
-            carry = __shfl_sync(0xffffffffu, vb, 31);
-            const bool la = ea < wn, lb = eb < wn;
-            const bool oka = la && va != 0 && pa < N_OUT, okb = lb && vb != 0 && pb < N_OUT;
-            bad |= (uint32_t)((la && !oka) || (lb && !okb));
-            if (oka) {
-                const uint32_t bit = va - 1 + pa;
-                atomicXor(region + (bit >> 5), 1u << (bit & 31));
-            }
-            if (okb) {
-                const uint32_t bit = vb - 1 + pb;
-                atomicXor(region + (bit >> 5), 1u << (bit & 31));
-            }
-        }
-        __syncwarp();
+    for (uint32_t k = 0; k < PATCH_AHEAD; ++k) {
+        const uint32_t aw = w0 + lane + 32 * k;
+        pw[k] = aw < wend ? __ldg(pp32 + aw) : 0u;
     }
-    if (bad) flag(A.status, 1u);
 }
 
-// The same patch step for runs that fit one window (at most PATCH_WIN entries), which is nearly
-// every tile at the patch densities the format is meant for.  Differences from patch_tile: a lane handles
-// the four entries of one staged d_patch word a round, straight from the register it was fetched into
-// (nothing but the marks goes through shared memory); marks are indexed by byte position in the staged
-// words and, since they grow along the run, "nearest mark at or before" is a running maximum -- three
-// maxima inside the lane, one ballot and one shuffle across lanes, one shuffle to carry it into the next
-// round.
-template <uint32_t G, uint32_t N_OUT, typename WT>
-SQNN_DEV void patch_tile_fast(const DecodeArgs &A, const PlanePtrs &P, uint32_t *region, uint32_t *stage,
-                              const uint32_t (&st)[4], uint32_t base, uint32_t total, WT win, uint32_t lane)
+// One patch entry: flips bit bit0 + pos of the region if the entry belongs to the run (t < total,
+// t = its index minus the run's base, as unsigned) and pos lies inside the tile.  Branch-free: the
+// reduction is predicated.  Returns pos if the entry belongs to the run, else 0 (for the range check).
+SQNN_DEV uint32_t flip_entry(uint32_t region_sa, uint32_t bit0, uint32_t tile_bits, uint32_t pos, uint32_t t, uint32_t total)
 {
-    const uint32_t w_np = P.w_np;
-    const uint32_t fm = (1u << w_np) - 1u;
-    uint32_t f[G];
-    uint32_t cnt = 0;
-#pragma unroll
-    for (uint32_t i = 0; i < G; ++i) {
-        f[i] = (uint32_t)win & fm;
-        win >>= w_np;
-        cnt += f[i];
-    }
-    uint32_t incl = cnt;
-#pragma unroll
-    for (uint32_t d = 1; d < 32; d <<= 1) {
-        const uint32_t v = __shfl_up_sync(0xffffffffu, incl, d);
-        if (lane >= d) incl += v;
-    }
-    if (__shfl_sync(0xffffffffu, incl, 31) != total) {      // counts disagree with the offsets
-        flag(A.status, 2u);
-        return;
-    }
-    const uint32_t ob = base & 3u;                           // entry 0 sits at byte `ob` of the staged words
-    const uint32_t rounds = (ob + total + 127u) >> 7;        // 128 byte positions a round, at most 4 rounds
-    uint32_t *marks32 = stage + STAGE_DP_WORDS;
-    uint2 *marks64 = reinterpret_cast<uint2 *>(marks32);
-    uint16_t *marks = reinterpret_cast<uint16_t *>(marks32);
-    for (uint32_t j = 0; j < rounds; ++j) marks64[32 * j + lane] = make_uint2(0u, 0u);
-    __syncwarp();
-    // mark = first tile bit of the slice + 1, dropped at the byte position of the slice's first entry
-    uint32_t run = ob + incl - cnt, mark = lane * G * N_OUT + 1u;
-#pragma unroll
-    for (uint32_t i = 0; i < G; ++i) {
-        if (f[i] != 0) marks[run] = (uint16_t)mark;
-        run += f[i];
-        mark += N_OUT;
-    }
-    __syncwarp();
-    const uint32_t lower = (1u << lane) - 1u;                // lanes below this one
-    uint32_t carry = 0, bad = 0;
-#pragma unroll
-    for (uint32_t j = 0; j < 4; ++j) {
-        if (j < rounds) {                                    // the same in every lane
-            const uint2 mm = marks64[32 * j + lane];
-            const uint32_t m0 = mm.x & 0xffffu, m1 = mm.x >> 16, m2 = mm.y & 0xffffu, m3 = mm.y >> 16;
-            const uint32_t last = max(max(m0, m1), max(m2, m3));
-            const uint32_t have = __ballot_sync(0xffffffffu, last != 0) & lower;
-            const uint32_t got = __shfl_sync(0xffffffffu, last, (31 - __clz((int)have)) & 31);
-            const uint32_t prev = have ? got : carry;
-            uint32_t v[4];
-            v[0] = max(m0, prev);
-            v[1] = max(m1, v[0]);
-            v[2] = max(m2, v[1]);
-            v[3] = max(m3, v[2]);
-            carry = __shfl_sync(0xffffffffu, v[3], 31);
-            const uint32_t w = st[j];
-            // byte q of this word is entry 4 * (32 j + lane) + q - ob: inside the run iff lo <= q < hi
-            const int32_t lo = (int32_t)ob - (int32_t)(4u * (32u * j + lane));
-            const int32_t hi = lo + (int32_t)total;
-#pragma unroll
-            for (int32_t q = 0; q < 4; ++q) {
-                if (q >= lo && q < hi) {
-                    const uint32_t pos = (w >> (8 * q)) & 0xffu;
-                    if (v[q] != 0 && pos < N_OUT) {
-                        const uint32_t bit = v[q] - 1u + pos;
-                        atomicXor(region + (bit >> 5), 1u << (bit & 31u));
-                    } else {
-                        bad = 1u;
-                    }
-                }
-            }
-        }
-    }
-    __syncwarp();
-    if (bad) flag(A.status, 1u);
+    uint32_t seen;
+    asm volatile("{\n .reg .pred p, q;\n .reg .b32 a, v, s, b;\n"
+                 " setp.lt.u32 q, %3, %4;\n"                    // the entry belongs to the run
+                 " setp.lt.and.u32 p, %2, %5, q;\n"             // ... and its position lies inside the tile
+                 " selp.u32 %0, %2, 0, q;\n"
+                 " add.u32 b, %2, %6;\n"
+                 " shr.u32 a, b, 5;\n shl.b32 a, a, 2;\n add.u32 a, a, %1;\n"
+                 " and.b32 s, b, 31;\n shl.b32 v, 1, s;\n"
+                 " @p red.shared.xor.b32 [a], v;\n}"
+                 : "=r"(seen) : "r"(region_sa), "r"(pos), "r"(t), "r"(total), "r"(tile_bits), "r"(bit0) : "memory");
+    return seen;
 }
 
-// Expands and patches the lane's G slices of one tile (already fetched into `in`, staged d_patch
-// words in `st`) into region[lane * W .. lane * W + W); the patch step then works on the whole
-// tile.  `stage` is the warp's STAGE_WORDS words of shared scratch.  WAIT_BULK: lane 0 first waits for its pending bulk copy out of
-// `region`, just before the region is overwritten.  Ends with the warp synchronised.
-template <int N_OUT, int N_IN, bool WAIT_BULK = false>
-SQNN_DEV void tile_decode(const DecodeArgs &A, const PlanePtrs &P, const TileIn<N_OUT, N_IN> &in,
-                          const uint32_t (&st)[4], uint32_t *region, const uint32_t *tab, uint32_t *stage,
-                          uint32_t lane)
+// Flips the patched positions of one format tile (Section 3.2) whose first bit is bit `bit0` of
+// the region.  Every lane's words of the tile must be in place (warp barrier before), and the
+// region is complete after the warp barrier that follows.  `pw`: words fetched by fetch_patches.
+SQNN_DEV void tile_patch(const DecodeArgs &A, const PlanePtrs &P, const TileRun &run, const uint32_t (&pw)[PATCH_AHEAD],
+                         uint32_t *region, uint32_t bit0, uint32_t tile_bits, uint32_t lane)
+{
+    if (run.end == run.base) return;                             // the same in every lane
+    const uint32_t region_sa = smem_addr(region);
+    const uint32_t total = run.end - run.base;
+    const uint32_t w0 = run.base >> 1, wend = (run.end + 1) >> 1;
+    // index, relative to the run, of the low entry of this lane's first word: -1 when the run starts
+    // in the high half of its first word (the unsigned compare in flip_entry then rejects it)
+    const uint32_t t0 = 2 * (w0 + lane) - run.base;
+    uint32_t top = 0;                                            // largest position seen
+#pragma unroll
+    for (uint32_t k = 0; k < PATCH_AHEAD; ++k) {
+        top = max(top, flip_entry(region_sa, bit0, tile_bits, pw[k] & 0xffffu, t0 + 64 * k, total));
+        top = max(top, flip_entry(region_sa, bit0, tile_bits, pw[k] >> 16, t0 + 64 * k + 1, total));
+    }
+    // longer runs: eight words (sixteen entries) per lane and round; the words of the next round are
+    // requested before this round's are used
+    constexpr uint32_t RB = 8;
+    const uint32_t *pp32 = reinterpret_cast<const uint32_t *>(P.pp);
+    uint32_t a0 = w0 + 32 * PATCH_AHEAD;
+    if (a0 < wend) {
+        uint32_t cur[RB], nxt[RB];
+        auto request = [&](uint32_t at, uint32_t (&w)[RB]) {
+#pragma unroll
+            for (uint32_t k = 0; k < RB; ++k) {
+                const uint32_t aw = at + lane + 32 * k;
+                w[k] = aw < wend ? __ldg(pp32 + aw) : 0u;
+            }
+        };
+        request(a0, cur);
+        for (; a0 < wend; a0 += 32 * RB) {
+            request(a0 + 32 * RB, nxt);
+            const uint32_t t = 2 * (a0 + lane) - run.base;
+#pragma unroll
+            for (uint32_t k = 0; k < RB; ++k) {
+                top = max(top, flip_entry(region_sa, bit0, tile_bits, cur[k] & 0xffffu, t + 64 * k, total));
+                top = max(top, flip_entry(region_sa, bit0, tile_bits, cur[k] >> 16, t + 64 * k + 1, total));
+            }
+#pragma unroll
+            for (uint32_t k = 0; k < RB; ++k) cur[k] = nxt[k];
+        }
+    }
+    if (top >= tile_bits) flag(A.status, 1u);
+}
+
+// Expands the lane's 8 slices of one tile into region[lane * W .. lane * W + W).  WAIT_BULK: lane 0
+// first waits for its pending bulk copy out of `region`, just before the region is overwritten.
+// REP: `tab` holds the replicated tables.
+template <int N_OUT, int N_IN, bool WAIT_BULK = false, bool REP = false>
+SQNN_DEV void tile_expand(const TileSeeds<N_OUT, N_IN> &in, uint32_t *region, const uint32_t *tab, uint32_t lane)
 {
     using S = Shape<N_OUT, N_IN>;
     constexpr uint32_t G = S::G, W = S::W, NW = S::NW, NWP = S::NWP, NCH = S::NCH, CB = S::CB;
@@ -477,10 +319,15 @@ SQNN_DEV void tile_decode(const DecodeArgs &A, const PlanePtrs &P, const TileIn<
     uint32_t *mine = region + lane * W;
 
     // seeds -> table entries
-    const uint32_t sh0 = (lane * S::SPAN) & 31u;
     uint32_t al[NSW];
+    if constexpr (S::ALIGNED) {
 #pragma unroll
-    for (uint32_t k = 0; k < NSW; ++k) al[k] = __funnelshift_r(in.raw[k], in.raw[k + 1], sh0);
+        for (uint32_t k = 0; k < NSW; ++k) al[k] = in.raw[k];
+    } else {
+        const uint32_t sh0 = (lane * S::SPAN) & 31u;
+#pragma unroll
+        for (uint32_t k = 0; k < NSW; ++k) al[k] = __funnelshift_r(in.raw[k], in.raw[k + 1], sh0);
+    }
     uint32_t x[G][NWP];
 #pragma unroll
     for (uint32_t i = 0; i < G; ++i) {
@@ -489,20 +336,17 @@ SQNN_DEV void tile_decode(const DecodeArgs &A, const PlanePtrs &P, const TileIn<
         uint32_t seed;
         if (s + n_in <= 32) seed = (al[w] >> s) & smask;
         else seed = __funnelshift_r(al[w], al[w + 1 < NSW ? w + 1 : w], s) & smask;
-        load_entry<NWP>(tab, seed & ((1u << CB) - 1u), x[i]);
+        load_entry<NWP, REP>(tab, seed & ((1u << CB) - 1u), lane, x[i]);
 #pragma unroll
         for (uint32_t ch = 1; ch < NCH; ++ch) {
             uint32_t y[NWP];
-            load_entry<NWP>(tab, (ch << CB) | ((seed >> (ch * CB)) & ((1u << CB) - 1u)), y);
+            load_entry<NWP, REP>(tab, (ch << CB) | ((seed >> (ch * CB)) & ((1u << CB) - 1u)), lane, y);
 #pragma unroll
             for (uint32_t k = 0; k < NW; ++k) x[i][k] ^= y[k];
         }
     }
-    if constexpr (WAIT_BULK) {                       // the bulk copy of the previous tile still reads `region`
-        if (lane == 0) bulk_wait_read<0>();
-        __syncwarp();
-    }
     // output word k = bits [32k, 32k + 32) of the concatenated entries (entry bits >= n_out are 0)
+    uint32_t out[W];
 #pragma unroll
     for (uint32_t k = 0; k < W; ++k) {
         const uint32_t i0 = (32 * k) / n_out, o = 32 * k - i0 * n_out;
@@ -514,45 +358,35 @@ SQNN_DEV void tile_decode(const DecodeArgs &A, const PlanePtrs &P, const TileIn<
         for (uint32_t i = i0 + 1; i < G; ++i) {
             if (filled < 32) { word |= x[i][0] << filled; filled += n_out; }
         }
-        mine[k] = word;
+        out[k] = word;
     }
-
-    // patches (warp-uniform branch: `total` is the same in every lane)
-    if (in.total != 0) {
-        __syncwarp();                                   // every lane's words are in place
-        const uint32_t nb = lane * G * P.w_np, sh = nb & 31u;
-        // the words fetched ahead hold at most PATCH_WIN entries (then alignment bytes + entries <= 511)
-        const bool one_window = in.total <= PATCH_WIN;                   // the same in every lane
-        if (G * P.w_np <= 32) {
-            const uint32_t win = __funnelshift_r(in.np0, in.np1, sh) &
-                                 (G * P.w_np == 32 ? 0xffffffffu : (1u << (G * P.w_np)) - 1u);
-            if (one_window) patch_tile_fast<G, n_out, uint32_t>(A, P, region, stage, st, in.base, in.total, win, lane);
-            else patch_tile<G, n_out, uint32_t>(A, P, region, stage, st, in.base, in.total, win, lane);
-        } else {
-            uint64_t win = (uint64_t)__funnelshift_r(in.np0, in.np1, sh) |
-                           ((uint64_t)__funnelshift_r(in.np1, in.np2, sh) << 32);
-            if (G * P.w_np < 64) win &= (1ull << (G * P.w_np)) - 1ull;
-            if (one_window) patch_tile_fast<G, n_out, uint64_t>(A, P, region, stage, st, in.base, in.total, win, lane);
-            else patch_tile<G, n_out, uint64_t>(A, P, region, stage, st, in.base, in.total, win, lane);
-        }
+    if constexpr (WAIT_BULK) {                       // the bulk copy of the previous tile still reads `region`
+        if (lane == 0) bulk_wait_read<0>();
+        __syncwarp();
     }
-    __syncwarp();
+    // the widest stores the lane's base allows (lane stride W words): conflict-free for every W
+    if constexpr (W % 4 == 0) {
+#pragma unroll
+        for (uint32_t k = 0; k < W; k += 4)
+            *reinterpret_cast<uint4 *>(mine + k) = make_uint4(out[k], out[k + 1], out[k + 2], out[k + 3]);
+    } else if constexpr (W % 2 == 0) {
+#pragma unroll
+        for (uint32_t k = 0; k < W; k += 2) *reinterpret_cast<uint2 *>(mine + k) = make_uint2(out[k], out[k + 1]);
+    } else {
+#pragma unroll
+        for (uint32_t k = 0; k < W; ++k) mine[k] = out[k];
+    }
 }
 
-// Fetch + decode of one tile without overlap (for the kernels that do more work per tile).
-template <int N_OUT, int N_IN>
-SQNN_DEV void decode_warp_tile(const DecodeArgs &A, uint32_t plane, uint64_t tile,
-                               uint32_t *region, const uint32_t *tab, uint32_t *stage, uint32_t lane);
-
-// Run-time shape: plain loops, every read through extract_bits.
-SQNN_DEV void decode_warp_tile_generic(const DecodeArgs &A, uint32_t plane, uint64_t tile,
-                                       uint32_t *region, const uint32_t *tab, uint32_t lane)
+// Run-time shape: plain loops, every read through extract_bits.  Ends with the warp synchronised.
+SQNN_DEV void decode_ktile_generic(const DecodeArgs &A, uint32_t plane, uint64_t ktile,
+                                   uint32_t *region, const uint32_t *tab, uint32_t lane)
 {
     const PlanePtrs &P = A.pl[plane];
     const uint32_t n_out = A.n_out, n_in = A.n_in, G = A.G, W = A.W;
     const uint32_t nw = A.nw, nwp = A.nwp, nch = A.nchunks, cb = A.cb;
     const uint32_t cmask = (1u << cb) - 1u;
-    const uint64_t s0 = (tile * 32 + lane) * G;
+    const uint64_t s0 = (ktile * 32 + lane) * G;
     uint32_t *mine = region + lane * W;
     uint64_t acc = 0;
     uint32_t have = 0, wp = 0;
@@ -568,47 +402,44 @@ SQNN_DEV void decode_warp_tile_generic(const DecodeArgs &A, uint32_t plane, uint
             if (have >= 32) { mine[wp++] = (uint32_t)acc; acc >>= 32; have -= 32; }
         }
     }
-    // Patches (Section 3.2): the lane's first entry sits at the block offset of the tile plus
-    // the n_patch counts of the lanes before it.
-    if (P.w_np != 0) {
-        uint32_t cnt = 0;
-        for (uint32_t i = 0; i < G; ++i) cnt += extract_bits(P.np, (s0 + i) * P.w_np, P.w_np);
-        uint32_t incl = cnt;
-#pragma unroll
-        for (uint32_t d = 1; d < 32; d <<= 1) {
-            const uint32_t o = __shfl_up_sync(0xffffffffu, incl, d);
-            if (lane >= d) incl += o;
-        }
-        if (cnt != 0) {
-            uint32_t at = __ldg(P.idx + tile * (G / 4)) + incl - cnt;
-            for (uint32_t i = 0; i < G; ++i) {
-                const uint32_t npi = extract_bits(P.np, (s0 + i) * P.w_np, P.w_np);
-                for (uint32_t k = 0; k < npi; ++k, ++at) {
-                    if (at >= P.n_dp) { flag(A.status, 2u); continue; }
-                    const uint32_t pos = P.dp[at];
-                    if (pos >= n_out) { flag(A.status, 1u); continue; }
-                    const uint32_t bit = i * n_out + pos;
-                    mine[bit >> 5] ^= 1u << (bit & 31);
-                }
-            }
+    __syncwarp();
+    // patches (Section 3.2), one format tile after the other
+    const uint32_t tile_bits = SQNN_TILE_SLICES * n_out;
+    const uint32_t region_sa = smem_addr(region);
+    uint32_t bad = 0;
+    for (uint32_t f = 0; f < A.KT; ++f) {
+        const uint64_t ft = ktile * A.KT + f;
+        uint32_t base = __ldg(P.idx + ft), end = __ldg(P.idx + ft + 1);
+        if (end < base || end > P.n_pp) { flag(A.status, 2u); continue; }
+        for (uint32_t e = base + lane; e < end; e += 32) {
+            const uint32_t pos = P.pp[e];
+            if (pos < tile_bits) smem_flip(region_sa, f * tile_bits + pos); else bad = 1;
         }
     }
+    if (bad) flag(A.status, 1u);
     __syncwarp();
 }
 
+// Fetch + expand + patch of one kernel tile without overlap (for the kernels that do more work per
+// tile).  `tab`: the tables in shared memory.  Ends with the warp synchronised.
 template <int N_OUT, int N_IN>
 SQNN_DEV void decode_warp_tile(const DecodeArgs &A, uint32_t plane, uint64_t tile,
-                               uint32_t *region, const uint32_t *tab, uint32_t *stage, uint32_t lane)
+                               uint32_t *region, const uint32_t *tab, uint32_t lane)
 {
     if constexpr (N_OUT != 0) {
+        using S = Shape<N_OUT, N_IN>;
         const PlanePtrs &P = A.pl[plane];
-        TileIn<N_OUT, N_IN> in;
-        uint32_t st[4];
-        tile_fetch<N_OUT, N_IN>(P, tile, lane, in);
-        stage_fetch<N_OUT, N_IN>(A, P, in, lane, st);
-        tile_decode<N_OUT, N_IN>(A, P, in, st, region, tab, stage, lane);
+        TileSeeds<N_OUT, N_IN> in;
+        uint32_t pw[PATCH_AHEAD];
+        fetch_seeds<N_OUT, N_IN>(P, tile, lane, in);
+        TileRun run = fetch_run(P, tile);
+        fetch_patches(A, P, run, lane, pw);
+        tile_expand<N_OUT, N_IN>(in, region, tab, lane);
+        __syncwarp();
+        tile_patch(A, P, run, pw, region, 0u, S::TILE_BITS, lane);
+        __syncwarp();
     } else {
-        decode_warp_tile_generic(A, plane, tile, region, tab, lane);
+        decode_ktile_generic(A, plane, tile, region, tab, lane);
     }
 }
 

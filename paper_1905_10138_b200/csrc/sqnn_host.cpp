@@ -2,6 +2,7 @@
 // packed blob format, its validation and size accounting.  No CUDA in this file.
 #include "sqnn.h"
 #include "sqnn_blob.h"
+#include "sqnn_layout.h"
 
 #include <algorithm>
 #include <cstdlib>
@@ -156,6 +157,56 @@ inline uint32_t read_field(const uint32_t *src, uint64_t index, uint32_t width)
     return (uint32_t)((v >> sh) & (((uint64_t)1 << width) - 1));
 }
 
+// The lookup tables of the network in the layout the kernels index (sqnn_layout.h).
+void build_tables(const uint32_t *rows, uint32_t n_out, uint32_t n_in, uint32_t *tab)
+{
+    const uint32_t nwp = sqnn::entry_words_padded(n_out);
+    const uint32_t nch = sqnn::table_chunks(n_in, nwp), cb = sqnn::chunk_bits(n_in, nwp);
+    std::memset(tab, 0, (size_t)sqnn::table_words(n_out, n_in) * 4);
+    for (uint32_t ch = 0; ch < nch; ++ch)
+        for (uint32_t v = 0; v < (1u << cb); ++v) {
+            // chunk bits that lie past n_in select no column
+            const uint64_t sel64 = (uint64_t)v << (ch * cb);
+            const uint32_t sel = (uint32_t)(sel64 & (n_in >= 32 ? 0xffffffffull : ((1ull << n_in) - 1ull)));
+            uint32_t *e = tab + (size_t)(((ch << cb) | v)) * nwp;
+            for (uint32_t j = 0; j < n_out; ++j)
+                e[j >> 5] |= (uint32_t)(__builtin_popcount(rows[j] & sel) & 1) << (j & 31);
+        }
+}
+
+struct BlobPlan {
+    sqnn_desc d;
+};
+
+// Section offsets of a device blob for the given patch totals.
+void plan_blob(uint64_t m, uint64_t n, uint32_t n_q, uint32_t n_out, uint32_t n_in, const uint64_t *n_pp, sqnn_desc *out)
+{
+    sqnn_desc d;
+    std::memset(&d, 0, sizeof d);
+    const uint64_t mn = m * n;
+    const uint64_t l = (mn + n_out - 1) / n_out;
+    const uint64_t lp = round_up(l, SQNN_PAD_SLICES);
+    d.m = m; d.n = n; d.slices = l; d.slices_padded = lp;
+    d.n_q = n_q; d.n_out = n_out; d.n_in = n_in; d.tile_slices = SQNN_TILE_SLICES;
+    d.tab_entry_words = sqnn::entry_words_padded(n_out);
+    d.tab_chunks = sqnn::table_chunks(n_in, d.tab_entry_words);
+    d.tab_chunk_bits = sqnn::chunk_bits(n_in, d.tab_entry_words);
+    uint64_t off = SQNN_BLOB_HEADER_BYTES;
+    d.off_xornet = off;
+    off += round_up((uint64_t)n_out * 4, 16) + 16;
+    d.off_tables = off;
+    d.tables_bytes = (uint64_t)sqnn::table_words(n_out, n_in) * 4;
+    off += round_up(d.tables_bytes, 16) + 16;
+    for (uint32_t i = 0; i < n_q; ++i) {
+        d.n_pp[i] = n_pp[i];
+        d.off_wc[i] = off;  off += round_up(lp * n_in / 8, 16) + 16;
+        d.off_idx[i] = off; off += round_up((lp / SQNN_TILE_SLICES + 1) * 4, 16) + 16;
+        d.off_pp[i] = off;  off += round_up(n_pp[i] * 2, 16) + 16;
+    }
+    d.total_bytes = off;
+    *out = d;
+}
+
 int build_blob(const sqnn_xornet *net, uint64_t m, uint64_t n, uint32_t n_q,
                const uint32_t *const *wc, const uint16_t *const *np, const uint8_t *const *dp8,
                const uint16_t *const *dp16, void **blob, size_t *blob_bytes)
@@ -163,34 +214,20 @@ int build_blob(const sqnn_xornet *net, uint64_t m, uint64_t n, uint32_t n_q,
     const uint64_t mn = m * n;
     const uint32_t n_out = net->n_out, n_in = net->n_in;
     const uint64_t l = (mn + n_out - 1) / n_out;
-    const uint64_t lp = round_up(l, SQNN_PAD_SLICES);
-    sqnn_desc d;
-    std::memset(&d, 0, sizeof d);
-    d.m = m; d.n = n; d.slices = l; d.slices_padded = lp;
-    d.n_q = n_q; d.n_out = n_out; d.n_in = n_in; d.block_slices = SQNN_BLOCK_SLICES;
-    d.w_dp = 8;
-    uint64_t off = SQNN_BLOB_HEADER_BYTES;
-    d.off_xornet = off;
-    off += round_up((uint64_t)n_out * 4, 16) + 16;
-    std::vector<uint64_t> ndp(n_q, 0);
+    uint64_t n_pp[SQNN_MAX_PLANES] = {0};
     for (uint32_t i = 0; i < n_q; ++i) {
-        uint32_t maxp = 0;
         uint64_t sum = 0;
         for (uint64_t s = 0; s < l; ++s) {
             if (np[i][s] > n_out) return SQNN_E_INVALID_ARG;
-            maxp = std::max<uint32_t>(maxp, np[i][s]);
             sum += np[i][s];
         }
-        ndp[i] = sum;
-        d.n_dp[i] = sum;
-        d.w_np[i] = ceil_lg_u64((uint64_t)maxp + 1);
-        d.off_wc[i] = off;  off += round_up(lp * n_in / 8, 16) + 16;
-        d.off_np[i] = off;  if (d.w_np[i]) off += round_up(lp * d.w_np[i] / 8, 16) + 16;
-        d.off_idx[i] = off; off += round_up((lp / SQNN_BLOCK_SLICES + 1) * 4, 16) + 16;
-        d.off_dp[i] = off;  off += round_up(sum, 16) + 16;
+        if (sum > 0xffffffffull) return SQNN_E_INVALID_ARG;
+        n_pp[i] = sum;
     }
-    d.total_bytes = off;
-    uint8_t *b = (uint8_t *)std::calloc(off, 1);
+    sqnn_desc d;
+    plan_blob(m, n, n_q, n_out, n_in, n_pp, &d);
+    const uint64_t lp = d.slices_padded;
+    uint8_t *b = (uint8_t *)std::calloc(d.total_bytes, 1);
     if (!b) return SQNN_E_NOMEM;
     sqnn_blob_header *h = (sqnn_blob_header *)b;
     std::memcpy(h->magic, SQNN_BLOB_MAGIC, 8);
@@ -198,32 +235,35 @@ int build_blob(const sqnn_xornet *net, uint64_t m, uint64_t n, uint32_t n_q,
     h->header_bytes = SQNN_BLOB_HEADER_BYTES;
     h->desc = d;
     std::memcpy(b + d.off_xornet, net->rows, (size_t)n_out * 4);
-    const uint32_t seed_limit_bits = n_in;
+    build_tables(net->rows, n_out, n_in, (uint32_t *)(b + d.off_tables));
     for (uint32_t i = 0; i < n_q; ++i) {
-        if (seed_limit_bits < 32)
+        if (n_in < 32)
             for (uint64_t s = 0; s < l; ++s)
-                if (wc[i][s] >> seed_limit_bits) { std::free(b); return SQNN_E_INVALID_ARG; }
+                if (wc[i][s] >> n_in) { std::free(b); return SQNN_E_INVALID_ARG; }
         pack_fields(wc[i], l, n_in, (uint32_t *)(b + d.off_wc[i]));
-        pack_fields(np[i], l, d.w_np[i], (uint32_t *)(b + d.off_np[i]));
         uint32_t *idx = (uint32_t *)(b + d.off_idx[i]);
-        uint8_t *dst = b + d.off_dp[i];
+        uint16_t *dst = (uint16_t *)(b + d.off_pp[i]);
         uint64_t run = 0;
-        const uint64_t blocks = lp / SQNN_BLOCK_SLICES;
-        for (uint64_t blk = 0; blk <= blocks; ++blk) {
-            idx[blk] = (uint32_t)run;
-            if (blk == blocks) break;
-            const uint64_t lo = blk * SQNN_BLOCK_SLICES, hi = std::min<uint64_t>(l, lo + SQNN_BLOCK_SLICES);
-            for (uint64_t s = lo; s < hi; ++s) run += np[i][s];
+        const uint64_t tiles = lp / SQNN_TILE_SLICES;
+        for (uint64_t t = 0; t <= tiles; ++t) {
+            idx[t] = (uint32_t)run;
+            if (t == tiles) break;
+            const uint64_t lo = t * SQNN_TILE_SLICES, hi = std::min<uint64_t>(l, lo + SQNN_TILE_SLICES);
+            for (uint64_t s = lo; s < hi; ++s) {
+                int64_t prev = -1;
+                for (uint32_t k = 0; k < np[i][s]; ++k, ++run) {
+                    const uint32_t pos = dp8 ? dp8[i][run] : dp16[i][run];
+                    // positions inside a slice ascend strictly; the last slice holds real positions only
+                    if (pos >= n_out || (int64_t)pos <= prev || s * n_out + pos >= mn) { std::free(b); return SQNN_E_INVALID_ARG; }
+                    prev = pos;
+                    dst[run] = (uint16_t)((s - lo) * n_out + pos);
+                }
+            }
         }
-        if (run != ndp[i] || ndp[i] > 0xffffffffull) { std::free(b); return SQNN_E_INVALID_ARG; }
-        for (uint64_t k = 0; k < ndp[i]; ++k) {
-            const uint32_t pos = dp8 ? dp8[i][k] : dp16[i][k];
-            if (pos >= n_out) { std::free(b); return SQNN_E_INVALID_ARG; }
-            dst[k] = (uint8_t)pos;
-        }
+        if (run != n_pp[i]) { std::free(b); return SQNN_E_INVALID_ARG; }
     }
     *blob = b;
-    *blob_bytes = off;
+    *blob_bytes = d.total_bytes;
     return SQNN_OK;
 }
 
@@ -272,7 +312,7 @@ static int encode_impl(const sqnn_xornet *net, const sqnn_planes *layer, bool ex
             const uint64_t *plane = layer->planes + (uint64_t)i * words;
             pa[i].wc.assign(l, 0);
             pa[i].np.assign(l, 0);
-            bool bad_seed = false;
+            int bad_seed = 0;
             // pass 1: seed and patch count of every slice (slices are independent)
 #pragma omp parallel for schedule(dynamic, 4096)
             for (int64_t s = 0; s < (int64_t)l; ++s) {
@@ -281,7 +321,11 @@ static int encode_impl(const sqnn_xornet *net, const sqnn_planes *layer, bool ex
                 uint32_t seed;
                 if (given) {
                     seed = given[i][s];
-                    if (n_in < 32 && (seed >> n_in)) { bad_seed = true; seed = 0; }
+                    if (n_in < 32 && (seed >> n_in)) {
+#pragma omp atomic write
+                        bad_seed = 1;
+                        seed = 0;
+                    }
                 } else {
                     seed = exhaustive ? encode_exhaustive(tab, n_in, sb) : encode_alg1(net->rows, n_out, sb);
                 }
@@ -382,60 +426,60 @@ int sqnn_describe_host(const void *blob, size_t blob_bytes, sqnn_desc *desc)
         return SQNN_E_BAD_BLOB;
     const sqnn_desc &d = h.desc;
     if (d.n_out < 1 || d.n_out > SQNN_MAX_N_OUT || d.n_in < 1 || d.n_in > SQNN_MAX_N_IN ||
-        d.n_q < 1 || d.n_q > SQNN_MAX_PLANES || d.block_slices != SQNN_BLOCK_SLICES || d.w_dp != 8)
+        d.n_q < 1 || d.n_q > SQNN_MAX_PLANES || d.tile_slices != SQNN_TILE_SLICES)
         return SQNN_E_BAD_BLOB;
     if (d.m == 0 || d.n == 0 || d.m > ((uint64_t)1 << 40) / d.n) return SQNN_E_BAD_BLOB;
-    const uint64_t mn = d.m * d.n;
-    const uint64_t l = (mn + d.n_out - 1) / d.n_out;
-    if (d.slices != l || d.slices_padded != round_up(l, SQNN_PAD_SLICES)) return SQNN_E_BAD_BLOB;
-    if (d.total_bytes != blob_bytes) return SQNN_E_BAD_BLOB;
-    const uint64_t lp = d.slices_padded;
-    auto section_ok = [&](uint64_t off, uint64_t payload) {
-        return (off % 16 == 0) && off >= SQNN_BLOB_HEADER_BYTES && payload <= blob_bytes &&
-               off <= blob_bytes - payload && blob_bytes - off - payload >= 16;
-    };
-    if (!section_ok(d.off_xornet, (uint64_t)d.n_out * 4)) return SQNN_E_BAD_BLOB;
+    for (uint32_t i = 0; i < d.n_q; ++i)
+        if (d.n_pp[i] > 0xffffffffull) return SQNN_E_BAD_BLOB;
+    // every offset and size is a fixed function of the shape and the patch totals
+    sqnn_desc want;
+    plan_blob(d.m, d.n, d.n_q, d.n_out, d.n_in, d.n_pp, &want);
+    if (std::memcmp(&want, &d, sizeof d) != 0 || d.total_bytes != blob_bytes) return SQNN_E_BAD_BLOB;
+    const uint64_t mn = d.m * d.n, l = d.slices, lp = d.slices_padded;
     const uint32_t *rows = (const uint32_t *)(b + d.off_xornet);
     if (d.n_in < 32)
         for (uint32_t j = 0; j < d.n_out; ++j)
             if (rows[j] >> d.n_in) return SQNN_E_BAD_BLOB;
-    uint64_t prev_end = d.off_xornet + (uint64_t)d.n_out * 4;
+    try {
+        std::vector<uint32_t> tab(sqnn::table_words(d.n_out, d.n_in));
+        build_tables(rows, d.n_out, d.n_in, tab.data());
+        if (std::memcmp(tab.data(), b + d.off_tables, (size_t)d.tables_bytes) != 0) return SQNN_E_BAD_BLOB;
+    } catch (const std::bad_alloc &) {
+        return SQNN_E_NOMEM;
+    }
+    const uint64_t tiles = lp / SQNN_TILE_SLICES;
+    const uint64_t tile_bits = (uint64_t)SQNN_TILE_SLICES * d.n_out;
     for (uint32_t i = 0; i < d.n_q; ++i) {
-        if (d.w_np[i] > 9 || d.n_dp[i] > 0xffffffffull) return SQNN_E_BAD_BLOB;
-        const uint64_t wc_bytes = lp * d.n_in / 8, np_bytes = lp * d.w_np[i] / 8;
-        const uint64_t idx_bytes = (lp / SQNN_BLOCK_SLICES + 1) * 4;
-        if (!section_ok(d.off_wc[i], wc_bytes) || d.off_wc[i] < prev_end) return SQNN_E_BAD_BLOB;
-        prev_end = d.off_wc[i] + wc_bytes;
-        if (d.w_np[i]) {
-            if (!section_ok(d.off_np[i], np_bytes) || d.off_np[i] < prev_end) return SQNN_E_BAD_BLOB;
-            prev_end = d.off_np[i] + np_bytes;
-        }
-        if (!section_ok(d.off_idx[i], idx_bytes) || d.off_idx[i] < prev_end) return SQNN_E_BAD_BLOB;
-        prev_end = d.off_idx[i] + idx_bytes;
-        if (!section_ok(d.off_dp[i], d.n_dp[i]) || d.off_dp[i] < prev_end) return SQNN_E_BAD_BLOB;
-        prev_end = d.off_dp[i] + d.n_dp[i];
         const uint32_t *wcs = (const uint32_t *)(b + d.off_wc[i]);
-        const uint32_t *nps = (const uint32_t *)(b + d.off_np[i]);
         const uint32_t *idx = (const uint32_t *)(b + d.off_idx[i]);
-        const uint8_t *dp = b + d.off_dp[i];
-        uint64_t run = 0;
-        const uint64_t blocks = lp / SQNN_BLOCK_SLICES;
-        for (uint64_t blk = 0; blk < blocks; ++blk) {
-            if (idx[blk] != run) return SQNN_E_BAD_BLOB;
-            for (uint64_t s = blk * SQNN_BLOCK_SLICES; s < (blk + 1) * SQNN_BLOCK_SLICES; ++s) {
-                const uint32_t p = read_field(nps, s, d.w_np[i]);
-                if (s >= l && (p != 0 || read_field(wcs, s, d.n_in) != 0)) return SQNN_E_BAD_BLOB;
-                if (p > d.n_out) return SQNN_E_BAD_BLOB;
-                run += p;
+        const uint16_t *pp = (const uint16_t *)(b + d.off_pp[i]);
+        for (uint64_t s = l; s < lp; ++s)
+            if (read_field(wcs, s, d.n_in) != 0) return SQNN_E_BAD_BLOB;
+        if (idx[0] != 0 || idx[tiles] != d.n_pp[i]) return SQNN_E_BAD_BLOB;
+        for (uint64_t t = 0; t < tiles; ++t) {
+            if (idx[t + 1] < idx[t] || idx[t + 1] > d.n_pp[i]) return SQNN_E_BAD_BLOB;
+            int64_t prev = -1;
+            for (uint64_t k = idx[t]; k < idx[t + 1]; ++k) {
+                const uint64_t pos = pp[k];
+                if (pos >= tile_bits || (int64_t)pos <= prev || t * tile_bits + pos >= mn) return SQNN_E_BAD_BLOB;
+                prev = (int64_t)pos;
             }
-            if (run > d.n_dp[i]) return SQNN_E_BAD_BLOB;
         }
-        if (idx[blocks] != run || run != d.n_dp[i]) return SQNN_E_BAD_BLOB;
-        for (uint64_t k = 0; k < d.n_dp[i]; ++k)
-            if (dp[k] >= d.n_out) return SQNN_E_BAD_BLOB;
     }
     *desc = d;
     return SQNN_OK;
+}
+
+// n_patch of every slice of one plane, from the patch positions of a validated blob.
+static void count_patches(const uint8_t *b, const sqnn_desc &d, uint32_t plane, uint16_t *np)
+{
+    const uint32_t *idx = (const uint32_t *)(b + d.off_idx[plane]);
+    const uint16_t *pp = (const uint16_t *)(b + d.off_pp[plane]);
+    std::memset(np, 0, sizeof(uint16_t) * (size_t)d.slices);
+    const uint64_t tiles = d.slices_padded / SQNN_TILE_SLICES;
+    for (uint64_t t = 0; t < tiles; ++t)
+        for (uint64_t k = idx[t]; k < idx[t + 1]; ++k)
+            ++np[t * SQNN_TILE_SLICES + pp[k] / d.n_out];
 }
 
 int sqnn_unpack_host(const void *blob, size_t blob_bytes, uint32_t plane,
@@ -450,16 +494,15 @@ int sqnn_unpack_host(const void *blob, size_t blob_bytes, uint32_t plane,
     const uint64_t l = d.slices;
     uint32_t *w = (uint32_t *)std::malloc(sizeof(uint32_t) * (l ? l : 1));
     uint16_t *p = (uint16_t *)std::malloc(sizeof(uint16_t) * (l ? l : 1));
-    uint16_t *q = (uint16_t *)std::malloc(sizeof(uint16_t) * (d.n_dp[plane] ? d.n_dp[plane] : 1));
+    uint16_t *q = (uint16_t *)std::malloc(sizeof(uint16_t) * (d.n_pp[plane] ? d.n_pp[plane] : 1));
     if (!w || !p || !q) { std::free(w); std::free(p); std::free(q); return SQNN_E_NOMEM; }
     const uint32_t *wcs = (const uint32_t *)(b + d.off_wc[plane]);
-    const uint32_t *nps = (const uint32_t *)(b + d.off_np[plane]);
-    for (uint64_t s = 0; s < l; ++s) {
-        w[s] = read_field(wcs, s, d.n_in);
-        p[s] = (uint16_t)read_field(nps, s, d.w_np[plane]);
-    }
-    for (uint64_t k = 0; k < d.n_dp[plane]; ++k) q[k] = b[d.off_dp[plane] + k];
-    *wc = w; *np = p; *dp = q; *n_dp = d.n_dp[plane];
+    for (uint64_t s = 0; s < l; ++s) w[s] = read_field(wcs, s, d.n_in);
+    count_patches(b, d, plane, p);
+    // positions ascend inside a tile, so they already stand in slice order, ascending inside a slice
+    const uint16_t *pp = (const uint16_t *)(b + d.off_pp[plane]);
+    for (uint64_t k = 0; k < d.n_pp[plane]; ++k) q[k] = (uint16_t)(pp[k] % d.n_out);
+    *wc = w; *np = p; *dp = q; *n_dp = d.n_pp[plane];
     return SQNN_OK;
 }
 
@@ -474,25 +517,32 @@ int sqnn_stats_host(const void *blob, size_t blob_bytes, sqnn_stats *stats)
     const uint64_t mn = d.m * d.n, l = d.slices, lp = d.slices_padded;
     stats->slices = l;
     double eq1_bits = 0.0;
-    for (uint32_t i = 0; i < d.n_q; ++i) {
-        const uint32_t *nps = (const uint32_t *)(b + d.off_np[i]);
-        uint32_t maxp = 0;
-        uint64_t sum = 0;
-        for (uint64_t s = 0; s < l; ++s) {
-            const uint32_t p = read_field(nps, s, d.w_np[i]);
-            maxp = std::max(maxp, p);
-            sum += p;
+    try {
+        std::vector<uint16_t> np(l ? l : 1);
+        for (uint32_t i = 0; i < d.n_q; ++i) {
+            count_patches(b, d, i, np.data());
+            uint32_t maxp = 0;
+            uint64_t sum = 0;
+            for (uint64_t s = 0; s < l; ++s) {
+                const uint32_t p = np[s];
+                maxp = std::max(maxp, p);
+                sum += p;
+                ++stats->patch_hist[p < SQNN_PATCH_HIST_BINS - 1 ? p : SQNN_PATCH_HIST_BINS - 1];
+            }
+            stats->patches[i] = sum;
+            stats->max_patch[i] = maxp;
+            // Eq. 1, literally: n_in/n_out * mn + l * ceil(lg max p) + sum p * ceil(lg n_out)
+            eq1_bits += (double)d.n_in / (double)d.n_out * (double)mn +
+                        (double)l * ceil_lg_u64(maxp) + (double)sum * ceil_lg_u64(d.n_out);
+            stats->bits_wc += (round_up(lp * d.n_in / 8, 16) + 16) * 8;
+            stats->bits_index += (round_up((lp / SQNN_TILE_SLICES + 1) * 4, 16) + 16) * 8;
+            stats->bits_dpatch += (round_up(sum * 2, 16) + 16) * 8;
         }
-        stats->patches[i] = sum;
-        stats->max_patch[i] = maxp;
-        // Eq. 1, literally: n_in/n_out * mn + l * ceil(lg max p) + sum p * ceil(lg n_out)
-        eq1_bits += (double)d.n_in / (double)d.n_out * (double)mn +
-                    (double)l * ceil_lg_u64(maxp) + (double)sum * ceil_lg_u64(d.n_out);
-        stats->bits_wc += (round_up(lp * d.n_in / 8, 16) + 16) * 8;
-        if (d.w_np[i]) stats->bits_npatch += (round_up(lp * d.w_np[i] / 8, 16) + 16) * 8;
-        stats->bits_index += (round_up((lp / SQNN_BLOCK_SLICES + 1) * 4, 16) + 16) * 8;
-        stats->bits_dpatch += (round_up(sum, 16) + 16) * 8;
+    } catch (const std::bad_alloc &) {
+        return SQNN_E_NOMEM;
     }
+    stats->bits_tables = (round_up(d.tables_bytes, 16) + 16) * 8;
+    stats->bits_index += stats->bits_tables;
     stats->bpw_eq1 = eq1_bits / (double)mn;
     stats->bpw_actual = (double)(stats->bits_wc + stats->bits_npatch + stats->bits_index + stats->bits_dpatch) / (double)mn;
     return SQNN_OK;
@@ -508,15 +558,20 @@ int sqnn_stats_blocked_host(const void *blob, size_t blob_bytes, uint64_t block_
     const uint8_t *b = (const uint8_t *)blob;
     const uint64_t mn = d.m * d.n, l = d.slices;
     uint64_t np_bits = 0, dp_entries = 0;
-    for (uint32_t i = 0; i < d.n_q; ++i) {
-        const uint32_t *nps = (const uint32_t *)(b + d.off_np[i]);
-        for (uint64_t s0 = 0; s0 < l; s0 += block_slices) {
-            const uint64_t s1 = std::min(l, s0 + block_slices);
-            uint32_t maxp = 0;
-            for (uint64_t s = s0; s < s1; ++s) maxp = std::max(maxp, read_field(nps, s, d.w_np[i]));
-            np_bits += (s1 - s0) * ceil_lg_u64(maxp);
+    try {
+        std::vector<uint16_t> np(l ? l : 1);
+        for (uint32_t i = 0; i < d.n_q; ++i) {
+            count_patches(b, d, i, np.data());
+            for (uint64_t s0 = 0; s0 < l; s0 += block_slices) {
+                const uint64_t s1 = std::min(l, s0 + block_slices);
+                uint32_t maxp = 0;
+                for (uint64_t s = s0; s < s1; ++s) maxp = std::max<uint32_t>(maxp, np[s]);
+                np_bits += (s1 - s0) * ceil_lg_u64(maxp);
+            }
+            dp_entries += d.n_pp[i];
         }
-        dp_entries += d.n_dp[i];
+    } catch (const std::bad_alloc &) {
+        return SQNN_E_NOMEM;
     }
     if (bits_npatch) *bits_npatch = np_bits;
     if (bpw_eq1)

@@ -7,7 +7,7 @@
 //   - the decode warps expand the weights of the step into the A stage (bf16, 128-byte rows,
 //     128-byte swizzle) -- the expanded weights exist only in shared memory;
 //   - one thread fetches the matching activations X[bc .. bc+N) x [64 columns] with TMA
-//     (no multicast: every CTA fetches its own tile);
+//     (every CTA fetches its own tile);
 //   - one thread issues tcgen05.mma (K = 16 each) that accumulate in tensor memory.
 // Column ranges of different CTAs are summed with fp32 atomics on Y (cleared beforehand).
 //
@@ -17,11 +17,9 @@
 // expansion is a few instructions per weight.  Otherwise one tile holds the rescaled weights
 // (+-alpha_1) + (+-alpha_2) + ... rounded to bf16, written sparsely from a per-row value table.
 //
-// Where the bits come from.  With a workspace the planes have been decoded to packed bits by the
-// tiled decode kernel; 128 x 512-bit boxes of them (and of the mask) are brought in by TMA when
-// rows start on 16-byte boundaries, by coalesced loads otherwise.  Without a workspace one thread
-// per (row, bit vector) walks the slices that cover its row segment (seed -> XOR tables -> patch
-// flips) itself.
+// Where the bits come from.  The planes have been decoded to packed bits in the workspace by the
+// tiled decode kernel (queued just before this one); 128 x 512-bit boxes of them (and of the mask)
+// are brought in by TMA when rows start on 16-byte boundaries, by coalesced loads otherwise.
 //
 // Every wait on an mbarrier is bounded; a wait that gives up sets SQNN_E_TIMEOUT in the status
 // word and makes all roles leave their loops, so the kernel always returns.
@@ -53,7 +51,7 @@ constexpr uint32_t MAX_STAGES = 4;
 constexpr uint64_t WAIT_LIMIT_CYCLES = 4000000000ull;   // about 2 s at 2 GHz
 
 struct MmaArgs {
-    DecodeArgs A;                 // with small tables (<= 4 KB)
+    DecodeArgs A;
     const uint32_t *mask32;
     uint64_t mask_words32;        // number of valid 32-bit mask words
     const float *alpha;
@@ -67,7 +65,7 @@ struct MmaArgs {
     uint32_t splits;              // CTAs per row tile
     uint32_t macros_per_split;
     uint32_t b_stage_bytes;
-    const uint32_t *bits32;       // decoded planes in the workspace (NULL: decode in this kernel)
+    const uint32_t *bits32;       // decoded planes in the workspace
     uint64_t plane_words32;       // 32-bit words per plane in the workspace
     uint32_t per_plane;           // 1: one sign tile and one accumulator per plane, scales in the epilogue
     uint32_t tma_bits;            // 1: the bit buffer is filled by TMA (rows of the packed planes 16-byte aligned)
@@ -182,95 +180,6 @@ SQNN_DEV bool decode_barrier_any(uint32_t flagged)
     return any != 0;
 }
 
-SQNN_DEV void or_bits(uint32_t *row, uint32_t dst, uint32_t v, uint32_t nb)
-{
-    const uint32_t w = dst >> 5, sh = dst & 31;
-    row[w] |= v << sh;
-    if (sh + nb > 32) row[w + 1] |= v >> (32 - sh);
-}
-
-// Where a row segment stands inside the slice stream of one plane.
-struct Cursor {
-    uint64_t s;      // current slice
-    uint32_t off;    // first position of the slice not yet consumed
-    uint32_t dpo;    // index of the slice's first d_patch entry
-};
-
-SQNN_DEV Cursor cursor_at(const PlanePtrs &P, uint32_t n_out, uint64_t p)
-{
-    Cursor c;
-    c.s = p / n_out;
-    c.off = (uint32_t)(p - c.s * n_out);
-    c.dpo = 0;
-    if (P.w_np != 0) {
-        const uint64_t first = c.s & ~(uint64_t)(SQNN_BLOCK_SLICES - 1);
-        c.dpo = __ldg(P.idx + (c.s >> 7));
-        for (uint64_t t = first; t < c.s; ++t) c.dpo += extract_bits(P.np, t * P.w_np, P.w_np);
-    }
-    return c;
-}
-
-// Phase 1 for one plane: bits [cursor, cursor + cnt) of the decoded plane into row[0 .. RB_WORDS).
-SQNN_DEV void decode_segment(const DecodeArgs &A, const PlanePtrs &P, const uint32_t *tab, Cursor &c,
-                             uint32_t cnt, uint32_t *row)
-{
-    const uint32_t n_out = A.n_out, n_in = A.n_in, nw = A.nw, nwp = A.nwp, nch = A.nchunks, cb = A.cb;
-    const uint32_t cmask = (1u << cb) - 1u;
-#pragma unroll
-    for (uint32_t k = 0; k < RB_WORDS; ++k) row[k] = 0;
-    uint32_t pos = 0;
-    while (pos < cnt) {
-        const uint32_t seed = extract_bits(P.wc, c.s * n_in, n_in);
-        const uint32_t np_s = P.w_np ? extract_bits(P.np, c.s * P.w_np, P.w_np) : 0u;
-        const uint32_t o = c.off;
-        for (uint32_t k = 0; k < nw; ++k) {
-            uint32_t lo = 32 * k;
-            uint32_t nb = n_out - lo < 32 ? n_out - lo : 32;
-            if (lo + nb <= o) continue;
-            uint32_t v = 0;
-            for (uint32_t ch = 0; ch < nch; ++ch)
-                v ^= tab[((ch << cb) | ((seed >> (ch * cb)) & cmask)) * nwp + k];
-            if (lo < o) { v >>= (o - lo); nb -= (o - lo); lo = o; }
-            const uint32_t d = pos + (lo - o);
-            if (d < MACRO) or_bits(row, d, v, nb);
-        }
-        for (uint32_t k = 0; k < np_s; ++k) {
-            const uint32_t at = c.dpo + k;
-            if (at >= P.n_dp) { flag(A.status, 2u); break; }
-            const uint32_t pk = P.dp[at];
-            if (pk >= n_out) { flag(A.status, 1u); continue; }
-            if (pk >= o) {
-                const uint32_t d = pos + pk - o;
-                if (d < MACRO) row[d >> 5] ^= 1u << (d & 31);
-            }
-        }
-        const uint32_t avail = n_out - o;
-        if (pos + avail <= cnt) { pos += avail; ++c.s; c.dpo += np_s; c.off = 0; }
-        else { c.off = o + (cnt - pos); pos = cnt; }
-    }
-}
-
-// Phase 1 for a vector that already exists as packed bits in global memory (the mask, or a plane
-// decoded into the workspace): bits [p0, p0 + cnt) into row[0 .. RB_WORDS), zero past cnt.
-SQNN_DEV void copy_segment(const uint32_t *__restrict__ src, uint64_t valid_words, uint64_t p0, uint32_t cnt,
-                           uint32_t *row)
-{
-    const uint64_t w0 = p0 >> 5;
-    const uint32_t sh = (uint32_t)(p0 & 31);
-    uint32_t raw[RB_WORDS];
-#pragma unroll
-    for (uint32_t k = 0; k < RB_WORDS; ++k) raw[k] = w0 + k < valid_words ? __ldg(src + w0 + k) : 0u;
-#pragma unroll
-    for (uint32_t k = 0; k < RB_WORDS - 1; ++k) {
-        uint32_t v = __funnelshift_r(raw[k], raw[k + 1], sh);
-        const uint32_t lo = 32 * k;
-        if (lo >= cnt) v = 0;
-        else if (lo + 32 > cnt) v &= (1u << (cnt - lo)) - 1u;
-        row[k] = v;
-    }
-    row[RB_WORDS - 1] = 0;
-}
-
 SQNN_DEV void tma_load_3d(void *sdst, const CUtensorMap *map, uint64_t *bar, int32_t x, int32_t y, int32_t z)
 {
     asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];\n"
@@ -293,8 +202,7 @@ k_decode_mma(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ C
     uint8_t *b_stages = a_stages + M.stages * a_stage_bytes;
     uint32_t *rb = reinterpret_cast<uint32_t *>(b_stages + (size_t)M.stages * M.b_stage_bytes);   // [buf][item][row][rbp]
     const uint32_t rb_buf_words = n_items * ROWS * rbp;
-    uint32_t *tab = rb + M.rb_bufs * rb_buf_words;
-    uint2 *lut256 = reinterpret_cast<uint2 *>(tab + table_words(A.n_in, A.nwp, A.nchunks, A.cb));   // [256][LUT_COPIES]
+    uint2 *lut256 = reinterpret_cast<uint2 *>(rb + M.rb_bufs * rb_buf_words);                          // [256][LUT_COPIES]
     __nv_bfloat16 *lut = reinterpret_cast<__nv_bfloat16 *>(lut256 + 256 * LUT_COPIES);                             // [row][16]
     float *alpha_s = reinterpret_cast<float *>(lut + ROWS * 16);         // [row][8]
     uint64_t *bars = reinterpret_cast<uint64_t *>(alpha_s + ROWS * 8);
@@ -327,7 +235,6 @@ k_decode_mma(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ C
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
     if (warp == DEC_WARPS + 1) tmem_alloc(tmem_slot, M.tmem_cols);
-    if (!M.bits32) build_tables(A, tab);                    // only the in-kernel decoder needs them
     if (tid < 256) {
         // 4 weights of one plane at a time: index = mask nibble << 4 | bit nibble -> 4 bf16 of -1, 0, +1
         uint32_t h[4];
@@ -374,16 +281,6 @@ k_decode_mma(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ C
 
         if (warp < DEC_WARPS) {
             // ------------------------------ decode warps ------------------------------
-            const uint32_t prow = tid & (ROWS - 1), pq = tid >> 7;          // phase-1 role: row, item class
-            const uint64_t r = r0 + prow;
-            const bool live = r < M.m;
-            Cursor cur[3];
-#pragma unroll
-            for (uint32_t q = 0; q < 3; ++q) {
-                const uint32_t item = pq + 4 * q;                            // plane index (mask = n_q)
-                if (item < A.n_q && live && !M.bits32)
-                    cur[q] = cursor_at(A.pl[item], A.n_out, r * M.n + (uint64_t)macro_begin * MACRO);
-            }
             uint32_t it = step_count, mi = macro_count;
             for (uint32_t mc = macro_begin; mc < macro_end; ++mc, ++mi) {
                 const uint64_t c0 = (uint64_t)mc * MACRO;
@@ -395,7 +292,7 @@ k_decode_mma(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ C
                 if (M.tma_bits) {
                     // the TMA thread fetches them as 128 x 64-byte boxes; wait for this buffer
                     stop = !mbar_wait(bits_full + buf, (mi >> 1) & 1u, abort_flag, A.status);
-                } else if (M.bits32) {
+                } else {
                     // planes exist as packed bits but rows are not 16-byte aligned: 16 consecutive
                     // lanes copy the 16 words of one row segment, 32 rows per pass
                     const uint32_t j = tid & 15;
@@ -419,21 +316,6 @@ k_decode_mma(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ C
                                 v = __funnelshift_r(lo_w, hi_w, sh) & keep;
                             }
                             rb[(item * ROWS + rl) * rbp + j] = v;
-                        }
-                    }
-                } else {
-#pragma unroll
-                    for (uint32_t q = 0; q < 3; ++q) {
-                        const uint32_t item = pq + 4 * q;
-                        if (item > A.n_q) break;
-                        uint32_t *rowbuf = rb + (item * ROWS + prow) * rbp;
-                        if (!live) {
-#pragma unroll
-                            for (uint32_t k = 0; k < RB_WORDS; ++k) rowbuf[k] = 0;
-                        } else if (item < A.n_q) {
-                            decode_segment(A, A.pl[item], tab, cur[q], cnt, rowbuf);
-                        } else {
-                            copy_segment(M.mask32, M.mask_words32, r * M.n + c0, cnt, rowbuf);
                         }
                     }
                 }
@@ -642,17 +524,6 @@ EncodeTiledFn encode_tiled_fn()
     return fn;
 }
 
-// Tables for the per-thread decoder: at most 4 KB.
-void small_tables(DecodeArgs *A)
-{
-    for (uint32_t c = 1; c <= 8; ++c) {
-        const uint32_t cb = (A->n_in + c - 1) / c;
-        if (cb <= 12 && (uint64_t)c * (1ull << cb) * A->nwp * 4 <= 4096) { A->nchunks = c; A->cb = cb; return; }
-    }
-    A->nchunks = 8;
-    A->cb = (A->n_in + 7) / 8;
-}
-
 }  // namespace
 
 // Workspace of the two-stage form: the decoded planes as packed bits (1 bit per weight and plane).
@@ -673,7 +544,6 @@ int mma_dispatch(const sqnn_desc *desc, const DecodeArgs &A0, const uint64_t *d_
 
     MmaArgs M;
     M.A = A0;
-    small_tables(&M.A);
     M.mask32 = (const uint32_t *)d_mask;
     M.mask_words32 = M.A.words64 * 2;
     M.alpha = d_alpha;
@@ -692,7 +562,7 @@ int mma_dispatch(const sqnn_desc *desc, const DecodeArgs &A0, const uint64_t *d_
     // accumulators fit tensor memory; otherwise one tile of rescaled bf16 weights.
     M.per_plane = (uint64_t)M.A.n_q * M.nbt <= 512 ? 1u : 0u;
     // The bit buffer is filled by TMA when the rows of the packed planes start on 16-byte boundaries.
-    M.tma_bits = (d_workspace && desc->n % 128 == 0 && ((uintptr_t)d_mask & 15) == 0) ? 1u : 0u;
+    M.tma_bits = (desc->n % 128 == 0 && ((uintptr_t)d_mask & 15) == 0) ? 1u : 0u;
     const size_t budget = 225 * 1024;        // + 1 KB of static shared memory stays within the 227 KB a block may have
     size_t fixed = 0, per_stage = 0;
     for (;;) {
@@ -702,7 +572,7 @@ int mma_dispatch(const sqnn_desc *desc, const DecodeArgs &A0, const uint64_t *d_
         M.tmem_cols = 32;
         while (M.tmem_cols < a_tiles * M.nbt) M.tmem_cols *= 2;
         fixed = (size_t)M.rb_bufs * (M.A.n_q + 1) * ROWS * M.rbp * 4 +
-                (size_t)table_words(M.A.n_in, M.A.nwp, M.A.nchunks, M.A.cb) * 4 + 256 * 8 * LUT_COPIES + ROWS * 16 * 2 +
+                256 * 8 * LUT_COPIES + ROWS * 16 * 2 +
                 ROWS * 8 * 4 + (3 * MAX_STAGES + 5) * 8 + 16 + 1024;
         per_stage = (size_t)a_tiles * A_STAGE_BYTES + M.b_stage_bytes;
         if (fixed + 2 * per_stage <= budget) break;
@@ -753,11 +623,9 @@ int mma_dispatch(const sqnn_desc *desc, const DecodeArgs &A0, const uint64_t *d_
         : cudaMemset2DAsync(d_y, (size_t)ldy * sizeof(float), 0, (size_t)desc->m * sizeof(float), batch, st);
     if (e != cudaSuccess) return SQNN_E_CUDA;
     if (ensure_dynamic_smem(reinterpret_cast<const void *>(k_decode_mma), smem) != SQNN_OK) return SQNN_E_CUDA;
-    if (d_workspace) {
-        // stage 1: the decode kernel writes the planes as packed bits into the workspace
-        const int rc = decode_bits_dispatch(A0, d_workspace, st);
-        if (rc != SQNN_OK) return rc;
-    }
+    // stage 1: the decode kernel writes the planes as packed bits into the workspace
+    const int rc = decode_bits_dispatch(A0, d_workspace, st);
+    if (rc != SQNN_OK) return rc;
     k_decode_mma<<<row_tiles * M.splits, THREADS, smem, st>>>(xmap, pmap, kmap, M);
     return cudaGetLastError() == cudaSuccess ? SQNN_OK : SQNN_E_CUDA;
 }

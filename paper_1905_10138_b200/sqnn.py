@@ -39,11 +39,15 @@ class Planes(ctypes.Structure):
                 ("planes", ctypes.c_void_p), ("mask", ctypes.c_void_p)]
 
 
+PATCH_HIST_BINS = 16
+
+
 class Stats(ctypes.Structure):
     _fields_ = [("slices", ctypes.c_uint64), ("patches", ctypes.c_uint64 * MAX_PLANES),
                 ("max_patch", ctypes.c_uint32 * MAX_PLANES),
                 ("bits_wc", ctypes.c_uint64), ("bits_npatch", ctypes.c_uint64),
                 ("bits_dpatch", ctypes.c_uint64), ("bits_index", ctypes.c_uint64),
+                ("bits_tables", ctypes.c_uint64), ("patch_hist", ctypes.c_uint64 * PATCH_HIST_BINS),
                 ("bpw_eq1", ctypes.c_double), ("bpw_actual", ctypes.c_double)]
 
     def as_dict(self, n_q: int) -> dict:
@@ -51,6 +55,7 @@ class Stats(ctypes.Structure):
                 "max_patch": [int(v) for v in self.max_patch[:n_q]],
                 "bits_wc": int(self.bits_wc), "bits_npatch": int(self.bits_npatch),
                 "bits_dpatch": int(self.bits_dpatch), "bits_index": int(self.bits_index),
+                "bits_tables": int(self.bits_tables), "patch_hist": [int(v) for v in self.patch_hist],
                 "bpw_eq1": float(self.bpw_eq1), "bpw_actual": float(self.bpw_actual)}
 
 
@@ -63,12 +68,13 @@ class Desc(ctypes.Structure):
     _fields_ = [("m", ctypes.c_uint64), ("n", ctypes.c_uint64), ("slices", ctypes.c_uint64),
                 ("slices_padded", ctypes.c_uint64),
                 ("n_q", ctypes.c_uint32), ("n_out", ctypes.c_uint32), ("n_in", ctypes.c_uint32),
-                ("block_slices", ctypes.c_uint32),
-                ("w_np", ctypes.c_uint32 * MAX_PLANES), ("w_dp", ctypes.c_uint32), ("reserved", ctypes.c_uint32),
-                ("off_xornet", ctypes.c_uint64),
-                ("off_wc", ctypes.c_uint64 * MAX_PLANES), ("off_np", ctypes.c_uint64 * MAX_PLANES),
-                ("off_idx", ctypes.c_uint64 * MAX_PLANES), ("off_dp", ctypes.c_uint64 * MAX_PLANES),
-                ("n_dp", ctypes.c_uint64 * MAX_PLANES), ("total_bytes", ctypes.c_uint64)]
+                ("tile_slices", ctypes.c_uint32),
+                ("tab_chunks", ctypes.c_uint32), ("tab_chunk_bits", ctypes.c_uint32),
+                ("tab_entry_words", ctypes.c_uint32), ("reserved", ctypes.c_uint32),
+                ("off_xornet", ctypes.c_uint64), ("off_tables", ctypes.c_uint64), ("tables_bytes", ctypes.c_uint64),
+                ("off_wc", ctypes.c_uint64 * MAX_PLANES), ("off_idx", ctypes.c_uint64 * MAX_PLANES),
+                ("off_pp", ctypes.c_uint64 * MAX_PLANES),
+                ("n_pp", ctypes.c_uint64 * MAX_PLANES), ("total_bytes", ctypes.c_uint64)]
 
 
 _lib = None
@@ -267,7 +273,8 @@ def sqnn_workspace_bytes(desc: Desc, batch: int) -> int:
 def sqnn_decode_matmul(desc: Desc, d_blob, d_mask, d_alpha, d_x, d_y, d_workspace=None, d_status=None,
                        stream=None):
     """Y[b, r] = sum_c W[r, c] X[b, c].  d_x: [batch, n] float32 or bfloat16 (row stride free);
-    d_y: [batch, m] float32.  Queues on ``stream``; does not synchronise."""
+    d_y: [batch, m] float32.  batch >= 16 needs ``d_workspace`` of ``sqnn_workspace_bytes`` bytes.
+    Queues on ``stream``; does not synchronise."""
     import torch
     if d_x.dim() != 2 or d_y.dim() != 2 or d_x.stride(1) != 1 or d_y.stride(1) != 1:
         raise ValueError("X and Y must be 2-D with unit inner stride")

@@ -90,10 +90,10 @@ def test_malformed_device_patch_entries_set_the_status_word_and_do_not_fault():
     blob, _ = H.blob_from_library(layer)
     dev = H.DeviceLayer(layer, blob)
     d = dev.desc
-    assert d.n_dp[0] > 0
+    assert d.n_pp[0] > 0
     clean = dev.decode_bits()
     assert dev.status_value() == 0
-    dev.blob[int(d.off_dp[0])] = 250                     # position >= n_out = 100
+    dev.blob[int(d.off_pp[0]) + 1] = 255                 # first entry becomes >= 65280 > 256 * n_out
     torch.cuda.synchronize()
     damaged = dev.decode_bits()
     assert dev.status_value() == 1

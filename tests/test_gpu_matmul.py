@@ -113,18 +113,16 @@ MMA = [
 ]
 
 
-@pytest.mark.parametrize("workspace", [True, False], ids=["ws", "nows"])
 @pytest.mark.parametrize("name,make,batch", MMA, ids=[g[0] for g in MMA])
-def test_fused_tensor_core_product_matches_fp64_oracle(name, make, batch, workspace):
-    """workspace=True: planes decoded to packed bits in the workspace first; False: the tensor-core
-    kernel decodes the slices itself."""
+def test_fused_tensor_core_product_matches_fp64_oracle(name, make, batch):
+    """The planes are decoded to packed bits in the workspace, the tensor-core kernel reads them."""
     import torch
     layer = make()
     layer.x_dtype = "bf16"
     x = layer.activations(batch)
     ref = reference(layer, x)
     dev = H.DeviceLayer(layer, H.blob_from_library(layer)[0])
-    y = dev.matmul(x, torch.bfloat16, workspace=workspace)
+    y = dev.matmul(x, torch.bfloat16)
     assert y.shape == (batch, layer.m)
     assert dev.status_value() == 0
     assert H.rel_err(y, ref) <= TOL_BF16, H.rel_err(y, ref)
@@ -149,10 +147,12 @@ def test_tensor_core_path_rejects_what_it_cannot_take():
     assert e.value.status == sqnn.E_UNSUPPORTED
     xok = torch.zeros((16, layer.n), dtype=torch.bfloat16, device="cuda")
     small = torch.zeros(256, dtype=torch.uint8, device="cuda")
-    with pytest.raises(sqnn.SqnnError) as e:                       # workspace given but too small
-        sqnn.sqnn_decode_matmul(dev.desc, dev.blob, dev.mask, dev.alpha, xok, y, small, dev.status)
-    assert e.value.status == sqnn.E_WORKSPACE
+    for ws in (small, None):                                       # workspace too small, or missing
+        with pytest.raises(sqnn.SqnnError) as e:
+            sqnn.sqnn_decode_matmul(dev.desc, dev.blob, dev.mask, dev.alpha, xok, y, ws, dev.status)
+        assert e.value.status == sqnn.E_WORKSPACE
     xb = torch.zeros((16, layer.n + 3), dtype=torch.bfloat16, device="cuda")[:, : layer.n]
+    ws = torch.zeros(sqnn.sqnn_workspace_bytes(dev.desc, 16), dtype=torch.uint8, device="cuda")
     with pytest.raises(sqnn.SqnnError) as e:                       # row pitch not a multiple of 16 bytes
-        sqnn.sqnn_decode_matmul(dev.desc, dev.blob, dev.mask, dev.alpha, xb, y, None, dev.status)
+        sqnn.sqnn_decode_matmul(dev.desc, dev.blob, dev.mask, dev.alpha, xb, y, ws, dev.status)
     assert e.value.status == sqnn.E_UNSUPPORTED

@@ -38,8 +38,8 @@ def test_library_exports_every_declared_symbol():
 
 def test_struct_layouts_match_the_header_sizes():
     # sizes computed by hand from include/sqnn.h (natural alignment)
-    assert ctypes.sizeof(sqnn.Desc) == 4 * 8 + 4 * 4 + 8 * 4 + 8 + 8 + 4 * 8 * 8 + 8 * 8 + 8
-    assert ctypes.sizeof(sqnn.Stats) == 8 + 64 + 32 + 32 + 16
+    assert ctypes.sizeof(sqnn.Desc) == 4 * 8 + 4 * 4 + 4 * 4 + 3 * 8 + 4 * 8 * 8 + 8
+    assert ctypes.sizeof(sqnn.Stats) == 8 + 64 + 32 + 32 + 8 + 16 * 8 + 16
 
 
 LAYERS = [
@@ -108,26 +108,63 @@ def test_blob_layout_invariants():
     layer = wl.make_layer(3, m=60, n=300)
     blob, _ = library_blob(layer)
     d = sqnn.sqnn_describe_host(blob)
-    assert d.total_bytes == blob.size and d.slices_padded % 1024 == 0 and d.block_slices == 128
+    assert d.total_bytes == blob.size and d.slices_padded % 1024 == 0 and d.tile_slices == 256
+    tiles = d.slices_padded // 256
     for i in range(d.n_q):
-        for off in (d.off_wc[i], d.off_np[i], d.off_idx[i], d.off_dp[i]):
+        for off in (d.off_wc[i], d.off_idx[i], d.off_pp[i]):
             assert off % 16 == 0
-        idx = blob[d.off_idx[i]: d.off_idx[i] + 4 * (d.slices_padded // 128 + 1)].view(np.uint32)
-        _, np_, _ = sqnn.sqnn_unpack_host(blob, i)
+        idx = blob[d.off_idx[i]: d.off_idx[i] + 4 * (tiles + 1)].view(np.uint32)
+        _, np_, dp = sqnn.sqnn_unpack_host(blob, i)
         padded = np.zeros(d.slices_padded, np.int64)
         padded[: np_.size] = np_
-        expect = np.concatenate([[0], np.cumsum(padded.reshape(-1, 128).sum(axis=1))])
+        expect = np.concatenate([[0], np.cumsum(padded.reshape(-1, 256).sum(axis=1))])
         assert np.array_equal(idx.astype(np.int64), expect)
-        assert idx[-1] == d.n_dp[i]
+        assert idx[-1] == d.n_pp[i]
+        # a stored entry is the bit position inside its tile: (slice in tile) * n_out + d_patch
+        pp = blob[d.off_pp[i]: d.off_pp[i] + 2 * d.n_pp[i]].view(np.uint16)
+        slice_of = np.repeat(np.arange(np_.size), np_)
+        assert np.array_equal(pp.astype(np.int64), (slice_of % 256) * d.n_out + dp)
     rows = blob[d.off_xornet: d.off_xornet + 4 * d.n_out].view(np.uint32)
     assert np.array_equal(rows, wl.network_rows(layer.M))
+
+
+def test_lookup_tables_in_the_blob_are_the_networks_outputs():
+    """Entry (chunk, value) of the stored tables = M . (value placed at the chunk's bit positions), checked
+    against the oracle's XOR network for every entry."""
+    for cfg, m, n in ((1, 20, 80), (3, 10, 120), (4, 8, 160)):
+        layer = wl.make_layer(cfg, m=m, n=n)
+        blob, _ = library_blob(layer)
+        d = sqnn.sqnn_describe_host(blob)
+        tab = blob[d.off_tables: d.off_tables + d.tables_bytes].view(np.uint32)
+        nwp, cb = d.tab_entry_words, d.tab_chunk_bits
+        assert d.tab_chunks * cb >= d.n_in and nwp * 32 >= d.n_out
+        rng = np.random.default_rng(cfg)
+        for ch in range(d.tab_chunks):
+            for v in rng.integers(0, 1 << cb, 64):
+                seed = (int(v) << (ch * cb)) & ((1 << d.n_in) - 1)
+                want = orc.xor_network(layer.M, [(seed >> t) & 1 for t in range(d.n_in)])
+                e = tab[((ch << cb) | int(v)) * nwp: ((ch << cb) | int(v)) * nwp + nwp]
+                got = wl.unpack_bits(e.astype(np.uint32).view(np.uint8), nwp * 32)
+                assert np.array_equal(got[: d.n_out], want) and not got[d.n_out:].any()
+
+
+def test_patch_histogram_counts_slices_by_n_patch():
+    layer = wl.make_sweep_layer(0, 3, m=64, n=1000)           # ~35 patches per slice: the last bin fills
+    blob, stats = library_blob(layer)
+    _, np_, _ = sqnn.sqnn_unpack_host(blob, 0)
+    want = np.bincount(np.minimum(np_, 15), minlength=16)
+    assert stats["patch_hist"] == want.tolist() and sum(stats["patch_hist"]) == stats["slices"]
+    light = wl.make_layer(2, m=96, n=1000)
+    blob, stats = library_blob(light)
+    _, np_, _ = sqnn.sqnn_unpack_host(blob, 0)
+    assert stats["patch_hist"] == np.bincount(np.minimum(np_, 15), minlength=16).tolist()
 
 
 def test_malformed_blobs_are_rejected_on_the_host():
     layer = wl.make_sweep_layer(1, 2, m=40, n=1000)           # has patches
     blob, _ = library_blob(layer)
     d = sqnn.sqnn_describe_host(blob)
-    assert d.n_dp[0] > 0
+    assert d.n_pp[0] > 1
 
     def bad(mutate):
         b = blob.copy()
@@ -136,11 +173,18 @@ def test_malformed_blobs_are_rejected_on_the_host():
             sqnn.sqnn_describe_host(b)
         assert e.value.status == sqnn.E_BAD_BLOB
 
+    def set_u16(b, off, v):
+        b[off: off + 2] = np.frombuffer(np.uint16(v).tobytes(), dtype=np.uint8)
+
+    pp0 = int(d.off_pp[0])
+    first, second = (int(v) for v in blob[pp0: pp0 + 4].view(np.uint16))
     bad(lambda b: b.__setitem__(0, b[0] ^ 1))                                  # magic
     bad(lambda b: b.__setitem__(8, 9))                                         # version
-    bad(lambda b: b.__setitem__(int(d.off_dp[0]), 255))                        # position >= n_out
-    bad(lambda b: b.__setitem__(int(d.off_idx[0]) + 4, b[int(d.off_idx[0]) + 4] ^ 1))   # offsets
-    bad(lambda b: b.__setitem__(int(d.off_np[0]), b[int(d.off_np[0])] ^ 1))    # n_patch sum
+    bad(lambda b: set_u16(b, pp0, 256 * d.n_out))                              # position outside the tile
+    bad(lambda b: set_u16(b, pp0 + 2, first))                                  # not ascending inside the tile
+    bad(lambda b: b.__setitem__(int(d.off_idx[0]) + 4, b[int(d.off_idx[0]) + 4] ^ 1))   # tile offsets
+    bad(lambda b: b.__setitem__(int(d.off_tables) + 5, b[int(d.off_tables) + 5] ^ 2))   # a table entry
+    bad(lambda b: b.__setitem__(int(d.off_wc[0]) + (d.slices * d.n_in + 7) // 8 + 1, 1))   # a padding slice with a seed
     with pytest.raises(sqnn.SqnnError):
         sqnn.sqnn_describe_host(blob[:-16])                                    # truncated
     with pytest.raises(sqnn.SqnnError):
@@ -149,6 +193,7 @@ def test_malformed_blobs_are_rejected_on_the_host():
     hdr[16:24] = np.frombuffer(np.uint64(1 << 50).tobytes(), dtype=np.uint8)   # absurd m
     with pytest.raises(sqnn.SqnnError):
         sqnn.sqnn_describe_host(hdr)
+    assert second > first
 
 
 def test_invalid_arguments_return_codes_not_crashes():
@@ -166,6 +211,9 @@ def test_invalid_arguments_return_codes_not_crashes():
     with pytest.raises(sqnn.SqnnError):      # patch position >= n_out
         sqnn.sqnn_pack_host(rows, 4, 1, 8, [np.array([3], np.uint32)], [np.array([1], np.uint16)],
                             [np.array([8], np.uint16)])
+    with pytest.raises(sqnn.SqnnError):      # positions of a slice must ascend
+        sqnn.sqnn_pack_host(rows, 4, 1, 8, [np.array([3], np.uint32)], [np.array([2], np.uint16)],
+                            [np.array([5, 2], np.uint16)])
     assert sqnn.status_string(0) == "ok" and "unknown" in sqnn.status_string(-99)
 
 

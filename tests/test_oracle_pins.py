@@ -208,6 +208,26 @@ def test_consistent_systems_need_no_patch():
         assert dp.size == 0
 
 
+def test_exhaustive_search_keeps_the_smallest_of_equally_good_seeds():
+    """Reading taken for Section 5.2 (the paper does not say which of several minimal seeds to keep): the
+    numerically smallest.  Hand-made slices whose optimal seeds are known by inspection."""
+    # one output = w0 xor w1, wanted 1: seeds 01 and 10 are both perfect, 00 and 11 both miss
+    M = np.array([[1, 1]], dtype=np.uint8)
+    wc, dp = orc.encode_slice(M, np.array([1], np.uint8), np.array([1], np.uint8), exhaustive=True)
+    assert wc.tolist() == [1, 0] and dp.size == 0                      # seed 1, not seed 2
+    # outputs (w0, w0, w1 xor w2) wanted (1, 0, 1): one of the first two care bits is lost whatever w0 is;
+    # the four seeds with w1 xor w2 = 1 tie at one patch: 2 (010), 3 (110), 4 (001), 5 (101) -> seed 2
+    M = np.array([[1, 0, 0], [1, 0, 0], [0, 1, 1]], dtype=np.uint8)
+    wq, care = np.array([1, 0, 1], np.uint8), np.ones(3, np.uint8)
+    wc, dp = orc.encode_slice(M, wq, care, exhaustive=True)
+    assert wc.tolist() == [0, 1, 0] and dp.tolist() == [0]
+    # a don't-care on the contested position breaks the tie the other way round
+    wc, dp = orc.encode_slice(M, wq, np.array([0, 1, 1], np.uint8), exhaustive=True)
+    assert wc.tolist() == [0, 1, 0] and dp.size == 0
+    wc, dp = orc.encode_slice(M, wq, np.array([1, 0, 1], np.uint8), exhaustive=True)
+    assert wc.tolist() == [1, 1, 0] and dp.size == 0                   # seed 3 is the smallest with w0 = 1
+
+
 def test_exhaustive_search_is_a_lower_bound_and_alg1_is_close():
     """Section 5.2 / 3.3: the exhaustive search minimises the patch count; Algorithm 1 needs
     somewhat more.  The paper reports up to 10 % more in its own (unspecified) experiments; at
