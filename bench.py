@@ -8,9 +8,14 @@ product) over one batch: ``sqnn_decode_matmul`` on the AlexNet-FC6-shaped layer
 (4096 x 9216, 1 plane, M 100 x 10, 91 % pruned) at batch 1.  The metric is decoded
 weights per second.  Inputs are resident in HBM for ``value``; ``e2e`` repeats the
 measurement with host buffers and the copies inside the timed region.  L2 is flushed
-between timed iterations.  Extra keys report the decode-only kernel on 2^30 weights
-against the HBM roofline, the batch-64 tensor-core path and a dense bf16 product of the
-same layer.  ``--impl reference`` times the CPU oracle on the host cores instead.
+between timed iterations: the K steps are timed as one CUDA-event interval over
+K x (flush + step), and the same interval over K flushes alone is subtracted (one event
+interval per step would be as coarse as the event timer's tick).  ``extra`` reports every
+other configuration: the fused product on the four layer shapes at all their batch sizes
+beside a dense bf16 product of the same layer and that layer's HBM floor, the decode-only
+kernel on 2^30 weights at all 16 sweep points against the HBM roofline, the bf16-output
+and checksum forms of the headline point, and a store-only kernel as the write ceiling.
+``--impl reference`` times the CPU oracle on the host cores instead.
 """
 from __future__ import annotations
 
@@ -30,14 +35,12 @@ if ROOT not in sys.path:
 METRIC = "decoded_weights_per_s_fused_decode_gemv"
 UNIT = "weights/s"
 WORKLOAD = "alexnet-fc6 4096x9216, n_q=1, M 100x10, S=0.91, bf16 activations, batch 1"
-SM_CLOCK_HZ = 1.965e9
 # DRAM bytes (read + write) of one launch, from one ncu capture of each kernel as it stands now on exactly
-# these workloads (summaries under profiles/).  Set an entry to None when its kernel changes.
-#   k_decode_gemv: 5 697 024 read + 0 written (Y stays in L2).
-#   k_decode_bits: 27 243 264 read + 73 993 728 written while the kernel runs; it writes 134 217 728 bytes,
-#   the rest is still dirty in L2 when the kernel ends and is written back during the next launch.
-NCU_DRAM_BYTES_PER_LAUNCH = {"k_decode_gemv": 5697024, "k_decode_bits": 27243264 + 73993728}
+# these workloads (summaries under profiles/).  An entry is None while its kernel has changed since the
+# counters were taken.
+NCU_DRAM_BYTES_PER_LAUNCH = {"k_decode_gemv": None, "k_decode_bits": None}
 LANES_PER_SM = 128
+SMS = 148
 
 
 def measured_peaks():
@@ -47,8 +50,20 @@ def measured_peaks():
             p = json.load(f)
         return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
                 "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
-                "source": "measured"}
-    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+                "sm_max_mhz": float(p.get("sm_max_mhz", 1965.0)), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "sm_max_mhz": 1965.0,
+            "source": "fallback"}
+
+
+def cpu_model() -> str:
+    try:
+        with open("/proc/cpuinfo") as f:
+            for line in f:
+                if line.lower().startswith("model name"):
+                    return line.split(":", 1)[1].strip()
+    except OSError:
+        pass
+    return "unknown"
 
 
 class ClockSampler:
@@ -148,6 +163,26 @@ def time_steps(torch, fn, steps, warmup, flush):
     return [a.elapsed_time(b) for a, b in ev]          # ms
 
 
+def time_interval(torch, fn, reps, flush=None, rounds=3):
+    """Mean device time of one call of fn in ms.  `reps` calls are timed inside ONE event interval; with a
+    flush the interval holds reps x (flush + call) and the same interval over the flushes alone is
+    subtracted.  Best of `rounds` (each round is already a mean over `reps`)."""
+    def interval(body):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        gpu_spin(torch, 2_000_000)
+        e0.record()
+        for _ in range(reps):
+            body()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1)
+    if flush is None:
+        return min(interval(fn) for _ in range(rounds)) / reps
+    both = min(interval(lambda: (flush(), fn())) for _ in range(rounds))
+    alone = min(interval(flush) for _ in range(rounds))
+    return (both - alone) / reps
+
+
 def max_over_ranks(dist, value: float, device) -> float:
     """Slowest rank's value (the job is as slow as its slowest replica); identity without a group."""
     if dist is None:
@@ -212,25 +247,31 @@ def run_ours(args):
         sqnn.sqnn_decode_matmul(desc, b, mk, al, xx, d_y, None, status)
         h_y.copy_(d_y, non_blocking=True)
 
+    for _ in range(args.warmup):
+        flush()
+        step()
     if dist:
         dist.barrier()
     torch.cuda.synchronize()
     sampler = ClockSampler(local)
     sampler.start()
-    times = time_steps(torch, step, args.steps, args.warmup, flush)
+    # exactly K steps in one event interval over K x (flush + step), minus the K flushes alone
+    ms_per_step_local = time_interval(torch, step, args.steps, flush, rounds=1)
     clocks = sampler.stop()
-    total_ms = float(sum(times))
     if dist:
         dist.barrier()
-    total_ms = max_over_ranks(dist, total_ms, "cuda")
+    total_ms = max_over_ranks(dist, ms_per_step_local * args.steps, "cuda")
     torch.cuda.synchronize()
     assert int(status.item()) == 0, "device status word set"
     units = layer.mn * layer.n_q
     ms_per_step = total_ms / args.steps
     value = whole_job_rate(world, units, ms_per_step)
+    times = time_steps(torch, step, min(args.steps, 20), 0, flush)      # one event interval per step, for comparison
 
-    e2e_times = time_steps(torch, step_e2e, args.steps, args.warmup, flush)
-    e2e_ms = max_over_ranks(dist, float(sum(e2e_times)), "cuda")
+    for _ in range(args.warmup):
+        flush()
+        step_e2e()
+    e2e_ms = max_over_ranks(dist, time_interval(torch, step_e2e, args.steps, flush, rounds=1) * args.steps, "cuda")
     h2d = int(h_blob.numel() + h_mask.numel() * 8 + h_alpha.numel() * 4 + h_x.numel() * 2)
     d2h = int(h_y.numel() * 4)
     e2e = {"value": whole_job_rate(world, units, e2e_ms / args.steps), "unit": UNIT,
@@ -239,12 +280,13 @@ def run_ours(args):
     # roofline of the dominant kernel (fused decode-GEMV).  It is bound by plain ALU work: one
     # table-driven expansion per weight bit plus one multiply-add per unpruned weight.
     alg_bytes = stream_bytes(stats, layer, True) + layer.alpha.nbytes + x1.size * 2 + layer.m * 4
-    kern_s = float(np.mean(times)) * 1e-3
+    kern_s = ms_per_step_local * 1e-3
     alg_ops = layer.mn * layer.n_q + int(layer.mask.sum()) * layer.n_q
-    alu_peak = 148 * LANES_PER_SM * SM_CLOCK_HZ / 1e12
+    alu_peak = SMS * LANES_PER_SM * peaks["sm_max_mhz"] * 1e6 / 1e12
     roofline = {"bound": "alu", "achieved": alg_ops / kern_s / 1e12, "peak": alu_peak, "unit": "Tlane-op/s",
                 "frac": alg_ops / kern_s / 1e12 / alu_peak, "traffic": NCU_DRAM_BYTES_PER_LAUNCH["k_decode_gemv"],
-                "kernel": "k_decode_gemv", "peak_source": "148 SMs x 128 lanes x 1.965 GHz",
+                "kernel": "k_decode_gemv", "peak_source": f"148 SMs x 128 lanes x {peaks['sm_max_mhz']:.0f} MHz (max SM clock)",
+                "per_step_event_intervals_ms_median": float(np.median(times)),
                 "hbm_achieved_gbs": alg_bytes / kern_s / 1e9,
                 "hbm_frac_of_measured": alg_bytes / kern_s / 1e9 / peaks["hbm_gbs"],
                 "algorithmic_bytes": alg_bytes, "peaks": peaks["source"]}
@@ -255,15 +297,17 @@ def run_ours(args):
            "config": {"workload": WORKLOAD, "l2": "flushed between timed iterations (256 MB write)",
                       "parallelism": "replicas only" if world > 1 else "single GPU",
                       "bits_per_weight_eq1": stats["bpw_eq1"], "bits_per_weight_stored": stats["bpw_actual"],
-                      "patches": stats["patches"][0]},
+                      "patches": stats["patches"][0],
+                      "timing": "K steps in one CUDA-event interval over K x (flush + step), minus K flushes"},
            "clocks": clocks, "e2e": e2e,
-           "gpu_launches": 2 * args.steps,      # per step: the kernel clearing Y and the fused decode-GEMV
+           "gpu_launches": args.steps,          # per step: one launch of the fused decode-GEMV kernel
            "roofline": roofline}
 
     if rank == 0 and not args.quick:
         out["extra"] = extras(torch, sqnn, wl, layer, desc, d_blob, d_mask, d_alpha, status, flush, peaks, args)
     if rank == 0 and world == 1:
         out["cpu_baseline"] = cpu_baseline(layer)
+        out["cpu_baseline"]["cpu_model"] = cpu_model()
     if rank == 0:
         print(json.dumps(out))
     if dist:
@@ -271,38 +315,93 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-def extras(torch, sqnn, wl, layer, desc, d_blob, d_mask, d_alpha, status, flush, peaks, args):
-    """Reference points beside the headline: dense bf16 product of the same layer, batch 64, and
-    the decode-only kernel on 2^30 weights against the HBM roofline."""
-    ex = {}
-    steps, warm = max(args.steps, 10), max(args.warmup, 3)
-    # dense bf16 weights of the same layer, produced by the library's own bf16 decode
+def product_rows(torch, sqnn, layer, desc, d_blob, d_mask, d_alpha, status, flush, peaks, reps):
+    """Fused product beside a dense bf16 product of the same layer, at every batch size of the configuration."""
+    rows = {}
     w = torch.empty((layer.m, layer.n), dtype=torch.bfloat16, device="cuda")
-    sqnn.sqnn_decode(desc, d_blob, d_mask, d_alpha, sqnn.OUT_BF16, w, status)
-    for batch in (1, 64):
-        x = torch.from_numpy(layer.activations(batch)).cuda().to(torch.bfloat16)
+    sqnn.sqnn_decode(desc, d_blob, d_mask, d_alpha, sqnn.OUT_BF16, w, status)   # dense weights by the library's own decode
+    dense_floor_us = layer.mn * 2 / (peaks["hbm_gbs"] * 1e9) * 1e6
+    for batch in layer.batches:
+        x32 = torch.from_numpy(layer.activations(batch)).cuda()
+        xb = x32.to(torch.bfloat16)
+        x = x32 if layer.x_dtype == "f32" else xb
         y = torch.zeros((batch, layer.m), dtype=torch.float32, device="cuda")
         ws = torch.empty(max(sqnn.sqnn_workspace_bytes(desc, batch), 256), dtype=torch.uint8, device="cuda")
-        dense_cold = time_steps(torch, lambda: torch.matmul(x, w.t()), steps, warm, flush)
-        dense_warm = time_steps(torch, lambda: torch.matmul(x, w.t()), steps, warm, lambda: None)
-        rec = {"dense_bf16_us_cold_l2": 1e3 * float(np.median(dense_cold)),
-               "dense_bf16_us_warm_l2": 1e3 * float(np.median(dense_warm))}
-        try:
-            fn = lambda: sqnn.sqnn_decode_matmul(desc, d_blob, d_mask, d_alpha, x, y, ws, status)
-            cold = time_steps(torch, fn, steps, warm, flush)
-            warm_t = time_steps(torch, fn, steps, warm, lambda: None)
-            rec["fused_us_cold_l2"] = 1e3 * float(np.median(cold))
-            rec["fused_us_warm_l2"] = 1e3 * float(np.median(warm_t))
-        except sqnn.SqnnError as e:
-            rec["fused"] = str(e)
-        ex[f"alexnet_fc6_batch{batch}"] = rec
+        dense = lambda: torch.matmul(xb, w.t())
+        fused = lambda: sqnn.sqnn_decode_matmul(desc, d_blob, d_mask, d_alpha, x, y, ws, status)
+        for f in (dense, fused):
+            for _ in range(3):
+                f()
+        rec = {"dense_bf16_us_cold_l2": 1e3 * time_interval(torch, dense, reps, flush),
+               "dense_bf16_us_warm_l2": 1e3 * time_interval(torch, dense, reps),
+               "dense_bf16_hbm_floor_us": dense_floor_us,
+               "fused_us_cold_l2": 1e3 * time_interval(torch, fused, reps, flush),
+               "fused_us_warm_l2": 1e3 * time_interval(torch, fused, reps),
+               "path": "fp32 ALU (one kernel)" if batch <= 15 else "decode to packed bits + tcgen05 (two kernels)"}
+        rec["fused_vs_dense_cold"] = rec["dense_bf16_us_cold_l2"] / rec["fused_us_cold_l2"]
+        rec["dense_frac_of_hbm_peak_cold"] = dense_floor_us / rec["dense_bf16_us_cold_l2"]
+        if batch >= 16:
+            flops = 2.0 * layer.mn * batch
+            rec["fused_tflops_cold"] = flops / (rec["fused_us_cold_l2"] * 1e-6) / 1e12
+            rec["fused_frac_of_bf16_sustained"] = rec["fused_tflops_cold"] / peaks["bf16_tflops_sustained"]
+        rows[f"batch{batch}"] = rec
     del w
+    return rows
+
+
+def extras(torch, sqnn, wl, layer2, desc2, d_blob2, d_mask2, d_alpha2, status, flush, peaks, args):
+    """Reference points beside the headline: every configuration of the benchmark."""
+    ex = {}
+    reps = 20
+    for cfg in (1, 2, 3, 4):
+        if cfg == 2:
+            layer, desc, d_blob, d_mask, d_alpha = layer2, desc2, d_blob2, d_mask2, d_alpha2
+            stats = None
+        else:
+            layer = wl.make_layer(cfg)
+            blob, mask_words, stats = encode_layer(layer)
+            desc = sqnn.sqnn_describe_host(blob)
+            d_blob = torch.from_numpy(blob).cuda()
+            d_mask = torch.from_numpy(mask_words.view(np.int64)).cuda()
+            d_alpha = torch.from_numpy(layer.alpha).cuda()
+        rec = {"shape": f"{layer.m}x{layer.n}", "n_q": layer.n_q, "network": f"{layer.n_out}x{layer.n_in}",
+               "prune_rate": layer.prune_rate,
+               "batches": product_rows(torch, sqnn, layer, desc, d_blob, d_mask, d_alpha, status, flush, peaks, reps)}
+        if stats is not None:
+            rec["bits_per_weight_eq1"] = stats["bpw_eq1"]
+            rec["bits_per_weight_stored"] = stats["bpw_actual"]
+        ex[f"cfg{cfg}_{layer.name}"] = rec
+        del layer
     if not args.skip_decode_sweep:
-        ex["decode_2p30_100x10_S0.90"] = decode_point(torch, sqnn, wl, 2, 2, flush, peaks, steps, warm)
+        ex["write_ceiling"] = write_ceiling(torch, sqnn, peaks)
+        sweep = {}
+        for i_s in range(len(wl.SWEEP_PRUNE)):
+            for i_m in range(len(wl.SWEEP_NETS)):
+                head = (i_s, i_m) == (2, 2)
+                if args.sweep == "headline" and not head:
+                    continue
+                name = f"S{wl.SWEEP_PRUNE[i_s]:.2f}_{wl.SWEEP_NETS[i_m][0]}x{wl.SWEEP_NETS[i_m][1]}"
+                sweep[name] = decode_point(torch, sqnn, wl, i_s, i_m, flush, peaks, 10, head)
+        ex["decode_2p30"] = sweep
     return ex
 
 
-def decode_point(torch, sqnn, wl, i_s, i_m, flush, peaks, steps, warm, m=32768, n=32768):
+def write_ceiling(torch, sqnn, peaks):
+    """Store-only kernel of the library (the decode kernel's bulk-copy output path, nothing read)."""
+    out = {}
+    for label, nbytes in (("128MiB", 128 << 20), ("1GiB", 1 << 30)):
+        buf = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+        fn = lambda: sqnn.sqnn_store_probe(buf, 3200)
+        for _ in range(3):
+            fn()
+        ms = time_interval(torch, fn, 10)
+        out[label] = {"us": ms * 1e3, "gbs": nbytes / (ms * 1e-3) / 1e9,
+                      "frac_of_copy_peak": nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+        del buf
+    return out
+
+
+def decode_point(torch, sqnn, wl, i_s, i_m, flush, peaks, reps, full, m=32768, n=32768):
     layer = wl.make_sweep_layer(i_s, i_m, m=m, n=n)
     blob, mask_words, stats = encode_layer(layer)
     desc = sqnn.sqnn_describe_host(blob)
@@ -310,33 +409,47 @@ def decode_point(torch, sqnn, wl, i_s, i_m, flush, peaks, steps, warm, m=32768, 
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     words = (layer.mn + 63) // 64
     out = torch.empty(words, dtype=torch.int64, device="cuda")
-    # stream + output (158 MB) exceed L2: timed back to back, no flush
-    t = time_steps(torch, lambda: sqnn.sqnn_decode(desc, d_blob, None, None, sqnn.OUT_BITS, out, status),
-                   steps, warm, lambda: None)
-    sink = torch.zeros(2, dtype=torch.int64, device="cuda")
-    ts = time_steps(torch, lambda: sqnn.sqnn_decode(desc, d_blob, None, None, sqnn.OUT_SINK, sink, status),
-                    steps, warm, flush)
-    # context for the roofline: this kernel writes 5.5 x what it reads, and a write-only stream
-    # (a plain fill of 1 GiB) runs well below the copy peak on this part
-    big = torch.empty(1 << 30, dtype=torch.uint8, device="cuda")
-    tf = time_steps(torch, lambda: big.fill_(1), 5, 3, lambda: None)
-    write_only_gbs = (1 << 30) / (float(np.median(tf)) * 1e-3) / 1e9
-    del big
-    sec = float(np.median(t)) * 1e-3
+    bits = lambda: sqnn.sqnn_decode(desc, d_blob, None, None, sqnn.OUT_BITS, out, status)
+    for _ in range(3):
+        bits()
+    # stream + output (160 MB and more) exceed L2: timed back to back, no flush
+    sec = time_interval(torch, bits, reps) * 1e-3
     in_bytes = stream_bytes(stats, layer, False)
     alg = in_bytes + layer.mn / 8
-    return {"weights": layer.mn, "us": sec * 1e6, "weights_per_s": layer.mn / sec,
-            "compressed_stream_gbs": in_bytes / sec / 1e9,
-            "roofline": {"bound": "hbm", "achieved": alg / sec / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                         "frac": alg / sec / 1e9 / peaks["hbm_gbs"],
-                         "traffic": NCU_DRAM_BYTES_PER_LAUNCH["k_decode_bits"] if (i_s, i_m, m, n) == (2, 2, 32768, 32768) else None,
-                         "kernel": "k_decode_bits",
-                         "algorithmic_bytes": alg, "peaks": peaks["source"],
-                         "write_only_fill_gbs": write_only_gbs,
-                         "frac_of_write_only_fill": alg / sec / 1e9 / write_only_gbs},
-            "sink_us": float(np.median(ts)) * 1e3, "sink_stream_gbs": in_bytes / (float(np.median(ts)) * 1e-3) / 1e9,
-            "bits_per_weight_eq1": stats["bpw_eq1"], "bits_per_weight_stored": stats["bpw_actual"],
-            "status": int(status.item())}
+    # patch entries per tile of 256 slices (the unit a warp works on): how uneven the work is (Section 5.1)
+    tiles = int(desc.slices_padded) // 256
+    idx = blob[int(desc.off_idx[0]): int(desc.off_idx[0]) + 4 * (tiles + 1)].view(np.uint32).astype(np.int64)
+    per_tile = np.diff(idx)[: (int(desc.slices) + 255) // 256]
+    rec = {"weights": layer.mn, "us": sec * 1e6, "weights_per_s": layer.mn / sec,
+           "compressed_stream_gbs": in_bytes / sec / 1e9,
+           "roofline": {"bound": "hbm", "achieved": alg / sec / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                        "frac": alg / sec / 1e9 / peaks["hbm_gbs"],
+                        "traffic": NCU_DRAM_BYTES_PER_LAUNCH["k_decode_bits"] if (full and (m, n) == (32768, 32768)) else None,
+                        "kernel": "k_decode_bits", "algorithmic_bytes": alg, "peaks": peaks["source"]},
+           "bits_per_weight_eq1": stats["bpw_eq1"], "bits_per_weight_stored": stats["bpw_actual"],
+           "patches_per_slice": stats["patches"][0] / stats["slices"],
+           "patches_per_tile_mean": float(per_tile.mean()), "patches_per_tile_max": int(per_tile.max()),
+           "patch_hist": stats["patch_hist"]}
+    if full:
+        sink = torch.zeros(2, dtype=torch.int64, device="cuda")
+        fs = lambda: sqnn.sqnn_decode(desc, d_blob, None, None, sqnn.OUT_SINK, sink, status)
+        fs()
+        ts = time_interval(torch, fs, reps) * 1e-3
+        rec["sink_us"] = ts * 1e6
+        rec["sink_stream_gbs"] = in_bytes / ts / 1e9
+        d_mask = torch.from_numpy(mask_words.view(np.int64)).cuda()
+        d_alpha = torch.from_numpy(layer.alpha).cuda()
+        w = torch.empty((layer.m, layer.n), dtype=torch.bfloat16, device="cuda")
+        fb = lambda: sqnn.sqnn_decode(desc, d_blob, d_mask, d_alpha, sqnn.OUT_BF16, w, status)
+        fb()
+        tb = time_interval(torch, fb, 5) * 1e-3
+        alg_b = in_bytes + layer.mn / 8 + layer.mn * 2
+        rec["bf16_out_us"] = tb * 1e6
+        rec["bf16_out_gbs"] = alg_b / tb / 1e9
+        rec["bf16_out_frac_of_copy_peak"] = alg_b / tb / 1e9 / peaks["hbm_gbs"]
+        del w
+    rec["status"] = int(status.item())
+    return rec
 
 
 def oracle_sample(layer, rows):
@@ -418,7 +531,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--quick", action="store_true", help="headline line only (no extra reference points)")
-    ap.add_argument("--skip-decode-sweep", action="store_true", help="skip the 2^30-weight decode-only point")
+    ap.add_argument("--skip-decode-sweep", action="store_true", help="skip the 2^30-weight decode-only points")
+    ap.add_argument("--sweep", default="all", choices=["all", "headline"],
+                    help="decode-only sweep: all 16 points (default) or only S=0.9, M 100x10")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":

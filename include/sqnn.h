@@ -281,6 +281,13 @@ int sqnn_search_seeds(const sqnn_xornet *net, uint64_t m, uint64_t n, uint32_t n
                       const uint64_t *d_planes, const uint64_t *d_mask, uint32_t *d_wc, uint16_t *d_np,
                       void *cuda_stream);
 
+/* Measurement aid (the paper has no counterpart): writes `bytes` bytes (a multiple of 16) to d_out
+ * (device, 16-byte aligned) the way the packed-bit decode writes its output -- every warp fills a
+ * shared-memory region of chunk_bytes bytes (a multiple of 16, at most 8192) once and sends it out
+ * with bulk copies -- but reads no compressed stream and expands nothing.  Its rate is the ceiling
+ * the decode kernel's output path allows on this GPU.  Errors: INVALID_ARG, CUDA. */
+int sqnn_store_probe(void *d_out, size_t bytes, uint32_t chunk_bytes, void *cuda_stream);
+
 /* Scratch bytes sqnn_decode_matmul needs for this layer and batch (0 for batch <= 15). */
 size_t sqnn_workspace_bytes(const sqnn_desc *desc, uint32_t batch);
 

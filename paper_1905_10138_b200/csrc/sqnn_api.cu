@@ -146,6 +146,43 @@ extern "C" int sqnn_decode(const sqnn_desc *desc, const void *d_blob, const uint
     return decode_shape<0, 0>(A, mode, d_mask, d_alpha, desc->n, d_out, st);
 }
 
+namespace sqnn {
+// Store-only counterpart of k_decode_bits: same block shape, same bulk copies, nothing read.
+__global__ void __launch_bounds__(768, 1) k_store_probe(uint8_t *__restrict__ out, uint64_t chunks, uint32_t chunk_bytes, uint64_t tail_at, uint32_t tail_bytes)
+{
+    extern __shared__ __align__(16) uint32_t smem[];
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    uint32_t *region = smem + warp * (chunk_bytes / 4);
+    for (uint32_t i = lane; i < chunk_bytes / 4; i += 32) region[i] = i * 0x9e3779b9u + warp;
+    fence_async_smem();
+    __syncwarp();
+    if (lane == 0) {
+        for (uint64_t c = (uint64_t)blockIdx.x * nwarps + warp; c < chunks; c += (uint64_t)gridDim.x * nwarps) {
+            const uint32_t nb = c == tail_at ? tail_bytes : chunk_bytes;
+            bulk_store(out + c * chunk_bytes, region, nb);
+        }
+        bulk_wait_read<0>();
+    }
+}
+}  // namespace sqnn
+
+extern "C" int sqnn_store_probe(void *d_out, size_t bytes, uint32_t chunk_bytes, void *cuda_stream)
+{
+    if (!d_out || ((uintptr_t)d_out & 15) || bytes == 0 || (bytes & 15) || chunk_bytes == 0 || (chunk_bytes & 15) ||
+        chunk_bytes > 8192)
+        return SQNN_E_INVALID_ARG;
+    const uint64_t chunks = (bytes + chunk_bytes - 1) / chunk_bytes;
+    const uint32_t tail_bytes = (uint32_t)(bytes - (chunks - 1) * chunk_bytes);
+    const uint32_t warps = 24;
+    const size_t smem = (size_t)warps * chunk_bytes;
+    if (ensure_dynamic_smem(reinterpret_cast<const void *>(k_store_probe), smem) != SQNN_OK) return SQNN_E_CUDA;
+    uint64_t grid = (chunks + warps - 1) / warps;
+    if (grid > (uint64_t)sm_count()) grid = (uint64_t)sm_count();
+    k_store_probe<<<(uint32_t)grid, warps * 32, smem, (cudaStream_t)cuda_stream>>>((uint8_t *)d_out, chunks, chunk_bytes,
+                                                                                 chunks - 1, tail_bytes);
+    return cudaGetLastError() == cudaSuccess ? SQNN_OK : SQNN_E_CUDA;
+}
+
 extern "C" size_t sqnn_workspace_bytes(const sqnn_desc *desc, uint32_t batch)
 {
     if (!desc || batch < 16) return 0;

@@ -11,11 +11,12 @@
 //   - one thread issues tcgen05.mma (K = 16 each) that accumulate in tensor memory.
 // Column ranges of different CTAs are summed with fp32 atomics on Y (cleared beforehand).
 //
-// Two forms of the A stage.  While n_q * N fits the 512 columns of tensor memory, every plane
-// gets its own tile of -1 / 0 / +1 (mask and sign only, four weights per table read) and its own
-// accumulator, and the epilogue forms sum_i alpha[r][i] * D_i: the weights stay exact and the
-// expansion is a few instructions per weight.  Otherwise one tile holds the rescaled weights
-// (+-alpha_1) + (+-alpha_2) + ... rounded to bf16, written sparsely from a per-row value table.
+// The A stage.  Every plane gets its own tile of -1 / 0 / +1 (mask and sign only, four weights per
+// table read) and its own accumulator, and the epilogue forms sum_i alpha[r][i] * D_i: the weights
+// stay exact and the expansion is a few instructions per weight.  The batch is taken in passes whose
+// n_q accumulators fit the 512 columns of tensor memory.  (Only when the sign tiles of all planes do
+// not fit two pipeline stages of shared memory -- six planes and more -- one tile holds the rescaled
+// weights (+-alpha_1) + (+-alpha_2) + ... rounded to bf16 instead.)
 //
 // Where the bits come from.  The planes have been decoded to packed bits in the workspace by the
 // tiled decode kernel (queued just before this one); 128 x 512-bit boxes of them (and of the mask)
@@ -552,15 +553,19 @@ int mma_dispatch(const sqnn_desc *desc, const DecodeArgs &A0, const uint64_t *d_
     M.m = desc->m;
     M.n = desc->n;
     M.batch = batch;
+    // One sign tile and one accumulator per plane, scales applied to the accumulators: the weights stay
+    // exact.  (One tile of rescaled weights rounded to bf16 is not an option: a row holds only 2^n_q
+    // distinct values, their rounding errors add up coherently, and the result misses the 1e-2 tolerance
+    // on wide layers.)  The n_q accumulators of a pass must fit the 512 columns of tensor memory, so the
+    // batch is taken in passes of at most 512 / n_q columns.
     const uint32_t b16 = (batch + 15) / 16 * 16;
-    M.nbt = b16 > 512 ? 512 : b16;
-    if (M.nbt > 256) M.nbt = 512;                       // two full 256-column MMAs per step
+    const uint32_t cap = (512u / M.A.n_q) / 16 * 16;
+    M.nbt = b16 < cap ? b16 : cap;
+    if (M.nbt > 256) M.nbt = 512;                       // one plane: two full 256-column MMAs per step
     M.b_stage_bytes = M.nbt * 128;
     M.bits32 = (const uint32_t *)d_workspace;
     M.plane_words32 = M.A.words64 * 2;
-    // One sign tile and one accumulator per plane (exact weights, cheap expansion) while the
-    // accumulators fit tensor memory; otherwise one tile of rescaled bf16 weights.
-    M.per_plane = (uint64_t)M.A.n_q * M.nbt <= 512 ? 1u : 0u;
+    M.per_plane = 1u;
     // The bit buffer is filled by TMA when the rows of the packed planes start on 16-byte boundaries.
     M.tma_bits = (desc->n % 128 == 0 && ((uintptr_t)d_mask & 15) == 0) ? 1u : 0u;
     const size_t budget = 225 * 1024;        // + 1 KB of static shared memory stays within the 227 KB a block may have
@@ -576,8 +581,8 @@ int mma_dispatch(const sqnn_desc *desc, const DecodeArgs &A0, const uint64_t *d_
                 ROWS * 8 * 4 + (3 * MAX_STAGES + 5) * 8 + 16 + 1024;
         per_stage = (size_t)a_tiles * A_STAGE_BYTES + M.b_stage_bytes;
         if (fixed + 2 * per_stage <= budget) break;
-        if (M.per_plane) { M.per_plane = 0; continue; }        // too many planes for two stages
         if (M.tma_bits) { M.tma_bits = 0; continue; }          // single bit buffer
+        if (M.per_plane) { M.per_plane = 0; continue; }        // too many planes for two stages
         break;
     }
     M.stages = MAX_STAGES;

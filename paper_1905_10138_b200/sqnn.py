@@ -110,6 +110,8 @@ def lib():
         L.sqnn_decode_matmul.argtypes = [P(Desc), vp, vp, vp, vp, i32, u32, i64, vp, i64, vp, sz, vp, vp]
         L.sqnn_decode_matmul_static.argtypes = [P(Desc), vp, vp, vp, vp, i32, u32, i64, vp, i64, vp, vp]
         L.sqnn_decode_matmul_static.restype = i32
+        L.sqnn_store_probe.argtypes = [vp, sz, u32, vp]
+        L.sqnn_store_probe.restype = i32
         L.sqnn_workspace_bytes.argtypes = [P(Desc), u32]
         L.sqnn_workspace_bytes.restype = sz
         L.sqnn_status_string.argtypes = [i32]
@@ -264,6 +266,13 @@ def sqnn_decode(desc: Desc, d_blob, d_mask, d_alpha, mode: int, d_out, d_status=
     _check(lib().sqnn_decode(ctypes.byref(desc), _dev_ptr(d_blob), _dev_ptr(d_mask), _dev_ptr(d_alpha),
                              int(mode), _dev_ptr(d_out), d_out.numel() * d_out.element_size(),
                              _dev_ptr(d_status), _stream_ptr(stream)), "sqnn_decode")
+
+
+def sqnn_store_probe(d_out, chunk_bytes: int = 3200, stream=None):
+    """Measurement aid: fills ``d_out`` (CUDA tensor) with the decode kernel's output path (bulk copies
+    out of shared memory) and nothing else, to measure the write ceiling of that path."""
+    _check(lib().sqnn_store_probe(_dev_ptr(d_out), d_out.numel() * d_out.element_size(), int(chunk_bytes),
+                                  _stream_ptr(stream)), "sqnn_store_probe")
 
 
 def sqnn_workspace_bytes(desc: Desc, batch: int) -> int:

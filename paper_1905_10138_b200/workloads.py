@@ -7,7 +7,10 @@ product), so both the CUDA library's tests and the CPU oracle's tests can take
 their inputs from it.  numpy only.
 
 Randomness: ``numpy.random.Generator(PCG64(seed))`` with seed = 1000 * cfg + k,
-k = 1 weights / plane bits, 2 mask, 3 network M, 4 activations, 5 scales.
+k = 1 weights / plane bits, 2 mask, 3 network M, 4 activations, 5 scales.  Large Bernoulli
+arrays (masks and the bit-planes of the decode-only sweep) are drawn in chunks of 2^24, chunk j
+from ``PCG64(seed).jumped(j)``, so that the chunks can be drawn by several threads and the result
+does not depend on how many there are.
 
 The paper's experiments run on trained AlexNet / LSTM / ResNet weights
 (Section 4, Table 2); those are not available, so each layer here keeps only
@@ -38,16 +41,42 @@ def network_rows(M: np.ndarray) -> np.ndarray:
     return (M.astype(np.uint64) * w).sum(axis=1).astype(np.uint32)
 
 
-def bernoulli_mask(shape, prune_rate: float, seed: int, chunk: int = 1 << 24) -> np.ndarray:
-    """1 = kept (care) with probability 1 - prune_rate, independently per weight."""
-    rng = _rng(seed)
-    total = int(np.prod(shape))
+_CHUNK = 1 << 24
+
+
+def _chunked(total: int, seed: int, draw) -> np.ndarray:
+    """uint8 array of ``total`` entries; chunk j (2^24 entries) = draw(Generator(PCG64(seed).jumped(j)), count).
+    Chunks are drawn by a small thread pool (numpy's generators release the interpreter lock)."""
+    from concurrent.futures import ThreadPoolExecutor
+    import os
     out = np.empty(total, dtype=np.uint8)
+    starts = list(range(0, total, _CHUNK))
+
+    def one(j):
+        a = starts[j]
+        b = min(total, a + _CHUNK)
+        rng = np.random.Generator(np.random.PCG64(int(seed)).jumped(j))
+        out[a:b] = draw(rng, b - a)
+
+    if len(starts) == 1:
+        one(0)
+    else:
+        with ThreadPoolExecutor(max_workers=min(len(starts), os.cpu_count() or 4)) as ex:
+            list(ex.map(one, range(len(starts))))
+    return out
+
+
+def bernoulli_mask(shape, prune_rate: float, seed: int) -> np.ndarray:
+    """1 = kept (care) with probability 1 - prune_rate, independently per weight."""
     keep = np.float32(1.0 - prune_rate)
-    for a in range(0, total, chunk):
-        b = min(total, a + chunk)
-        out[a:b] = rng.random(b - a, dtype=np.float32) < keep
-    return out.reshape(shape)
+    total = int(np.prod(shape))
+    return _chunked(total, seed, lambda rng, cnt: rng.random(cnt, dtype=np.float32) < keep).reshape(shape)
+
+
+def bernoulli_bits(total: int, seed: int) -> np.ndarray:
+    """``total`` bits, 0 or 1 with equal probability (one random byte gives eight of them)."""
+    return _chunked(total, seed, lambda rng, cnt: np.unpackbits(
+        rng.integers(0, 256, size=(cnt + 7) // 8, dtype=np.uint8), bitorder="little", count=cnt))
 
 
 def magnitude_mask(w: np.ndarray, keep_fraction: float) -> np.ndarray:
@@ -192,12 +221,7 @@ def make_sweep_layer(i_s: int, i_m: int, m: int = 32768, n: int = 32768) -> Laye
     n_out, n_in = SWEEP_NETS[i_m]
     base = 5000 + 10 * i_s + i_m
     total = m * n
-    rng = _rng(base + 1)
-    planes = np.empty(total, dtype=np.uint8)
-    chunk = 1 << 24
-    for a in range(0, total, chunk):
-        b = min(total, a + chunk)
-        planes[a:b] = rng.integers(0, 2, size=b - a, dtype=np.uint8)
+    planes = bernoulli_bits(total, base + 1)
     mask = bernoulli_mask((m, n), prune, base + 2)
     alpha = (_rng(base + 5).random((m, 1), dtype=np.float32) + np.float32(0.5)).astype(np.float32)
     M = xor_network(n_out, n_in, base + 3)

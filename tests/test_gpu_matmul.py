@@ -126,13 +126,16 @@ def test_fused_tensor_core_product_matches_fp64_oracle(name, make, batch):
     assert y.shape == (batch, layer.m)
     assert dev.status_value() == 0
     assert H.rel_err(y, ref) <= TOL_BF16, H.rel_err(y, ref)
-    # tighter: the kernel either keeps the weights exact (one sign tile per plane, scales applied to
-    # the accumulators) or rounds the rescaled weights to bf16; against the matching fp64 product
-    # only the fp32 accumulation order differs
-    ref_bits = H.oracle_decode(layer, H.oracle_encode(layer))
-    _, wbf = orc.reconstruct(ref_bits, layer.mask, layer.alpha, want_f32=False)
-    w = (wbf.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
-    assert min(H.rel_err(y, ref), H.rel_err(y, x.astype(np.float64) @ w.T)) <= 2e-4
+    # tighter: up to four planes the kernel keeps the weights exact (one sign tile per plane, scales applied
+    # to the accumulators), so against the oracle's product only the fp32 accumulation order differs; with
+    # more planes it rounds the rescaled weights to bf16 and is held against the fp64 product of those
+    if layer.n_q <= 4:
+        assert H.rel_err(y, ref) <= 2e-4, H.rel_err(y, ref)
+    else:
+        ref_bits = H.oracle_decode(layer, H.oracle_encode(layer))
+        _, wbf = orc.reconstruct(ref_bits, layer.mask, layer.alpha, want_f32=False)
+        w = (wbf.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+        assert H.rel_err(y, x.astype(np.float64) @ w.T) <= 2e-4
 
 
 def test_tensor_core_path_rejects_what_it_cannot_take():
