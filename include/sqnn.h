@@ -171,13 +171,42 @@ int sqnn_stats_host(const void *blob, size_t blob_bytes, sqnn_stats *stats);
 
 /* Blocked n_patch assignment (Section 5.2): what Eq. 1 gives when the n_patch field width is
  * chosen per block of `block_slices` consecutive slices (from that block's own largest count)
- * instead of once per plane.  Accounting only: the stored format keeps one width per plane.
+ * instead of once per plane, Eq. 1 taken literally (sqnn_store_host builds the format itself).
  * *bits_npatch = sum over planes and blocks of (slices in the block) * ceil(lg max p of the block),
  * *bpw_eq1 = Eq. 1's bits per weight with that middle term (the block widths themselves, which the
  * paper does not count, are not counted).  Either output may be NULL.  Errors: INVALID_ARG
  * (block_slices = 0), BAD_BLOB. */
 int sqnn_stats_blocked_host(const void *blob, size_t blob_bytes, uint64_t block_slices,
                             double *bpw_eq1, uint64_t *bits_npatch);
+
+/* Sizes of a storage-form buffer (sqnn_store_host): bits of the seed streams, of the per-block width
+ * bytes, of the n_patch fields and of the d_patch entries over all planes, the whole buffer in
+ * bytes (header, rows of M and byte padding of each stream included) and bits per weight of the
+ * four streams together. */
+typedef struct sqnn_store_info {
+    uint64_t bits_wc, bits_widths, bits_npatch, bits_dpatch;
+    uint64_t total_bytes;
+    double bpw;
+} sqnn_store_info;
+
+/* Storage form of a layer: the three parts of Section 3.2 packed for files, with the blocked n_patch
+ * assignment of Section 5.2 made real.  Per plane: the w^c stream (n_in bits per slice, l slices, no
+ * padding slices); one width byte per block of `block_slices` consecutive slices, w = ceil(lg(max
+ * n_patch of the block + 1)) -- the narrowest field that can hold every count of the block, 0 for a
+ * block without patches (Eq. 1 writes ceil(lg max p), which cannot hold the value max p when it is a
+ * power of two; sqnn_stats_blocked_host reports that literal figure); the n_patch fields, w bits each,
+ * block after block; the d_patch entries, ceil(lg n_out) bits each, slice order.  How a block's width
+ * reaches the decoder is not stated in the paper; the width bytes are this library's answer and are
+ * counted.  blob: a device blob (validated first).  *stored is allocated by the library (sqnn_free).
+ * info may be NULL.  Errors: INVALID_ARG (NULL, block_slices = 0), BAD_BLOB, NOMEM. */
+int sqnn_store_host(const void *blob, size_t blob_bytes, uint64_t block_slices,
+                    void **stored, size_t *stored_bytes, sqnn_store_info *info);
+
+/* Inverse of sqnn_store_host: validates a storage-form buffer (magic, sizes, every count <= n_out and
+ * within its block's width, every position < n_out and ascending inside a slice) and rebuilds the
+ * device blob, byte for byte the one sqnn_store_host was given.  *blob is allocated by the library
+ * (sqnn_free).  Errors: INVALID_ARG, BAD_BLOB, NOMEM. */
+int sqnn_load_host(const void *stored, size_t stored_bytes, void **blob, size_t *blob_bytes);
 
 /* Result of sqnn_fifo_model_host. */
 typedef struct sqnn_fifo_result {

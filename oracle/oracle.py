@@ -60,6 +60,7 @@ def _L():
         lib.orc_matmul.argtypes = [i64, i64, i32, vp, vp, vp, vp, i64, vp]
         lib.orc_eq1.argtypes = [i64, i32, i32, vp, vp]
         lib.orc_eq1_blocked.argtypes = [i64, i32, i32, vp, i64, vp]
+        lib.orc_blocked_field_bits.argtypes = [i64, vp, i64, vp]
         lib.orc_fifo_model.argtypes = [i64, vp, i32, i32, i32, vp]
         lib.orc_csr_relative_time.argtypes = [i64, vp, i32]
         lib.orc_csr_relative_time.restype = ctypes.c_double
@@ -216,6 +217,16 @@ def eq1_blocked(mn: int, n_out: int, n_in: int, np_, block: int) -> dict:
     _L().orc_eq1_blocked(mn, n_out, n_in, _p(np_), block, _p(out))
     return {"r": out[0], "bits_npatch": out[1], "blocks": int(out[2]), "bits_widths": out[3],
             "bits_per_weight": 1.0 / out[0]}
+
+
+def blocked_field_bits(np_, block: int) -> dict:
+    """Bits of the n_patch fields when every block of `block` slices gets the narrowest field that holds
+    all its counts, ceil(lg(max p + 1)) (Section 5.2 as a stored format)."""
+    np_ = np.ascontiguousarray(np_, dtype=np.uint16)
+    assert block >= 1
+    out = np.zeros(2, dtype=np.float64)
+    _L().orc_blocked_field_bits(np_.size, _p(np_), block, _p(out))
+    return {"bits_npatch": int(out[0]), "blocks": int(out[1])}
 
 
 def fifo_model(np_, n_fifo: int, rate: int, depth: int) -> dict:

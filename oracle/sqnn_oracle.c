@@ -441,6 +441,30 @@ void orc_eq1_blocked(int64_t mn, int n_out, int n_in, const uint16_t *np, int64_
 }
 
 /* ------------------------------------------------------------------------- */
+/* Blocked n_patch assignment (Section 5.2) as a stored format: a field must  */
+/* be able to hold every count of its block, the largest included, so its     */
+/* width is ceil(lg(max p of the block + 1)) bits (Eq. 1's ceil(lg max p)     */
+/* cannot hold max p when that is a power of two; same reading as for the     */
+/* per-plane width).  out[0] = sum over blocks of (slices in the block) *     */
+/* width, out[1] = number of blocks.                                          */
+/* ------------------------------------------------------------------------- */
+void orc_blocked_field_bits(int64_t l, const uint16_t *np, int64_t block, double *out)
+{
+    double bits = 0.0;
+    int64_t blocks = 0;
+    for (int64_t s0 = 0; s0 < l; s0 += block) {
+        int64_t s1 = s0 + block < l ? s0 + block : l;
+        int64_t maxp = 0;
+        for (int64_t s = s0; s < s1; ++s)
+            if (np[s] > maxp) maxp = np[s];
+        bits += (double)(s1 - s0) * (double)ceil_lg(maxp + 1);
+        blocks += 1;
+    }
+    out[0] = bits;
+    out[1] = (double)blocks;
+}
+
+/* ------------------------------------------------------------------------- */
 /* Patch-data FIFO of one XOR-gate network (Section 5.1), cycle by cycle.     */
 /* Reading of the section (it gives no equations):                            */
 /*  - the network decrypts one slice per cycle when nothing holds it up;      */

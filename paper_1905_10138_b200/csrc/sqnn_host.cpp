@@ -580,6 +580,190 @@ int sqnn_stats_blocked_host(const void *blob, size_t blob_bytes, uint64_t block_
     return SQNN_OK;
 }
 
+// ---------------------------------------------------------------------------------------------
+// storage form
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+const char STORE_MAGIC[8] = {'S', 'Q', 'N', 'N', 'S', 'T', 'R', '1'};
+
+struct StoreHeader {
+    char magic[8];
+    uint64_t m, n, block_slices, total_bytes;
+    uint32_t n_q, n_out, n_in, reserved;
+    uint64_t n_dp[SQNN_MAX_PLANES];
+    uint64_t reserved2;
+};
+static_assert(sizeof(StoreHeader) == 128, "storage header is 128 bytes");
+
+struct BitWriter {
+    std::vector<uint8_t> &buf;
+    uint64_t acc = 0;
+    uint32_t have = 0;
+    explicit BitWriter(std::vector<uint8_t> &b) : buf(b) {}
+    void put(uint32_t v, uint32_t width)
+    {
+        if (width == 0) return;
+        acc |= (uint64_t)v << have;
+        have += width;
+        while (have >= 8) { buf.push_back((uint8_t)acc); acc >>= 8; have -= 8; }
+    }
+    void flush() { if (have) { buf.push_back((uint8_t)acc); acc = 0; have = 0; } }     // streams start on a byte
+};
+
+struct BitReader {
+    const uint8_t *p, *end;
+    uint64_t acc = 0;
+    uint32_t have = 0;
+    bool ok = true;
+    BitReader(const uint8_t *b, const uint8_t *e) : p(b), end(e) {}
+    uint32_t get(uint32_t width)
+    {
+        if (width == 0) return 0;
+        while (have < width) {
+            if (p >= end) { ok = false; return 0; }
+            acc |= (uint64_t)*p++ << have;
+            have += 8;
+        }
+        const uint32_t v = (uint32_t)(acc & (((uint64_t)1 << width) - 1));
+        acc >>= width;
+        have -= width;
+        return v;
+    }
+    void align() { acc = 0; have = 0; }
+};
+
+}  // namespace
+
+int sqnn_store_host(const void *blob, size_t blob_bytes, uint64_t block_slices,
+                    void **stored, size_t *stored_bytes, sqnn_store_info *info)
+{
+    if (!stored || !stored_bytes || block_slices == 0) return SQNN_E_INVALID_ARG;
+    sqnn_desc d;
+    int rc = sqnn_describe_host(blob, blob_bytes, &d);
+    if (rc != SQNN_OK) return rc;
+    try {
+        const uint8_t *b = (const uint8_t *)blob;
+        const uint64_t l = d.slices;
+        const uint32_t w_dp = ceil_lg_u64(d.n_out);
+        StoreHeader h;
+        std::memset(&h, 0, sizeof h);
+        std::memcpy(h.magic, STORE_MAGIC, 8);
+        h.m = d.m; h.n = d.n; h.block_slices = block_slices;
+        h.n_q = d.n_q; h.n_out = d.n_out; h.n_in = d.n_in;
+        std::vector<uint8_t> out(sizeof h, 0);
+        out.insert(out.end(), b + d.off_xornet, b + d.off_xornet + (size_t)d.n_out * 4);
+        sqnn_store_info si;
+        std::memset(&si, 0, sizeof si);
+        std::vector<uint16_t> np(l ? l : 1);
+        for (uint32_t i = 0; i < d.n_q; ++i) {
+            h.n_dp[i] = d.n_pp[i];
+            const uint32_t *wcs = (const uint32_t *)(b + d.off_wc[i]);
+            const uint16_t *pp = (const uint16_t *)(b + d.off_pp[i]);
+            count_patches(b, d, i, np.data());
+            BitWriter bw(out);
+            for (uint64_t s = 0; s < l; ++s) bw.put(read_field(wcs, s, d.n_in), d.n_in);
+            bw.flush();
+            si.bits_wc += l * d.n_in;
+            const uint64_t blocks = (l + block_slices - 1) / block_slices;
+            std::vector<uint8_t> widths(blocks);
+            for (uint64_t k = 0; k < blocks; ++k) {
+                uint32_t maxp = 0;
+                for (uint64_t s = k * block_slices; s < std::min(l, (k + 1) * block_slices); ++s) maxp = std::max<uint32_t>(maxp, np[s]);
+                widths[k] = (uint8_t)ceil_lg_u64((uint64_t)maxp + 1);
+            }
+            out.insert(out.end(), widths.begin(), widths.end());
+            si.bits_widths += blocks * 8;
+            for (uint64_t s = 0; s < l; ++s) {
+                bw.put(np[s], widths[s / block_slices]);
+                si.bits_npatch += widths[s / block_slices];
+            }
+            bw.flush();
+            for (uint64_t k = 0; k < d.n_pp[i]; ++k) bw.put(pp[k] % d.n_out, w_dp);
+            bw.flush();
+            si.bits_dpatch += d.n_pp[i] * w_dp;
+        }
+        h.total_bytes = out.size();
+        std::memcpy(out.data(), &h, sizeof h);
+        uint8_t *res = (uint8_t *)std::malloc(out.size());
+        if (!res) return SQNN_E_NOMEM;
+        std::memcpy(res, out.data(), out.size());
+        *stored = res;
+        *stored_bytes = out.size();
+        si.total_bytes = out.size();
+        si.bpw = (double)(si.bits_wc + si.bits_widths + si.bits_npatch + si.bits_dpatch) / (double)(d.m * d.n);
+        if (info) *info = si;
+        return SQNN_OK;
+    } catch (const std::bad_alloc &) {
+        return SQNN_E_NOMEM;
+    }
+}
+
+int sqnn_load_host(const void *stored, size_t stored_bytes, void **blob, size_t *blob_bytes)
+{
+    if (!stored || !blob || !blob_bytes) return SQNN_E_INVALID_ARG;
+    if (stored_bytes < sizeof(StoreHeader)) return SQNN_E_BAD_BLOB;
+    const uint8_t *b = (const uint8_t *)stored, *end = b + stored_bytes;
+    StoreHeader h;
+    std::memcpy(&h, b, sizeof h);
+    if (std::memcmp(h.magic, STORE_MAGIC, 8) != 0 || h.total_bytes != stored_bytes) return SQNN_E_BAD_BLOB;
+    if (h.n_out < 1 || h.n_out > SQNN_MAX_N_OUT || h.n_in < 1 || h.n_in > SQNN_MAX_N_IN || h.n_q < 1 ||
+        h.n_q > SQNN_MAX_PLANES || h.m == 0 || h.n == 0 || h.m > ((uint64_t)1 << 40) / h.n || h.block_slices == 0)
+        return SQNN_E_BAD_BLOB;
+    try {
+        const uint64_t mn = h.m * h.n, l = (mn + h.n_out - 1) / h.n_out;
+        const uint32_t w_dp = ceil_lg_u64(h.n_out);
+        const uint8_t *p = b + sizeof h;
+        if ((uint64_t)(end - p) < (uint64_t)h.n_out * 4) return SQNN_E_BAD_BLOB;
+        std::vector<uint32_t> rows(h.n_out);
+        std::memcpy(rows.data(), p, (size_t)h.n_out * 4);
+        p += (size_t)h.n_out * 4;
+        std::vector<PlaneArrays> pa(h.n_q);
+        std::vector<std::vector<uint16_t>> dp16(h.n_q);
+        for (uint32_t i = 0; i < h.n_q; ++i) {
+            if (h.n_dp[i] > 0xffffffffull) return SQNN_E_BAD_BLOB;
+            BitReader br(p, end);
+            pa[i].wc.resize(l);
+            pa[i].np.resize(l);
+            for (uint64_t s = 0; s < l; ++s) pa[i].wc[s] = br.get(h.n_in);
+            if (!br.ok) return SQNN_E_BAD_BLOB;
+            br.align();
+            const uint64_t blocks = (l + h.block_slices - 1) / h.block_slices;
+            if ((uint64_t)(end - br.p) < blocks) return SQNN_E_BAD_BLOB;
+            const uint8_t *widths = br.p;
+            br.p += blocks;
+            uint64_t sum = 0;
+            for (uint64_t s = 0; s < l; ++s) {
+                const uint32_t w = widths[s / h.block_slices];
+                if (w > 9) return SQNN_E_BAD_BLOB;
+                const uint32_t v = br.get(w);
+                if (v > h.n_out) return SQNN_E_BAD_BLOB;
+                pa[i].np[s] = (uint16_t)v;
+                sum += v;
+            }
+            if (!br.ok || sum != h.n_dp[i]) return SQNN_E_BAD_BLOB;
+            br.align();
+            dp16[i].resize(sum ? sum : 1);
+            for (uint64_t k = 0; k < sum; ++k) dp16[i][k] = (uint16_t)br.get(w_dp);
+            if (!br.ok) return SQNN_E_BAD_BLOB;
+            br.align();
+            p = br.p;
+        }
+        if (p != end) return SQNN_E_BAD_BLOB;
+        sqnn_xornet net{h.n_out, h.n_in, rows.data()};
+        if (h.n_in < 32)
+            for (uint32_t j = 0; j < h.n_out; ++j)
+                if (rows[j] >> h.n_in) return SQNN_E_BAD_BLOB;
+        std::vector<const uint32_t *> wcp(h.n_q);
+        std::vector<const uint16_t *> npp(h.n_q), dpp(h.n_q);
+        for (uint32_t i = 0; i < h.n_q; ++i) { wcp[i] = pa[i].wc.data(); npp[i] = pa[i].np.data(); dpp[i] = dp16[i].data(); }
+        const int rc = build_blob(&net, h.m, h.n, h.n_q, wcp.data(), npp.data(), nullptr, dpp.data(), blob, blob_bytes);
+        return rc == SQNN_E_INVALID_ARG ? SQNN_E_BAD_BLOB : rc;     // bad contents, not a bad call
+    } catch (const std::bad_alloc &) {
+        return SQNN_E_NOMEM;
+    }
+}
+
 int sqnn_fifo_model_host(const uint16_t *np, uint64_t l, uint32_t n_fifo, uint32_t rate, uint32_t depth,
                          sqnn_fifo_result *result)
 {

@@ -59,6 +59,11 @@ class Stats(ctypes.Structure):
                 "bpw_eq1": float(self.bpw_eq1), "bpw_actual": float(self.bpw_actual)}
 
 
+class StoreInfo(ctypes.Structure):
+    _fields_ = [("bits_wc", ctypes.c_uint64), ("bits_widths", ctypes.c_uint64), ("bits_npatch", ctypes.c_uint64),
+                ("bits_dpatch", ctypes.c_uint64), ("total_bytes", ctypes.c_uint64), ("bpw", ctypes.c_double)]
+
+
 class FifoResult(ctypes.Structure):
     _fields_ = [("cycles", ctypes.c_uint64), ("stall_bandwidth", ctypes.c_uint64),
                 ("stall_empty", ctypes.c_uint64), ("stall_full", ctypes.c_uint64), ("peak", ctypes.c_uint64)]
@@ -102,6 +107,10 @@ def lib():
         L.sqnn_stats_host.argtypes = [vp, sz, P(Stats)]
         L.sqnn_stats_blocked_host.argtypes = [vp, sz, u64, P(ctypes.c_double), P(u64)]
         L.sqnn_stats_blocked_host.restype = i32
+        L.sqnn_store_host.argtypes = [vp, sz, u64, P(vp), P(sz), P(StoreInfo)]
+        L.sqnn_store_host.restype = i32
+        L.sqnn_load_host.argtypes = [vp, sz, P(vp), P(sz)]
+        L.sqnn_load_host.restype = i32
         L.sqnn_fifo_model_host.argtypes = [vp, u64, u32, u32, u32, P(FifoResult)]
         L.sqnn_fifo_model_host.restype = i32
         L.sqnn_free.argtypes = [vp]
@@ -226,6 +235,23 @@ def sqnn_stats_blocked_host(blob: np.ndarray, block_slices: int) -> dict:
     _check(lib().sqnn_stats_blocked_host(_np_ptr(blob), blob.size, int(block_slices), ctypes.byref(bpw),
                                          ctypes.byref(bits)), "sqnn_stats_blocked_host")
     return {"bpw_eq1": bpw.value, "bits_npatch": int(bits.value)}
+
+
+def sqnn_store_host(blob: np.ndarray, block_slices: int):
+    """Device blob -> storage form with per-block n_patch widths (Sections 3.2, 5.2).  Returns (bytes, info dict)."""
+    blob = np.ascontiguousarray(blob, dtype=np.uint8)
+    out, nbytes, info = ctypes.c_void_p(), ctypes.c_size_t(), StoreInfo()
+    _check(lib().sqnn_store_host(_np_ptr(blob), blob.size, int(block_slices), ctypes.byref(out), ctypes.byref(nbytes),
+                                 ctypes.byref(info)), "sqnn_store_host")
+    return _take(out, nbytes.value), {k: getattr(info, k) for k, _ in StoreInfo._fields_}
+
+
+def sqnn_load_host(stored: np.ndarray) -> np.ndarray:
+    """Storage form -> device blob."""
+    stored = np.ascontiguousarray(stored, dtype=np.uint8)
+    out, nbytes = ctypes.c_void_p(), ctypes.c_size_t()
+    _check(lib().sqnn_load_host(_np_ptr(stored), stored.size, ctypes.byref(out), ctypes.byref(nbytes)), "sqnn_load_host")
+    return _take(out, nbytes.value)
 
 
 def sqnn_fifo_model_host(n_patch: np.ndarray, n_fifo: int, rate: int, depth: int) -> dict:

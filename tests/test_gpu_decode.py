@@ -82,6 +82,32 @@ def test_library_encoded_blob_decodes_to_the_same_bits():
         assert np.array_equal(got[i], wl.pack_bits(ref[i]))
 
 
+def test_layer_restored_from_the_storage_form_with_mixed_block_widths_decodes_bit_exactly():
+    """Section 5.2: a layer whose blocks of 128 slices need different n_patch widths (0 bits where a region
+    is fully pruned) goes through the storage form and back, then through the GPU decoder."""
+    rng = np.random.default_rng(61)
+    m, n = 96, 4000
+    keep = np.concatenate([np.zeros(32), np.full(32, 0.35), np.full(32, 0.04)])          # per row
+    mask = (rng.random((m, n)) < keep[:, None]).astype(np.uint8)
+    planes = rng.integers(0, 2, (1, m, n), dtype=np.uint8)
+    layer = wl.Layer(name="mixed", cfg=0, m=m, n=n, n_q=1, n_out=100, n_in=10, prune_rate=0.0,
+                     M=wl.xor_network(100, 10, 62), planes=planes, mask=mask,
+                     alpha=np.ones((m, 1), np.float32), x_dtype="f32", batches=(1,), seed_x=63)
+    blob, _ = H.blob_from_library(layer)
+    _, np_, _ = sqnn.sqnn_unpack_host(blob, 0)
+    per_block = [int(np_[a:a + 128].max()) for a in range(0, np_.size, 128)]
+    widths = {int(np.ceil(np.log2(p + 1))) for p in per_block}
+    assert 0 in widths and len(widths) >= 3
+    stored, info = sqnn.sqnn_store_host(blob, 128)
+    assert info["bits_npatch"] == orc.blocked_field_bits(np_, 128)["bits_npatch"] < np_.size * max(widths)
+    restored = sqnn.sqnn_load_host(stored)
+    assert np.array_equal(restored, blob)
+    dev = H.DeviceLayer(layer, restored)
+    ref = H.oracle_decode(layer, H.oracle_encode(layer))
+    assert np.array_equal(dev.decode_bits()[0], wl.pack_bits(ref[0]))
+    assert dev.status_value() == 0
+
+
 def test_malformed_device_patch_entries_set_the_status_word_and_do_not_fault():
     """The host validator rejects such blobs; if a device copy is damaged anyway the kernel
     skips the entry and reports through the status word."""

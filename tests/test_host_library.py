@@ -267,3 +267,61 @@ def test_fifo_model_matches_the_oracle():
                 assert got[key] == ref[key], (key, n_fifo, rate, depth)
     with pytest.raises(sqnn.SqnnError):
         sqnn.sqnn_fifo_model_host(cases[0], 0, 1, 1)
+
+
+@pytest.mark.parametrize("name,make", LAYERS[:6], ids=[n for n, _ in LAYERS[:6]])
+def test_storage_form_with_blocked_npatch_widths_round_trips(name, make):
+    """Section 5.2 as a format: per-block field widths, sizes against the oracle's accounting, and the device
+    blob rebuilt byte for byte."""
+    layer = make()
+    blob, stats = library_blob(layer)
+    ref = oracle_arrays(layer)
+    l = (layer.mn + layer.n_out - 1) // layer.n_out
+    lg_n_out = int(np.ceil(np.log2(layer.n_out)))
+    for block in (1, 16, 128, l, 3 * l):
+        stored, info = sqnn.sqnn_store_host(blob, block)
+        want = [orc.blocked_field_bits(a[1], block) for a in ref]
+        assert info["bits_npatch"] == sum(w["bits_npatch"] for w in want)
+        assert info["bits_widths"] == 8 * sum(w["blocks"] for w in want)
+        assert info["bits_wc"] == layer.n_q * l * layer.n_in
+        assert info["bits_dpatch"] == sum(int(a[1].sum()) for a in ref) * lg_n_out
+        assert info["total_bytes"] == stored.size
+        assert info["bpw"] == pytest.approx((info["bits_wc"] + info["bits_widths"] + info["bits_npatch"] +
+                                             info["bits_dpatch"]) / layer.mn)
+        assert np.array_equal(sqnn.sqnn_load_host(stored), blob)
+    with pytest.raises(sqnn.SqnnError):
+        sqnn.sqnn_store_host(blob, 0)
+
+
+def test_storage_form_dense_region_case_and_rejection_of_damaged_buffers():
+    """Section 5.2's motivating case: patches concentrated in one region.  One field width for the whole plane
+    pays for the worst slice everywhere; per-block widths pay only where the patches are (blocks without
+    patches take no n_patch bits at all)."""
+    n_out, n_in, l = 100, 10, 2048
+    rng = np.random.default_rng(3)
+    M = wl.xor_network(n_out, n_in, 77)
+    wc = rng.integers(0, 1 << n_in, l).astype(np.uint32)
+    counts = np.zeros(l, dtype=np.uint16)
+    counts[512:640] = rng.integers(1, 8, 128)                  # one busy block of 128 slices
+    dp = np.concatenate([np.sort(rng.choice(n_out, c, replace=False)) for c in counts if c]).astype(np.uint16)
+    blob = sqnn.sqnn_pack_host(wl.network_rows(M), n_in, l, n_out, [wc], [counts], [dp])
+    whole, info_whole = sqnn.sqnn_store_host(blob, l)
+    blocked, info_blocked = sqnn.sqnn_store_host(blob, 128)
+    assert info_whole["bits_npatch"] == l * 3                   # max 7 -> 3 bits for every slice
+    assert info_blocked["bits_npatch"] == 128 * 3               # only the busy block stores counts
+    assert info_blocked["bits_npatch"] == orc.blocked_field_bits(counts, 128)["bits_npatch"]
+    assert info_blocked["bits_widths"] == 8 * 16
+    assert blocked.size < whole.size
+    for stored in (whole, blocked):
+        assert np.array_equal(sqnn.sqnn_load_host(stored), blob)
+    # damaged buffers: magic, truncated, a width byte that no longer matches the counts, trailing bytes
+    def bad(buf):
+        with pytest.raises(sqnn.SqnnError) as e:
+            sqnn.sqnn_load_host(buf)
+        assert e.value.status == sqnn.E_BAD_BLOB
+    b = blocked.copy(); b[0] ^= 1; bad(b)
+    bad(blocked[:-3])
+    bad(np.concatenate([blocked, np.zeros(4, np.uint8)]))
+    widths_at = 128 + 4 * n_out + (l * n_in + 7) // 8           # header, rows of M, seed stream
+    b = blocked.copy(); b[widths_at + 4] = 0; bad(b)            # the busy block's width set to 0: counts no longer add up
+    b = blocked.copy(); b[widths_at + 4] = 12; bad(b)           # a width no count needs

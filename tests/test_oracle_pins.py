@@ -569,3 +569,22 @@ def test_csr_relative_time():
     groups = nnz.reshape(-1, 32)
     assert t == pytest.approx(groups.max(axis=1).sum() / (nnz.sum() / 32))
     assert t > 1.05                                                   # Section 5.1: CSR rows vary
+
+
+def test_blocked_field_widths_that_can_hold_every_count():
+    """Section 5.2 as a stored format: hand-computed widths ceil(lg(max p + 1)) per block."""
+    p = np.array([0, 0, 1, 0, 3, 4, 0, 0, 0, 7, 8, 2, 1], dtype=np.uint16)
+    # blocks of 4: max (1, 4, 8, 1) -> widths (1, 3, 4, 1) over (4, 4, 4, 1) slices
+    assert orc.blocked_field_bits(p, 4) == {"bits_npatch": 4 * 1 + 4 * 3 + 4 * 4 + 1 * 1, "blocks": 4}
+    # one block: max 8 needs 4 bits (Eq. 1's ceil(lg 8) = 3 could not hold the value 8)
+    assert orc.blocked_field_bits(p, 100) == {"bits_npatch": 13 * 4, "blocks": 1}
+    # blocks of one slice: 0 -> 0 bits, 1 -> 1, 2..3 -> 2, 4..7 -> 3, 8 -> 4
+    assert orc.blocked_field_bits(p, 1)["bits_npatch"] == 0 + 0 + 1 + 0 + 2 + 3 + 0 + 0 + 0 + 3 + 4 + 2 + 1
+    assert orc.blocked_field_bits(np.zeros(9, np.uint16), 2) == {"bits_npatch": 0, "blocks": 5}
+    # never narrower than Eq. 1's literal width, and at most one bit wider per slice
+    rng = np.random.default_rng(5)
+    q = rng.poisson(2.0, 1000).astype(np.uint16)
+    for block in (1, 7, 128, 1000):
+        literal = orc.eq1_blocked(1000 * 80, 80, 16, q, block)["bits_npatch"]
+        real = orc.blocked_field_bits(q, block)["bits_npatch"]
+        assert literal <= real <= literal + 1000
