@@ -147,6 +147,17 @@ int sqnn_encode_host(const sqnn_xornet *net, const sqnn_planes *layer, uint32_t 
 int sqnn_encode_seeds_host(const sqnn_xornet *net, const sqnn_planes *layer, const uint32_t *const *wc,
                            void **blob, size_t *blob_bytes, sqnn_stats *stats);
 
+/* Algorithm 1 (Section 3.3) on one flattened plane for networks the device format does not take:
+ * up to 64 inputs and up to 4096 outputs (the sweeps of Section 3.3 run n_in up to 60 with the best
+ * n_out in the hundreds).  Host only; no blob is built.  rows[j] bit t = M[j][t] (64-bit rows);
+ * plane / mask: packed bits of mn positions as in sqnn_planes.  Outputs, allocated by the library
+ * (sqnn_free): wc[l] seeds, np[l] patch counts, dp[*n_dp] positions in slice order, ascending inside
+ * a slice, l = ceil(mn / n_out); *bpw_eq1 (may be NULL) = Eq. 1's bits per weight, taken literally.
+ * Same readings as sqnn_encode_host.  Errors: INVALID_ARG, NOMEM. */
+int sqnn_encode_wide_host(uint32_t n_out, uint32_t n_in, const uint64_t *rows, uint64_t mn,
+                          const uint64_t *plane, const uint64_t *mask,
+                          uint64_t **wc, uint16_t **np, uint16_t **dp, uint64_t *n_dp, double *bpw_eq1);
+
 /* Packs logical per-plane arrays (the three parts of the format, Section 3.2) into a blob:
  * wc[i][s] seed of slice s (bit t = w^c[t]), np[i][s] = n_patch, dp[i] = all d_patch entries of
  * plane i in slice order.  Arrays are host, length l, l and sum(np[i]).  Errors: INVALID_ARG

@@ -581,6 +581,93 @@ int sqnn_stats_blocked_host(const void *blob, size_t blob_bytes, uint64_t block_
 }
 
 // ---------------------------------------------------------------------------------------------
+// Algorithm 1 with 64-bit rows of M (host only)
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+inline uint32_t bit_at(const uint64_t *words, uint64_t p) { return (uint32_t)((words[p >> 6] >> (p & 63)) & 1); }
+
+// Seed of one slice (positions [p0, p1) of the plane) by the same incremental elimination as
+// encode_alg1, and the list of care positions the seed does not reproduce.
+inline uint64_t encode_alg1_wide(const uint64_t *rows, const uint64_t *plane, const uint64_t *mask,
+                                 uint64_t p0, uint64_t p1, std::vector<uint16_t> &wrong)
+{
+    uint64_t prow[64];
+    uint32_t pcol[64];
+    uint8_t prhs[64];
+    uint32_t npiv = 0;
+    for (uint64_t p = p0; p < p1; ++p) {
+        if (!bit_at(mask, p)) continue;
+        uint64_t a = rows[p - p0];
+        uint8_t b = (uint8_t)bit_at(plane, p);
+        for (uint32_t q = 0; q < npiv; ++q)
+            if ((a >> pcol[q]) & 1) { a ^= prow[q]; b ^= prhs[q]; }
+        if (a == 0) continue;
+        const uint32_t col = (uint32_t)__builtin_ctzll(a);
+        for (uint32_t q = 0; q < npiv; ++q)
+            if ((prow[q] >> col) & 1) { prow[q] ^= a; prhs[q] ^= b; }
+        prow[npiv] = a; prhs[npiv] = b; pcol[npiv] = col;
+        ++npiv;
+    }
+    uint64_t seed = 0;
+    for (uint32_t q = 0; q < npiv; ++q)
+        if (prhs[q]) seed |= (uint64_t)1 << pcol[q];
+    wrong.clear();
+    for (uint64_t p = p0; p < p1; ++p)
+        if (bit_at(mask, p) && (uint32_t)(__builtin_popcountll(rows[p - p0] & seed) & 1) != bit_at(plane, p))
+            wrong.push_back((uint16_t)(p - p0));
+    return seed;
+}
+
+}  // namespace
+
+int sqnn_encode_wide_host(uint32_t n_out, uint32_t n_in, const uint64_t *rows, uint64_t mn,
+                          const uint64_t *plane, const uint64_t *mask,
+                          uint64_t **wc, uint16_t **np, uint16_t **dp, uint64_t *n_dp, double *bpw_eq1)
+{
+    if (!rows || !plane || !mask || !wc || !np || !dp || !n_dp || n_out < 1 || n_out > 4096 || n_in < 1 || n_in > 64 ||
+        mn == 0 || mn > ((uint64_t)1 << 40))
+        return SQNN_E_INVALID_ARG;
+    if (n_in < 64)
+        for (uint32_t j = 0; j < n_out; ++j)
+            if (rows[j] >> n_in) return SQNN_E_INVALID_ARG;
+    try {
+        const uint64_t l = (mn + n_out - 1) / n_out;
+        std::vector<uint64_t> seeds(l);
+        std::vector<std::vector<uint16_t>> lists(l);
+#pragma omp parallel
+        {
+            std::vector<uint16_t> wrong;
+#pragma omp for schedule(dynamic, 256)
+            for (int64_t s = 0; s < (int64_t)l; ++s) {
+                const uint64_t p0 = (uint64_t)s * n_out, p1 = std::min(mn, p0 + n_out);
+                seeds[s] = encode_alg1_wide(rows, plane, mask, p0, p1, wrong);
+                lists[s] = wrong;
+            }
+        }
+        uint64_t total = 0, maxp = 0;
+        for (uint64_t s = 0; s < l; ++s) { total += lists[s].size(); maxp = std::max<uint64_t>(maxp, lists[s].size()); }
+        uint64_t *w = (uint64_t *)std::malloc(sizeof(uint64_t) * l);
+        uint16_t *c = (uint16_t *)std::malloc(sizeof(uint16_t) * l);
+        uint16_t *q = (uint16_t *)std::malloc(sizeof(uint16_t) * (total ? total : 1));
+        if (!w || !c || !q) { std::free(w); std::free(c); std::free(q); return SQNN_E_NOMEM; }
+        uint64_t at = 0;
+        for (uint64_t s = 0; s < l; ++s) {
+            w[s] = seeds[s];
+            c[s] = (uint16_t)lists[s].size();
+            for (uint16_t v : lists[s]) q[at++] = v;
+        }
+        *wc = w; *np = c; *dp = q; *n_dp = total;
+        if (bpw_eq1)
+            *bpw_eq1 = ((double)n_in / (double)n_out * (double)mn + (double)l * ceil_lg_u64(maxp) +
+                        (double)total * ceil_lg_u64(n_out)) / (double)mn;
+        return SQNN_OK;
+    } catch (const std::bad_alloc &) {
+        return SQNN_E_NOMEM;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
 // storage form
 // ---------------------------------------------------------------------------------------------
 namespace {

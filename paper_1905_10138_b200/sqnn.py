@@ -107,6 +107,8 @@ def lib():
         L.sqnn_stats_host.argtypes = [vp, sz, P(Stats)]
         L.sqnn_stats_blocked_host.argtypes = [vp, sz, u64, P(ctypes.c_double), P(u64)]
         L.sqnn_stats_blocked_host.restype = i32
+        L.sqnn_encode_wide_host.argtypes = [u32, u32, vp, u64, vp, vp, P(vp), P(vp), P(vp), P(u64), P(ctypes.c_double)]
+        L.sqnn_encode_wide_host.restype = i32
         L.sqnn_store_host.argtypes = [vp, sz, u64, P(vp), P(sz), P(StoreInfo)]
         L.sqnn_store_host.restype = i32
         L.sqnn_load_host.argtypes = [vp, sz, P(vp), P(sz)]
@@ -235,6 +237,23 @@ def sqnn_stats_blocked_host(blob: np.ndarray, block_slices: int) -> dict:
     _check(lib().sqnn_stats_blocked_host(_np_ptr(blob), blob.size, int(block_slices), ctypes.byref(bpw),
                                          ctypes.byref(bits)), "sqnn_stats_blocked_host")
     return {"bpw_eq1": bpw.value, "bits_npatch": int(bits.value)}
+
+
+def sqnn_encode_wide_host(rows64, n_in, mn, plane_words, mask_words):
+    """Algorithm 1 for networks of up to 64 inputs / 4096 outputs (host only, no blob).  rows64: uint64 [n_out].
+    Returns (wc uint64 [l], np uint16 [l], dp uint16 [sum np], bits per weight by Eq. 1)."""
+    rows64 = np.ascontiguousarray(rows64, dtype=np.uint64)
+    plane_words = np.ascontiguousarray(plane_words, dtype=np.uint64)
+    mask_words = np.ascontiguousarray(mask_words, dtype=np.uint64)
+    if plane_words.size != (mn + 63) // 64 or mask_words.size != plane_words.size:
+        raise ValueError("packed plane / mask size mismatch")
+    wc, np_, dp, n_dp, bpw = ctypes.c_void_p(), ctypes.c_void_p(), ctypes.c_void_p(), ctypes.c_uint64(), ctypes.c_double()
+    _check(lib().sqnn_encode_wide_host(int(rows64.size), int(n_in), _np_ptr(rows64), int(mn), _np_ptr(plane_words),
+                                       _np_ptr(mask_words), ctypes.byref(wc), ctypes.byref(np_), ctypes.byref(dp),
+                                       ctypes.byref(n_dp), ctypes.byref(bpw)), "sqnn_encode_wide_host")
+    l = (mn + rows64.size - 1) // rows64.size
+    return (_take(wc, 8 * l).view(np.uint64), _take(np_, 2 * l).view(np.uint16),
+            _take(dp, 2 * int(n_dp.value)).view(np.uint16), float(bpw.value))
 
 
 def sqnn_store_host(blob: np.ndarray, block_slices: int):

@@ -10,10 +10,11 @@
 Inputs follow the experiment of Section 3.3: every element is a don't-care with probability S,
 otherwise 0 or 1 with equal probability; M is drawn with equal probability per entry.  The paper's
 curves come without numbers except the point "about 0.83 at n_in = 20, S = 0.9, n_out near 200";
-the sweeps reproduce the shape of the curves around it.  The library takes n_in <= 32 and n_out <= 256,
-so the n_in sweep stops at 32 (the paper's runs to 60) and its lines flatten once the best n_out
-would lie beyond 256 (from n_in = 24 at S = 0.9, from n_in = 16 at S = 0.95).  Everything here is host work: encoder, Eq. 1
-accounting and the FIFO model are the library's C functions; this file only loops and prints.
+the sweeps reproduce the shape of the curves around it.  The device format takes n_in <= 32 and
+n_out <= 256; the figures go further (n_in to 60, best n_out in the hundreds), so the sweeps use the
+library's wide host encoder (64-bit rows of M, n_out up to 4096), which builds no blob.  Everything
+here is host work: encoder, Eq. 1 accounting and the FIFO model are the library's C functions; this
+file only loops and prints.
 """
 from __future__ import annotations
 
@@ -37,14 +38,17 @@ def encode_counts(count: int, prune_rate: float, n_out: int, n_in: int, seed: in
 
 def memory_reduction(count: int, prune_rate: float, n_out: int, n_in: int, seed: int = 1) -> dict:
     """One point of the first figure: the parts of Eq. 1 in bits per weight and 1 - 1/r."""
-    stats, n_patch, _ = encode_counts(count, prune_rate, n_out, n_in, seed)
+    bits, care = wl.synthetic_plane(count, prune_rate, seed)
+    M = wl.xor_network(n_out, n_in, seed + 1)
+    _, n_patch, _, bpw = sqnn.sqnn_encode_wide_host(wl.network_rows64(M), n_in, count, wl.pack_bits(bits),
+                                                    wl.pack_bits(care))
+    patches = int(n_patch.astype(np.int64).sum())
     lg_out = int(np.ceil(np.log2(n_out)))
-    bits_dp = stats["patches"][0] * lg_out / count
+    bits_dp = patches * lg_out / count
     bits_wc = n_in / n_out
-    bpw = stats["bpw_eq1"]
     return {"n_out": n_out, "n_in": n_in, "S": prune_rate, "bits_wc": bits_wc, "bits_dpatch": bits_dp,
             "bits_npatch": max(bpw - bits_wc - bits_dp, 0.0), "bits_per_weight": bpw, "reduction": 1.0 - bpw,
-            "patches_per_slice": stats["patches"][0] / stats["slices"]}
+            "patches_per_slice": patches / n_patch.size}
 
 
 def reduction_vs_n_out(count: int, prune_rate: float, n_in: int, n_outs, seed: int = 1):
@@ -54,9 +58,9 @@ def reduction_vs_n_out(count: int, prune_rate: float, n_in: int, n_outs, seed: i
 def best_reduction(count: int, prune_rate: float, n_in: int, seed: int = 1, step: float = 1.15):
     """Walks n_out upwards from n_in / (1 - S) / 2 until the reduction has fallen twice in a row (the
     figure's lines 'stop when the memory reduction begins to fall'); returns the best point."""
-    n_out = min(max(n_in + 1, int(n_in / (1.0 - prune_rate) / 2)), 200)
+    n_out = max(n_in + 1, int(n_in / (1.0 - prune_rate) / 2))
     best, falls = None, 0
-    while n_out <= 256 and falls < 2:
+    while n_out <= 4096 and falls < 2:
         p = memory_reduction(count, prune_rate, n_out, n_in, seed)
         if best is None or p["reduction"] > best["reduction"]:
             best, falls = p, 0
@@ -82,12 +86,6 @@ def fifo_table(count: int, prune_rate: float, n_out: int, n_in: int, banks=(1, 2
     return out
 
 
-def conv_as_matrix(c_out: int, c_in: int, kh: int, kw: int):
-    """A 4-D convolution tensor is flattened like any other weight tensor (Section 3.1): rows = output
-    channels, columns = c_in * kh * kw."""
-    return c_out, c_in * kh * kw
-
-
 def main():
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
     ap.add_argument("what", choices=["grace", "n_in", "prune", "fifo", "blocked", "conv"])
@@ -100,9 +98,9 @@ def main():
             print(f"{p['n_out']:6d}  {p['bits_wc']:.4f}  {p['bits_npatch']:.4f}   {p['bits_dpatch']:.4f}   {p['reduction']:.4f}")
     elif a.what == "n_in":
         print("best memory reduction over n_out\n  n_in   S=0.8 (n_out)   S=0.9 (n_out)   S=0.95 (n_out)")
-        for n_in in (12, 16, 20, 24, 28, 32):
+        for n_in in (12, 16, 20, 24, 28, 32, 40, 48, 60):
             cells = [best_reduction(a.count, s, n_in, a.seed) for s in (0.8, 0.9, 0.95)]
-            print(f"{n_in:6d}   " + "   ".join(f"{c['reduction']:.4f} ({c['n_out']:3d})" for c in cells))
+            print(f"{n_in:6d}   " + "   ".join(f"{c['reduction']:.4f} ({c['n_out']:4d})" for c in cells))
     elif a.what == "prune":
         print("n_in = 20\n    S    best reduction (n_out)   S - reduction")
         for s in (0.5, 0.6, 0.7, 0.8, 0.85, 0.9, 0.95):
@@ -129,10 +127,15 @@ def main():
             b = sqnn.sqnn_stats_blocked_host(blob, block)
             print(f"{block:8d}   {b['bits_npatch'] / count:.4f}                  {b['bpw_eq1']:.4f}")
     else:
-        m, n = conv_as_matrix(64, 64, 3, 3)
-        print(f"conv 64 x 64 x 3 x 3 as a {m} x {n} matrix, S = 0.9, M 100 x 10")
-        p = memory_reduction(m * n, 0.9, 100, 10, a.seed)
-        print(f"bits/weight {p['bits_per_weight']:.4f}, reduction {p['reduction']:.4f}, patches/slice {p['patches_per_slice']:.3f}")
+        print("ResNet-shaped 3 x 3 convolutions, 2-bit binary codes, 70 % pruned, M 40 x 12 (Section 3.1: a 4-D tensor\n"
+              "is flattened like any other)\n  c_out x c_in x 3 x 3   weights   patches/slice   bits/weight (Eq. 1)   stored")
+        for c in (16, 32, 64, 128):
+            layer = wl.make_conv_layer(c, c, 3, 3, seed=a.seed)
+            planes = np.concatenate([wl.pack_bits(layer.planes[i]) for i in range(layer.n_q)])
+            _, st = sqnn.sqnn_encode_host(wl.network_rows(layer.M), layer.n_in, layer.m, layer.n, layer.n_q, planes,
+                                          wl.pack_bits(layer.mask))
+            print(f"  {c:4d} x {c:4d} x 3 x 3   {layer.mn:8d}   {sum(st['patches']) / (layer.n_q * st['slices']):8.3f}        "
+                  f"{st['bpw_eq1']:.4f}              {st['bpw_actual']:.4f}")
 
 
 if __name__ == "__main__":

@@ -66,6 +66,16 @@ def _chunked(total: int, seed: int, draw) -> np.ndarray:
     return out
 
 
+def network_rows64(M: np.ndarray) -> np.ndarray:
+    """As network_rows for up to 64 inputs (uint64 rows)."""
+    n_out, n_in = M.shape
+    assert n_in <= 64
+    out = np.zeros(n_out, dtype=np.uint64)
+    for t in range(n_in):
+        out |= M[:, t].astype(np.uint64) << np.uint64(t)
+    return out
+
+
 def bernoulli_mask(shape, prune_rate: float, seed: int) -> np.ndarray:
     """1 = kept (care) with probability 1 - prune_rate, independently per weight."""
     keep = np.float32(1.0 - prune_rate)
@@ -208,6 +218,23 @@ def make_layer(cfg: int, m: int | None = None, n: int | None = None) -> Layer:
     return Layer(name=name, cfg=cfg, m=m, n=n, n_q=n_q, n_out=n_out, n_in=n_in, prune_rate=prune,
                  M=M, planes=planes, mask=mask, alpha=alpha, x_dtype=xdt, batches=batches,
                  seed_x=base + 4)
+
+
+def make_conv_layer(c_out: int, c_in: int, kh: int, kw: int, n_q: int = 2, prune: float = 0.70,
+                    n_out: int = 40, n_in: int = 12, seed: int = 1) -> Layer:
+    """A convolution layer in the shape of the paper's ResNet32 experiment (Section 4: 2-bit codes, 70 %
+    pruned): a 4-D weight tensor [c_out][c_in][kh][kw] ~ N(0, sqrt(2 / fan_in)), flattened in that order
+    (Section 3.1), i.e. a matrix of c_out rows and c_in * kh * kw columns; magnitude pruning over the layer,
+    greedy binary codes per output channel.  Its product is the layer applied to im2col patches."""
+    base = 7000 + 10 * int(seed)
+    fan_in = c_in * kh * kw
+    w4 = _rng(base + 1).standard_normal((c_out, c_in, kh, kw), dtype=np.float32) * np.float32(np.sqrt(2.0 / fan_in))
+    w = np.ascontiguousarray(w4).reshape(c_out, fan_in)
+    mask = magnitude_mask(w, 1.0 - prune)
+    planes, alpha = binary_code_quantize(w, mask, n_q)
+    return Layer(name=f"conv-{c_out}x{c_in}x{kh}x{kw}", cfg=7, m=c_out, n=fan_in, n_q=n_q, n_out=n_out, n_in=n_in,
+                 prune_rate=prune, M=xor_network(n_out, n_in, base + 3), planes=planes, mask=mask, alpha=alpha,
+                 x_dtype="bf16", batches=(1, 8, 64), seed_x=base + 4)
 
 
 SWEEP_PRUNE = (0.60, 0.80, 0.90, 0.95)

@@ -159,3 +159,25 @@ def test_tensor_core_path_rejects_what_it_cannot_take():
     with pytest.raises(sqnn.SqnnError) as e:                       # row pitch not a multiple of 16 bytes
         sqnn.sqnn_decode_matmul(dev.desc, dev.blob, dev.mask, dev.alpha, xb, y, ws, dev.status)
     assert e.value.status == sqnn.E_UNSUPPORTED
+
+
+def test_convolution_tensor_goes_through_decode_and_product():
+    """Section 3.1: a 4-D convolution tensor is flattened like any other weight tensor.  A ResNet-shaped 3 x 3
+    layer (2-bit codes, 70 % pruned) is encoded, decoded on the GPU bit for bit, and applied to batches of
+    im2col patch vectors (the product a convolution layer performs) on both product paths."""
+    import torch
+    layer = wl.make_conv_layer(128, 128, 3, 3)
+    arrays = H.oracle_encode(layer)
+    ref_bits = H.oracle_decode(layer, arrays)
+    blob, _ = H.blob_from_library(layer)
+    assert np.array_equal(blob, H.blob_from_oracle(layer, arrays))          # the two encoders agree byte for byte
+    dev = H.DeviceLayer(layer, blob)
+    got = dev.decode_bits()
+    for i in range(layer.n_q):
+        assert np.array_equal(got[i], wl.pack_bits(ref_bits[i]))
+    for batch, tol in ((1, TOL_F32), (8, TOL_F32), (64, TOL_BF16)):
+        x = layer.activations(batch)                                        # patch vectors of c_in * kh * kw values
+        y = dev.matmul(x, torch.bfloat16)
+        ref = orc.matmul(ref_bits, layer.mask, layer.alpha, x.astype(np.float64))
+        assert H.rel_err(y, ref) <= tol, (batch, H.rel_err(y, ref))
+    assert dev.status_value() == 0

@@ -51,5 +51,35 @@ def test_fifo_banks_and_csr_rows():
     assert light["n_fifo"][2] < 1.01                 # few patches: two banks already remove the stalls
 
 
-def test_conv_tensor_is_flattened_to_rows_of_output_channels():
-    assert sweeps.conv_as_matrix(64, 32, 3, 3) == (64, 288)
+def test_n_in_sweep_reaches_the_papers_range():
+    """Second figure of Section 3.3: the best reduction keeps growing with n_in up to 60, the best n_out moves
+    into the hundreds (beyond what the device format stores), and the gap to S shrinks."""
+    best = {n_in: sweeps.best_reduction(20000, 0.9, n_in) for n_in in (20, 40, 60)}
+    red = [best[k]["reduction"] for k in (20, 40, 60)]
+    assert red[0] < red[1] < red[2] < 0.9
+    assert best[40]["n_out"] > 256 and best[60]["n_out"] > best[40]["n_out"]
+    assert 0.9 - red[2] < 0.04
+
+
+def test_wide_host_encoder_matches_the_oracle_bit_for_bit():
+    """Algorithm 1 with 64-bit rows of M (n_in = 40, 60, 64; n_out beyond 256) against the oracle's."""
+    from oracle import oracle as orc
+    from paper_1905_10138_b200 import sqnn, workloads as wl
+    for n_out, n_in, count, S in ((300, 40, 9000, 0.9), (600, 60, 12000, 0.9), (333, 64, 7001, 0.8), (90, 33, 4000, 0.5)):
+        bits, care = wl.synthetic_plane(count, S, 5)
+        M = wl.xor_network(n_out, n_in, 6)
+        wc, np_, dp, bpw = sqnn.sqnn_encode_wide_host(wl.network_rows64(M), n_in, count, wl.pack_bits(bits), wl.pack_bits(care))
+        r_wc, r_np, r_dp = orc.encode_plane(M, bits, care)
+        assert np.array_equal(wc, r_wc) and np.array_equal(np_, r_np) and np.array_equal(dp, r_dp)
+        assert bpw == pytest.approx(orc.eq1(count, n_out, n_in, r_np)["bits_per_weight"], rel=1e-12)
+        out = orc.decode_plane(M, count, wc, np_, dp)
+        assert np.array_equal(out[care == 1], bits[care == 1])
+    with pytest.raises(sqnn.SqnnError):
+        sqnn.sqnn_encode_wide_host(np.zeros(8, np.uint64), 65, 64, np.zeros(1, np.uint64), np.zeros(1, np.uint64))
+
+
+def test_conv_layer_is_a_flattened_4d_tensor():
+    from paper_1905_10138_b200 import workloads as wl
+    layer = wl.make_conv_layer(16, 8, 3, 3)
+    assert (layer.m, layer.n, layer.n_q) == (16, 72, 2)
+    assert abs(layer.mask.mean() - 0.30) < 0.01 and layer.alpha.shape == (16, 2)
