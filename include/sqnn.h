@@ -328,6 +328,14 @@ int sqnn_search_seeds(const sqnn_xornet *net, uint64_t m, uint64_t n, uint32_t n
  * the decode kernel's output path allows on this GPU.  Errors: INVALID_ARG, CUDA. */
 int sqnn_store_probe(void *d_out, size_t bytes, uint32_t chunk_bytes, void *cuda_stream);
 
+/* For the library's own tests (the paper has no counterpart; not meant for applications).  Bit 0 of
+ * `flags` makes the loader role of the tensor-core kernel issue no loads, so that the bounded waits of
+ * the roles that consume its data run out: the kernel then reports 6 (= -SQNN_E_TIMEOUT) through
+ * d_status, frees its tensor memory and returns; Y is left incomplete.  wait_limit_cycles is the number
+ * of SM clock cycles such a wait may take (0 = the default, about two seconds).  Applies to calls made
+ * after it, process-wide. */
+void sqnn_set_debug_flags(uint32_t flags, uint64_t wait_limit_cycles);
+
 /* Scratch bytes sqnn_decode_matmul needs for this layer and batch (0 for batch <= 15). */
 size_t sqnn_workspace_bytes(const sqnn_desc *desc, uint32_t batch);
 

@@ -73,7 +73,7 @@ void orc_xor_network(int n_out, int n_in, const uint8_t *M, const uint8_t *wc, u
 /* in that column gets the pivot row added.  pivot_col[i] receives the pivot  */
 /* column of row i for i < rank.  Returns the rank of the coefficient part.   */
 /* ------------------------------------------------------------------------- */
-static int make_rref(uint8_t *a, int rows, int n_in, int *pivot_col)
+static int gauss_jordan_gf2(uint8_t *a, int rows, int n_in, int *pivot_col)
 {
     const int w = n_in + 1;
     int rank = 0;
@@ -101,7 +101,7 @@ static int make_rref(uint8_t *a, int rows, int n_in, int *pivot_col)
 }
 
 /* A reduced system is solvable iff no row reads 0 ... 0 | 1. */
-static int is_solved(const uint8_t *a, int rows, int n_in)
+static int is_consistent(const uint8_t *a, int rows, int n_in)
 {
     const int w = n_in + 1;
     for (int i = 0; i < rows; ++i) {
@@ -115,12 +115,13 @@ static int is_solved(const uint8_t *a, int rows, int n_in)
 /* ------------------------------------------------------------------------- */
 /* Algorithm 1 (patch searching) on one slice.                                */
 /*                                                                            */
-/* Care positions are tried in ascending order.  A care row is appended to    */
-/* mat; the whole of mat is brought to reduced row-echelon form; if the       */
-/* system became unsolvable the row is taken out again.  After the loop the   */
-/* kept system is solved with every free variable set to 0 (the reading that  */
-/* makes w^c unique), the network is evaluated on w^c, and the care positions */
-/* whose produced bit differs from the wanted bit form d_patch.               */
+/* Care positions are tried in ascending order.  The equation of a care bit   */
+/* joins the kept equations; a fresh copy of all kept equations is brought to */
+/* reduced row-echelon form; if the system turned inconsistent the equation   */
+/* is dropped again (that care bit will be a patch).  After the loop the kept */
+/* system is solved with every free variable set to 0 (the reading that makes */
+/* w^c unique), the network is evaluated on w^c, and the care positions whose */
+/* produced bit differs from the wanted bit form d_patch.                     */
 /*                                                                            */
 /* wq[j], care[j] in {0,1};  wc gets n_in bits;  dpatch needs room for n_out  */
 /* entries.  Returns n_patch, or -1 if memory ran out.                        */
@@ -129,37 +130,37 @@ int orc_encode_slice(int n_out, int n_in, const uint8_t *M, const uint8_t *wq,
                      const uint8_t *care, uint8_t *wc, uint16_t *dpatch)
 {
     const int w = n_in + 1;
-    uint8_t *mat = (uint8_t *)malloc((size_t)(n_out > 0 ? n_out : 1) * w);
+    uint8_t *kept = (uint8_t *)malloc((size_t)(n_out > 0 ? n_out : 1) * w);
     uint8_t *work = (uint8_t *)malloc((size_t)(n_out > 0 ? n_out : 1) * w);
     int *pivot_col = (int *)malloc(sizeof(int) * (size_t)(n_in > 0 ? n_in : 1));
     uint8_t *decoded = (uint8_t *)malloc((size_t)(n_out > 0 ? n_out : 1));
-    if (!mat || !work || !pivot_col || !decoded) {
-        free(mat); free(work); free(pivot_col); free(decoded);
+    if (!kept || !work || !pivot_col || !decoded) {
+        free(kept); free(work); free(pivot_col); free(decoded);
         return -1;
     }
     int rows = 0;
     for (int i = 0; i < n_out; ++i) {
         if (!care[i]) continue;                     /* only not-pruned bits */
-        for (int t = 0; t < n_in; ++t) mat[rows * w + t] = M[i * n_in + t];
-        mat[rows * w + n_in] = wq[i];
+        for (int t = 0; t < n_in; ++t) kept[rows * w + t] = M[i * n_in + t];
+        kept[rows * w + n_in] = wq[i];
         ++rows;
-        memcpy(work, mat, (size_t)rows * w);
-        make_rref(work, rows, n_in, pivot_col);
-        if (!is_solved(work, rows, n_in)) --rows;   /* remove the last row */
+        memcpy(work, kept, (size_t)rows * w);
+        gauss_jordan_gf2(work, rows, n_in, pivot_col);
+        if (!is_consistent(work, rows, n_in)) --rows;   /* this care bit cannot be met: drop its equation */
     }
     /* Solve the kept equations: pivot variables take the right-hand side of   */
     /* their row, free variables are 0.                                        */
     for (int t = 0; t < n_in; ++t) wc[t] = 0;
     if (rows > 0) {
-        memcpy(work, mat, (size_t)rows * w);
-        int rank = make_rref(work, rows, n_in, pivot_col);
+        memcpy(work, kept, (size_t)rows * w);
+        int rank = gauss_jordan_gf2(work, rows, n_in, pivot_col);
         for (int i = 0; i < rank; ++i) wc[pivot_col[i]] = work[i * w + n_in];
     }
     orc_xor_network(n_out, n_in, M, wc, decoded);
     int n_patch = 0;
     for (int i = 0; i < n_out; ++i)
         if (care[i] && decoded[i] != wq[i]) dpatch[n_patch++] = (uint16_t)i;
-    free(mat); free(work); free(pivot_col); free(decoded);
+    free(kept); free(work); free(pivot_col); free(decoded);
     return n_patch;
 }
 
@@ -233,7 +234,12 @@ int64_t orc_encode_plane(int64_t mn, int n_out, int n_in, const uint8_t *M,
         uint8_t *wq = (uint8_t *)calloc((size_t)n_out, 1);
         uint8_t *cr = (uint8_t *)calloc((size_t)n_out, 1);
         uint8_t wc[64];
-        if (!wq || !cr) { failed = 1; free(wq); free(cr); continue; }
+        if (!wq || !cr) {
+#pragma omp atomic write
+            failed = 1;
+            free(wq); free(cr);
+            continue;
+        }
         for (int j = 0; j < n_out; ++j) {
             int64_t p = s * n_out + j;
             if (p < mn) { wq[j] = bits[p]; cr[j] = care[p]; }
@@ -241,7 +247,11 @@ int64_t orc_encode_plane(int64_t mn, int n_out, int n_in, const uint8_t *M,
         int np = exhaustive
             ? orc_encode_slice_exhaustive(n_out, n_in, M, wq, cr, wc, all_dp + s * n_out)
             : orc_encode_slice(n_out, n_in, M, wq, cr, wc, all_dp + s * n_out);
-        if (np < 0) { failed = 1; np = 0; }
+        if (np < 0) {
+#pragma omp atomic write
+            failed = 1;
+            np = 0;
+        }
         uint64_t v = 0;
         for (int t = 0; t < n_in; ++t) v |= ((uint64_t)wc[t]) << t;
         wc_out[s] = v;

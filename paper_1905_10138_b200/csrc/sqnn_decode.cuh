@@ -89,6 +89,27 @@ template <int PENDING>
 SQNN_DEV void cp_async_wait_group() { asm volatile("cp.async.wait_group %0;\n" :: "n"(PENDING) : "memory"); }
 SQNN_DEV void cp_async_wait_all() { asm volatile("cp.async.wait_all;\n" ::: "memory"); }
 
+// Read-only global loads that stay where they are written: the compiler may not move a volatile asm
+// statement past another one, so a load issued ahead of time is not sunk down to its first use.
+SQNN_DEV uint32_t ldg_ahead(const uint32_t *p)
+{
+    uint32_t v;
+    asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(v) : "l"(p));
+    return v;
+}
+SQNN_DEV uint2 ldg_ahead(const uint2 *p)
+{
+    uint2 v;
+    asm volatile("ld.global.nc.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p));
+    return v;
+}
+SQNN_DEV uint4 ldg_ahead(const uint4 *p)
+{
+    uint4 v;
+    asm volatile("ld.global.nc.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+
 // Flips one bit of a shared-memory word (address given as a 32-bit shared address).
 SQNN_DEV void smem_flip(uint32_t region_sa, uint32_t bit)
 {
@@ -204,22 +225,22 @@ SQNN_DEV void fetch_seeds(const PlanePtrs &P, uint64_t tile, uint32_t lane, Tile
     using S = Shape<N_OUT, N_IN>;
     const uint32_t *w = P.wc + tile * (8 * S::n_in) + ((lane * S::SPAN) >> 5);
     if constexpr (S::ALIGNED && S::NSW == 4) {
-        const uint4 v = __ldg(reinterpret_cast<const uint4 *>(w));
+        const uint4 v = ldg_ahead(reinterpret_cast<const uint4 *>(w));
         s.raw[0] = v.x; s.raw[1] = v.y; s.raw[2] = v.z; s.raw[3] = v.w;
     } else if constexpr (S::ALIGNED && S::NSW == 2) {
-        const uint2 v = __ldg(reinterpret_cast<const uint2 *>(w));
+        const uint2 v = ldg_ahead(reinterpret_cast<const uint2 *>(w));
         s.raw[0] = v.x; s.raw[1] = v.y;
     } else {
 #pragma unroll
-        for (uint32_t k = 0; k < S::NRAW; ++k) s.raw[k] = __ldg(w + k);     // sections end with slack
+        for (uint32_t k = 0; k < S::NRAW; ++k) s.raw[k] = ldg_ahead(w + k);     // sections end with slack
     }
 }
 
 SQNN_DEV TileRun fetch_run(const PlanePtrs &P, uint64_t tile)
 {
     TileRun r;
-    r.base = __ldg(P.idx + tile);
-    r.end = __ldg(P.idx + tile + 1);
+    r.base = ldg_ahead(P.idx + tile);
+    r.end = ldg_ahead(P.idx + tile + 1);
     return r;
 }
 
@@ -236,7 +257,8 @@ SQNN_DEV void fetch_patches(const DecodeArgs &A, const PlanePtrs &P, TileRun &ru
 #pragma unroll
     for (uint32_t k = 0; k < PATCH_AHEAD; ++k) {
         const uint32_t aw = w0 + lane + 32 * k;
-        pw[k] = aw < wend ? __ldg(pp32 + aw) : 0u;
+        pw[k] = 0u;
+        if (aw < wend) pw[k] = ldg_ahead(pp32 + aw);
     }
 }
 

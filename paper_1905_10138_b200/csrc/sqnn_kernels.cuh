@@ -43,25 +43,26 @@ SQNN_DEV TilePos advance(TilePos p, uint32_t by, uint32_t live, uint32_t n_q)
 // works on its next tile (it waits for the copy only when it is about to overwrite the region).
 // Global loads run two tiles ahead: while tile t is expanded, the seeds and the patch offsets of
 // tile t + 2 and the patch entries of tile t + 1 (whose offsets arrived an iteration ago) are in
-// flight.  With a compile-time shape the lookup tables sit in shared memory in replicated form
-// (every lane of a load wavefront reads its own copy in its own banks), one block per SM.
+// flight.  REP: the lookup tables sit in shared memory in replicated form (every lane of a load
+// wavefront reads its own copy in its own banks); filling them takes a few microseconds, which pays
+// once a warp has several tiles to decode.  One block per SM.
 // SINK = true: XOR of all those words instead of storing them.
 constexpr uint32_t DECODE_BITS_THREADS = 768;
 template <int N_OUT, int N_IN>
-inline uint32_t decode_bits_table_words(const DecodeArgs &A)
+inline uint32_t decode_bits_table_words(const DecodeArgs &A, bool rep)
 {
-    if constexpr (N_OUT != 0) return table_words_replicated(N_OUT, N_IN);
+    if constexpr (N_OUT != 0) return rep ? table_words_replicated(N_OUT, N_IN) : A.tab_words;
     else return A.tab_words;
 }
 // ONE_PLANE: the layer has a single plane (its stream pointers are then kernel constants instead of
 // being looked up by a plane index in every step).
-template <int N_OUT, int N_IN, bool SINK, bool ONE_PLANE>
+template <int N_OUT, int N_IN, bool SINK, bool ONE_PLANE, bool REP>
 __global__ void __launch_bounds__(DECODE_BITS_THREADS, 1)
 k_decode_bits(DecodeArgs A, uint64_t *__restrict__ out)
 {
     extern __shared__ __align__(16) uint32_t smem[];
     uint32_t tab_words_s;
-    if constexpr (N_OUT != 0) {
+    if constexpr (N_OUT != 0 && REP) {
         tab_words_s = table_words_replicated(N_OUT, N_IN);       // filled below, after the first fetches are out
     } else {
         tables_request(A, smem);
@@ -111,8 +112,9 @@ k_decode_bits(DecodeArgs A, uint64_t *__restrict__ out)
         uint32_t wa[PATCH_AHEAD], wb[PATCH_AHEAD], wc[PATCH_AHEAD];
         if (pa.plane < A.n_q) { fetch_seeds<N_OUT, N_IN>(plane_of(pa), pa.tile, lane, sa); ra = fetch_run(plane_of(pa), pa.tile); }
         if (pb.plane < A.n_q) { fetch_seeds<N_OUT, N_IN>(plane_of(pb), pb.tile, lane, sb); rb = fetch_run(plane_of(pb), pb.tile); }
-        tables_replicate<entry_words_padded(N_OUT)>(A, smem);
+        if constexpr (REP) tables_replicate<entry_words_padded(N_OUT)>(A, smem);
         if (pa.plane < A.n_q) fetch_patches(A, plane_of(pa), ra, lane, wa);
+        if constexpr (!REP) cp_async_wait_all();
         __syncthreads();                                 // the tables are in place
         auto step = [&](TilePos &p0, TileSeeds<N_OUT, N_IN> &s0, TileRun &r0, uint32_t (&w0)[PATCH_AHEAD],
                         TilePos &p1, TileRun &r1, uint32_t (&w1)[PATCH_AHEAD],
@@ -120,7 +122,7 @@ k_decode_bits(DecodeArgs A, uint64_t *__restrict__ out)
             p2 = advance(p1, stride, live, A.n_q);
             if (p2.plane < A.n_q) { fetch_seeds<N_OUT, N_IN>(plane_of(p2), p2.tile, lane, s2); r2 = fetch_run(plane_of(p2), p2.tile); }
             if (p1.plane < A.n_q) fetch_patches(A, plane_of(p1), r1, lane, w1);
-            tile_expand<N_OUT, N_IN, !SINK, true>(s0, region, smem, lane);
+            tile_expand<N_OUT, N_IN, !SINK, REP>(s0, region, smem, lane);
             __syncwarp();
             tile_patch(A, plane_of(p0), r0, w0, region, 0u, S::TILE_BITS, lane);
             __syncwarp();
@@ -294,21 +296,27 @@ inline int launch_decode(const DecodeArgs &A, sqnn_out_mode mode, const uint64_t
 {
     size_t smem = 0;
     if (mode == SQNN_OUT_BITS || mode == SQNN_OUT_SINK) {
-        // one block per SM: the (replicated) tables and one region per warp
-        const size_t tab = (size_t)decode_bits_table_words<N_OUT, N_IN>(A) * 4, per_warp = (size_t)32 * A.W * 4;
+        // one block per SM: the tables and one region per warp.  The replicated tables are worth their
+        // fill only when a warp gets several tiles.
+        const uint64_t live = (A.words64 + 16ull * A.W - 1) / (16ull * A.W);
+        if (live * A.n_q >= (1ull << 31)) return SQNN_E_UNSUPPORTED;
+        const bool rep = N_OUT != 0 && live * A.n_q >= 3ull * (DECODE_BITS_THREADS / 32) * (uint64_t)sm_count();
+        const size_t tab = (size_t)decode_bits_table_words<N_OUT, N_IN>(A, rep) * 4, per_warp = (size_t)32 * A.W * 4;
         const size_t limit = 224 * 1024;
         if (tab + per_warp > limit) return SQNN_E_UNSUPPORTED;
         uint32_t warps = (uint32_t)((limit - tab) / per_warp);
         if (warps > DECODE_BITS_THREADS / 32) warps = DECODE_BITS_THREADS / 32;
         smem = tab + warps * per_warp;
-        const uint64_t live = (A.words64 + 16ull * A.W - 1) / (16ull * A.W);
-        if (live * A.n_q >= (1ull << 31)) return SQNN_E_UNSUPPORTED;
         const uint32_t grid = grid_for(live * A.n_q, warps, 1);
-#define SQNN_BITS_LAUNCH(SINKV, ONEV)                                                                    \
+#define SQNN_BITS_LAUNCH2(SINKV, ONEV, REPV)                                                             \
     do {                                                                                                 \
-        auto k = k_decode_bits<N_OUT, N_IN, SINKV, ONEV>;                                                \
+        auto k = k_decode_bits<N_OUT, N_IN, SINKV, ONEV, REPV>;                                          \
         if (prepare(k, smem)) return SQNN_E_CUDA;                                                        \
         k<<<grid, warps * 32, smem, st>>>(A, (uint64_t *)d_out);                                         \
+    } while (0)
+#define SQNN_BITS_LAUNCH(SINKV, ONEV)                                                                    \
+    do {                                                                                                 \
+        if (rep) SQNN_BITS_LAUNCH2(SINKV, ONEV, true); else SQNN_BITS_LAUNCH2(SINKV, ONEV, false);       \
     } while (0)
         if (mode == SQNN_OUT_BITS) {
             if (A.n_q == 1) SQNN_BITS_LAUNCH(false, true); else SQNN_BITS_LAUNCH(false, false);
@@ -316,6 +324,7 @@ inline int launch_decode(const DecodeArgs &A, sqnn_out_mode mode, const uint64_t
             if (cudaMemsetAsync(d_out, 0, 8, st) != cudaSuccess) return SQNN_E_CUDA;
             if (A.n_q == 1) SQNN_BITS_LAUNCH(true, true); else SQNN_BITS_LAUNCH(true, false);
         }
+#undef SQNN_BITS_LAUNCH2
 #undef SQNN_BITS_LAUNCH
     } else {
         const uint32_t warps = pick_warps(A, A.n_q + 1, &smem, 8, 200 * 1024);

@@ -1,77 +1,81 @@
 // K4: decryption fused with the product for batch >= 16 on the 5th-generation tensor cores.
 //
-//   Y[b][r] = sum_c W[r][c] X[b][c],   D (TMEM, fp32) [128 rows of W x N batch columns]
-//                                      += A (shared, bf16, K-major) [128 x 64] . B (shared) [N x 64]^T
+//   Y[b][r] = sum_i alpha[r][i] * sum_c s_i[r][c] X[b][c],      s_i = mask * (2 b_i - 1) in {-1, 0, +1}
 //
-// One CTA owns 128 rows of W and a range of columns.  Per 64-column step
-//   - the decode warps expand the weights of the step into the A stage (bf16, 128-byte rows,
-//     128-byte swizzle) -- the expanded weights exist only in shared memory;
-//   - one thread fetches the matching activations X[bc .. bc+N) x [64 columns] with TMA
-//     (every CTA fetches its own tile);
-//   - one thread issues tcgen05.mma (K = 16 each) that accumulate in tensor memory.
-// Column ranges of different CTAs are summed with fp32 atomics on Y (cleared beforehand).
+//   D (TMEM, fp32) [128 batch rows x 256 weight rows] += A (shared, bf16, K-major) [128 x 64] . B (shared) [256 x 64]^T
 //
-// The A stage.  Every plane gets its own tile of -1 / 0 / +1 (mask and sign only, four weights per
-// table read) and its own accumulator, and the epilogue forms sum_i alpha[r][i] * D_i: the weights
-// stay exact and the expansion is a few instructions per weight.  The batch is taken in passes whose
-// n_q accumulators fit the 512 columns of tensor memory.  (Only when the sign tiles of all planes do
-// not fit two pipeline stages of shared memory -- six planes and more -- one tile holds the rescaled
-// weights (+-alpha_1) + (+-alpha_2) + ... rounded to bf16 instead.)
+// One CTA owns 256 rows of W of ONE plane and a range of columns.  Per 64-column step
+//   - one thread fetches the activations X[bc .. bc+128) x [64 columns] with TMA into the A stage (every CTA
+//     fetches its own tile; rows past the batch are filled with zeros by the copy engine);
+//   - the decode warps expand the plane's sign tile -1 / 0 / +1 (mask and sign only, four weights per table
+//     read) into the B stage (bf16, 128-byte rows, 128-byte swizzle) -- the expanded weights exist only in
+//     shared memory;
+//   - one thread issues tcgen05.mma (M = 128, N = 256, K = 16 each) that accumulate in tensor memory.
+// A tcgen05.mma of M = 128 takes about as long whatever its N, so the weight rows sit on the N side at the
+// full N = 256.  The scale alpha[r][i] is applied to the accumulator in the epilogue, so the weights stay
+// exact (one tile of rescaled weights rounded to bf16 would not meet the tolerance: a row has only 2^n_q
+// distinct values and their rounding errors add up coherently).  Planes and column ranges of different CTAs
+// are summed with fp32 vector reductions on Y (cleared beforehand).  Batches beyond 128 are taken 128 rows
+// at a time, two accumulators (256 batch rows) per pass over the columns.
 //
-// Where the bits come from.  The planes have been decoded to packed bits in the workspace by the
-// tiled decode kernel (queued just before this one); 128 x 512-bit boxes of them (and of the mask)
-// are brought in by TMA when rows start on 16-byte boundaries, by coalesced loads otherwise.
+// Where the bits come from.  The planes have been decoded to packed bits in the workspace by the tiled
+// decode kernel (queued just before this one) and sit in L2.  A decode thread owns (row, half of a 64-column
+// step); when rows start on 16-byte boundaries it takes the bits of 256 columns with one 16-byte load per
+// vector (plane, mask) and trades words with its neighbour by shuffle, otherwise it reads word by word.
 //
-// Every wait on an mbarrier is bounded; a wait that gives up sets SQNN_E_TIMEOUT in the status
-// word and makes all roles leave their loops, so the kernel always returns.
+// Every wait on an mbarrier is bounded; a wait that gives up sets SQNN_E_TIMEOUT in the status word and
+// makes all roles leave their loops, so the kernel always frees its tensor memory and returns.
 #include "sqnn_launch.h"
 
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include <atomic>
 #include <mutex>
 
 namespace sqnn {
 
 namespace {
 
-constexpr uint32_t ROWS = 128;            // rows of W per CTA = MMA M
+constexpr uint32_t NROWS = 256;           // rows of W per CTA = MMA N
+constexpr uint32_t MB = 128;              // batch rows per accumulator = MMA M
 constexpr uint32_t KC = 64;               // columns per pipeline step
-constexpr uint32_t MACRO = 512;           // columns decoded to bits at a time
+constexpr uint32_t MACRO = 256;           // columns whose bits a decode thread takes at a time
 constexpr uint32_t STEPS_PER_MACRO = MACRO / KC;
-constexpr uint32_t RB_WORDS = MACRO / 32 + 1;   // words per row of the bit buffer (odd stride)
-// Copies of the 256-entry sign table, interleaved entry by entry: lane l reads copy l % LUT_COPIES, so two lanes
-// can only collide on a bank when they agree in l % LUT_COPIES.
-constexpr uint32_t LUT_COPIES = 8;
+constexpr uint32_t LUT_COPIES = 16;       // copies of the 256-entry sign table: lane l of a half-warp reads copy l
 constexpr uint32_t DEC_WARPS = 16;
 constexpr uint32_t DEC_THREADS = DEC_WARPS * 32;
 constexpr uint32_t THREADS = DEC_THREADS + 64;  // + TMA warp + MMA warp
-constexpr uint32_t A_STAGE_BYTES = ROWS * KC * 2;
+constexpr uint32_t B_STAGE_BYTES = NROWS * KC * 2;
+constexpr uint32_t A_TILE_BYTES = MB * KC * 2;
 constexpr uint32_t MAX_STAGES = 4;
 constexpr uint64_t WAIT_LIMIT_CYCLES = 4000000000ull;   // about 2 s at 2 GHz
 
+// Set by sqnn_set_debug_flags (for the library's own tests).
+std::atomic<uint32_t> g_debug_flags{0};
+std::atomic<uint64_t> g_debug_wait_cycles{0};
+
 struct MmaArgs {
-    DecodeArgs A;
+    const uint32_t *bits32;       // decoded planes in the workspace
+    uint64_t plane_words32;       // 32-bit words per plane in the workspace
     const uint32_t *mask32;
     uint64_t mask_words32;        // number of valid 32-bit mask words
     const float *alpha;
     float *y;
     int64_t ldy;
     uint64_t m, n;
-    uint32_t batch;               // total batch
-    uint32_t nbt;                 // batch columns per pass (multiple of 16, <= 512)
-    uint32_t tmem_cols;           // power of two >= nbt, >= 32
+    uint32_t n_q;
+    uint32_t batch;
+    uint32_t nchunks;             // accumulators (128 batch rows each) per pass: 1 or 2
     uint32_t stages;
-    uint32_t splits;              // CTAs per row tile
+    uint32_t splits;              // CTAs per (row tile, plane)
     uint32_t macros_per_split;
-    uint32_t b_stage_bytes;
-    const uint32_t *bits32;       // decoded planes in the workspace
-    uint64_t plane_words32;       // 32-bit words per plane in the workspace
-    uint32_t per_plane;           // 1: one sign tile and one accumulator per plane, scales in the epilogue
-    uint32_t tma_bits;            // 1: the bit buffer is filled by TMA (rows of the packed planes 16-byte aligned)
-    uint32_t rbp;                 // words per row of the bit buffer
-    uint32_t rb_bufs;             // bit buffers (2 with TMA)
+    uint32_t aligned;             // 1: rows of the packed vectors start on 16-byte boundaries
+    uint32_t vec_y;               // 1: Y rows allow 16-byte vector reductions
+    uint32_t skip_loads;          // test only: the TMA role issues no loads
+    uint64_t wait_limit;          // cycles a bounded wait may take
+    uint32_t *status;
 };
 
 // ---------------------------------------------------------------------------------------
@@ -101,14 +105,14 @@ SQNN_DEV bool mbar_try(uint64_t *bar, uint32_t parity)
     return ok != 0;
 }
 // Bounded wait.  Returns false if the wait was abandoned (limit reached or another role gave up).
-SQNN_DEV bool mbar_wait(uint64_t *bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t *status)
+SQNN_DEV bool mbar_wait(uint64_t *bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t *status, uint64_t limit)
 {
     if (mbar_try(bar, parity)) return true;
     const long long t0 = clock64();
     while (true) {
         if (mbar_try(bar, parity)) return true;
         if (*abort_flag) return false;
-        if ((uint64_t)(clock64() - t0) > WAIT_LIMIT_CYCLES) {
+        if ((uint64_t)(clock64() - t0) > limit) {
             *abort_flag = 1u;
             if (status) atomicMax(status, (uint32_t)(-SQNN_E_TIMEOUT));
             return false;
@@ -144,12 +148,22 @@ SQNN_DEV void mma_commit(uint64_t *bar)
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n"
                  :: "r"(smem_addr(bar)) : "memory");
 }
-SQNN_DEV void tmem_ld8(uint32_t taddr, uint32_t (&v)[8])
+// 32 consecutive accumulator columns of this thread's lane (one wait for the whole load).
+SQNN_DEV void tmem_ld32(uint32_t taddr, uint32_t (&v)[32])
 {
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];\n"
-                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                 "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                 "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n"
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+                   "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+                   "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+                   "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
                  : "r"(taddr) : "memory");
     asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+}
+SQNN_DEV void red_add_v4(float *gdst, float a, float b, float c, float d)
+{
+    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};\n" :: "l"(gdst), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
 }
 
 // Shared-memory matrix descriptor of a K-major bf16 tile with 128-byte rows and 128-byte
@@ -169,7 +183,7 @@ SQNN_DEV uint64_t smem_desc_sw128(uint32_t addr)
 // Instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = n.
 SQNN_DEV uint32_t instr_desc_bf16(uint32_t n)
 {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((n >> 3) << 17) | ((ROWS >> 4) << 24);
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((n >> 3) << 17) | ((MB >> 4) << 24);
 }
 
 // Barrier over the decode threads that also ORs a flag, so that all of them take the same exit.
@@ -181,63 +195,61 @@ SQNN_DEV bool decode_barrier_any(uint32_t flagged)
     return any != 0;
 }
 
-SQNN_DEV void tma_load_3d(void *sdst, const CUtensorMap *map, uint64_t *bar, int32_t x, int32_t y, int32_t z)
+// 32 bits of a packed vector starting at bit position p (words past `valid` read as zero).
+SQNN_DEV uint32_t bits_at(const uint32_t *__restrict__ src, uint64_t valid, uint64_t p)
 {
-    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];\n"
-                 :: "r"(smem_addr(sdst)), "l"(map), "r"(smem_addr(bar)), "r"(x), "r"(y), "r"(z) : "memory");
+    const uint64_t w = p >> 5;
+    const uint32_t sh = (uint32_t)(p & 31);
+    const uint32_t lo = w < valid ? __ldg(src + w) : 0u;
+    const uint32_t hi = (sh != 0 && w + 1 < valid) ? __ldg(src + w + 1) : 0u;
+    return __funnelshift_r(lo, hi, sh);
 }
 
 __global__ void __launch_bounds__(THREADS, 1)
-k_decode_mma(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ CUtensorMap pmap,
-             const __grid_constant__ CUtensorMap kmap, const MmaArgs M)
+k_decode_mma(const __grid_constant__ CUtensorMap xmap, const MmaArgs M)
 {
     extern __shared__ __align__(16) uint8_t smem_raw[];
-    const DecodeArgs &A = M.A;
-    const uint32_t n_items = A.n_q + 1;                                  // planes + mask
-    const uint32_t a_tiles = M.per_plane ? A.n_q : 1;                    // A tiles per stage
-    const uint32_t rbp = M.rbp;                                          // words per row of the bit buffer
     // carve shared memory (A / B stages need 1024-byte alignment for the 128-byte swizzle)
     uint8_t *base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    uint8_t *a_stages = base;
-    const uint32_t a_stage_bytes = a_tiles * A_STAGE_BYTES;
-    uint8_t *b_stages = a_stages + M.stages * a_stage_bytes;
-    uint32_t *rb = reinterpret_cast<uint32_t *>(b_stages + (size_t)M.stages * M.b_stage_bytes);   // [buf][item][row][rbp]
-    const uint32_t rb_buf_words = n_items * ROWS * rbp;
-    uint2 *lut256 = reinterpret_cast<uint2 *>(rb + M.rb_bufs * rb_buf_words);                          // [256][LUT_COPIES]
-    __nv_bfloat16 *lut = reinterpret_cast<__nv_bfloat16 *>(lut256 + 256 * LUT_COPIES);                             // [row][16]
-    float *alpha_s = reinterpret_cast<float *>(lut + ROWS * 16);         // [row][8]
-    uint64_t *bars = reinterpret_cast<uint64_t *>(alpha_s + ROWS * 8);
+    uint8_t *b_stages = base;                                               // [stage][256 rows][128 B]
+    const uint32_t a_stage_bytes = M.nchunks * A_TILE_BYTES;
+    uint8_t *a_stages = b_stages + M.stages * B_STAGE_BYTES;                 // [stage][chunk][128 rows][128 B]
+    uint2 *lut256 = reinterpret_cast<uint2 *>(a_stages + M.stages * a_stage_bytes);   // [256][LUT_COPIES]
+    float *alpha_s = reinterpret_cast<float *>(lut256 + 256 * LUT_COPIES);  // [256]
+    uint64_t *bars = reinterpret_cast<uint64_t *>(alpha_s + NROWS);
     uint64_t *full_a = bars, *full_b = bars + MAX_STAGES, *empty = bars + 2 * MAX_STAGES;
     uint64_t *accum = bars + 3 * MAX_STAGES;
-    uint64_t *bits_full = accum + 1, *bits_empty = accum + 3;
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(accum + 5);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(accum + 1);
     volatile uint32_t *abort_flag = tmem_slot + 1;
 
     const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const uint32_t row_tile = blockIdx.x / M.splits, split = blockIdx.x % M.splits;
-    const uint64_t r0 = (uint64_t)row_tile * ROWS;
+    // work item: (row tile, plane, column range)
+    const uint32_t split = blockIdx.x % M.splits;
+    const uint32_t plane = (blockIdx.x / M.splits) % M.n_q;
+    const uint32_t row_tile = blockIdx.x / (M.splits * M.n_q);
+    const uint64_t r0 = (uint64_t)row_tile * NROWS;
     const uint32_t total_macros = (uint32_t)((M.n + MACRO - 1) / MACRO);
     const uint32_t macro_begin = split * M.macros_per_split;
     const uint32_t macro_end = macro_begin + M.macros_per_split < total_macros ? macro_begin + M.macros_per_split : total_macros;
     const uint32_t total_steps = (uint32_t)((M.n + KC - 1) / KC);
+    const uint32_t step_begin = macro_begin * STEPS_PER_MACRO;
+    const uint32_t step_end = macro_end * STEPS_PER_MACRO < total_steps ? macro_end * STEPS_PER_MACRO : total_steps;
+    const uint32_t nsteps = step_end > step_begin ? step_end - step_begin : 0;
+    const uint32_t tmem_cols = M.nchunks * NROWS;                            // 256 or 512
 
     if (tid == 0) {
         for (uint32_t s = 0; s < MAX_STAGES; ++s) {
-            mbar_init(full_a + s, DEC_WARPS);        // one arrival per decode warp
-            mbar_init(full_b + s, 1);
+            mbar_init(full_b + s, DEC_WARPS);        // one arrival per decode warp
+            mbar_init(full_a + s, 1);
             mbar_init(empty + s, 1);
         }
         mbar_init(accum, 1);
-        for (uint32_t s = 0; s < 2; ++s) {
-            mbar_init(bits_full + s, 1);
-            mbar_init(bits_empty + s, DEC_WARPS);
-        }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
-    if (warp == DEC_WARPS + 1) tmem_alloc(tmem_slot, M.tmem_cols);
+    if (warp == DEC_WARPS + 1) tmem_alloc(tmem_slot, tmem_cols);
     if (tid < 256) {
-        // 4 weights of one plane at a time: index = mask nibble << 4 | bit nibble -> 4 bf16 of -1, 0, +1
+        // 4 weights at a time: index = mask nibble << 4 | bit nibble -> 4 bf16 of -1, 0, +1
         uint32_t h[4];
 #pragma unroll
         for (uint32_t k = 0; k < 4; ++k)
@@ -245,25 +257,9 @@ k_decode_mma(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ C
 #pragma unroll
         for (uint32_t c = 0; c < LUT_COPIES; ++c)
             lut256[tid * LUT_COPIES + c] = make_uint2(h[0] | (h[1] << 16), h[2] | (h[3] << 16));
-    }
-    if (tid < ROWS) {
-        // per-row scales and the table of all 2^n_q weight values (index bit i = plane i, bit 3 = mask)
-        const uint64_t r = r0 + tid;
-        float al[8];
-#pragma unroll
-        for (uint32_t i = 0; i < 8; ++i) {
-            al[i] = (i < A.n_q && r < M.m) ? __ldg(M.alpha + r * A.n_q + i) : 0.0f;
-            alpha_s[tid * 8 + i] = al[i];
-        }
-        for (uint32_t e = 0; e < 16; ++e) {
-            float s = 0.0f;
-            if (e & 8u) {
-#pragma unroll
-                for (uint32_t i = 0; i < 3; ++i)
-                    if (i < A.n_q) s = __fadd_rn(s, ((e >> i) & 1u) ? al[i] : -al[i]);
-            }
-            lut[tid * 16 + e] = __float2bfloat16_rn(s);
-        }
+    } else if (tid < 256 + NROWS) {
+        const uint64_t r = r0 + (tid - 256);
+        alpha_s[tid - 256] = r < M.m ? __ldg(M.alpha + r * M.n_q + plane) : 0.0f;
     }
     tc_fence_before();
     __syncthreads();
@@ -271,189 +267,145 @@ k_decode_mma(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ C
     const uint32_t tmem_base = *tmem_slot;
 
     uint32_t step_count = 0;                    // pipeline steps issued so far (all roles count alike)
-    uint32_t macro_count = 0;                   // bit-buffer fills so far
     uint32_t accum_parity = 0;
-    for (uint32_t bc = 0; bc < M.batch; bc += M.nbt) {
-        const uint32_t step_begin = macro_begin * STEPS_PER_MACRO;
-        uint32_t step_end = macro_end * STEPS_PER_MACRO;
-        if (step_end > total_steps) step_end = total_steps;
-        const uint32_t nsteps = step_end > step_begin ? step_end - step_begin : 0;
-        const uint32_t nmacros = macro_end > macro_begin ? macro_end - macro_begin : 0;
-
+    for (uint32_t bc = 0; bc < M.batch; bc += MB * M.nchunks) {
         if (warp < DEC_WARPS) {
             // ------------------------------ decode warps ------------------------------
-            uint32_t it = step_count, mi = macro_count;
-            for (uint32_t mc = macro_begin; mc < macro_end; ++mc, ++mi) {
-                const uint64_t c0 = (uint64_t)mc * MACRO;
-                const uint32_t cnt = (uint32_t)(M.n - c0 < MACRO ? M.n - c0 : MACRO);
-                const uint32_t buf = M.tma_bits ? (mi & 1u) : 0u;
-                const uint32_t *rbb = rb + buf * rb_buf_words;
-                bool stop = false;
-                // phase 1: the bit vectors of the 128 rows x MACRO columns into the bit buffer
-                if (M.tma_bits) {
-                    // the TMA thread fetches them as 128 x 64-byte boxes; wait for this buffer
-                    stop = !mbar_wait(bits_full + buf, (mi >> 1) & 1u, abort_flag, A.status);
-                } else {
-                    // planes exist as packed bits but rows are not 16-byte aligned: 16 consecutive
-                    // lanes copy the 16 words of one row segment, 32 rows per pass
-                    const uint32_t j = tid & 15;
+            // thread = (row, half): 32 columns of a 64-column step; two threads of a row are neighbours
+            const uint32_t row = tid >> 1, half = tid & 1, sw = row & 7;
+            const uint64_t r = r0 + row;
+            const bool live = r < M.m;
+            const uint32_t *src_b = M.bits32 + (uint64_t)plane * M.plane_words32;
+            const uint2 *lut_mine = lut256 + (lane & (LUT_COPIES - 1));
+            // shared addresses: this row inside stage 0, its four 16-byte chunks (swizzled), this lane's table copy
+            const uint32_t brow0 = smem_addr(b_stages) + (row >> 3) * 1024 + sw * 128;
+            uint32_t chunk_off[4];
 #pragma unroll
-                    for (uint32_t pass = 0; pass < ROWS / 32; ++pass) {
-                        const uint32_t rl = pass * 32 + (tid >> 4);
-                        const uint64_t rr = r0 + rl;
-                        const uint64_t p0 = rr * M.n + c0;
-                        const uint64_t w = (p0 >> 5) + j;
-                        const uint32_t sh = (uint32_t)(p0 & 31);
-                        const uint32_t lo = 32 * j;
-                        uint32_t keep = 0;                        // bits of this word that lie in [0, cnt)
-                        if (rr < M.m && lo < cnt) keep = lo + 32 > cnt ? (1u << (cnt - lo)) - 1u : 0xffffffffu;
-                        for (uint32_t item = 0; item <= A.n_q; ++item) {
-                            const uint32_t *src = item < A.n_q ? M.bits32 + (uint64_t)item * M.plane_words32 : M.mask32;
-                            const uint64_t valid = item < A.n_q ? M.plane_words32 : M.mask_words32;
-                            uint32_t v = 0;
-                            if (keep) {
-                                const uint32_t lo_w = w < valid ? __ldg(src + w) : 0u;
-                                const uint32_t hi_w = w + 1 < valid ? __ldg(src + w + 1) : 0u;
-                                v = __funnelshift_r(lo_w, hi_w, sh) & keep;
-                            }
-                            rb[(item * ROWS + rl) * rbp + j] = v;
-                        }
+            for (uint32_t j = 0; j < 4; ++j) chunk_off[j] = ((half * 4 + j) ^ sw) << 4;
+            const uint32_t lut_sa = smem_addr(lut_mine);
+            uint32_t stage = step_count % M.stages, use = step_count / M.stages;       // advanced step by step below
+            bool stop = false;
+            // bits of the current macro: aligned rows -> 4 words of this thread's 128 columns per vector
+            uint4 cur_m = make_uint4(0, 0, 0, 0), cur_b = make_uint4(0, 0, 0, 0);
+            auto fetch_macro = [&](uint32_t mc, uint4 &vm, uint4 &vb) {
+                vm = vb = make_uint4(0, 0, 0, 0);
+                const uint64_t c = (uint64_t)mc * MACRO + 128 * half;       // first column of this thread's 128
+                if (live && c < M.n) {
+                    const uint64_t w = (r * M.n + c) >> 5;                  // a multiple of 4
+                    if (w + 4 <= M.mask_words32) vm = ldg_ahead(reinterpret_cast<const uint4 *>(M.mask32 + w));
+                    else {
+                        vm.x = w < M.mask_words32 ? __ldg(M.mask32 + w) : 0u;
+                        vm.y = w + 1 < M.mask_words32 ? __ldg(M.mask32 + w + 1) : 0u;
+                        vm.z = w + 2 < M.mask_words32 ? __ldg(M.mask32 + w + 2) : 0u;
+                    }
+                    if (w + 4 <= M.plane_words32) vb = ldg_ahead(reinterpret_cast<const uint4 *>(src_b + w));
+                    else {
+                        vb.x = w < M.plane_words32 ? __ldg(src_b + w) : 0u;
+                        vb.y = w + 1 < M.plane_words32 ? __ldg(src_b + w + 1) : 0u;
+                        vb.z = w + 2 < M.plane_words32 ? __ldg(src_b + w + 2) : 0u;
                     }
                 }
-                if (!M.tma_bits) asm volatile("bar.sync 1, %0;\n" :: "n"(DEC_THREADS) : "memory");
-                // phase 2: steps of 64 columns; one thread per (row, 16 columns)
-                const uint32_t steps_here = stop ? 0u : (cnt + KC - 1) / KC;
-                const uint32_t row = tid >> 2, quarter = tid & 3, sw = row & 7;
-                const uint2 *lut_mine = lut256 + (lane & (LUT_COPIES - 1));
-                for (uint32_t ks = 0; ks < steps_here; ++ks, ++it) {
-                    const uint32_t stage = it % M.stages, use = it / M.stages;
+            };
+            if (M.aligned && macro_begin < macro_end) fetch_macro(macro_begin, cur_m, cur_b);
+            for (uint32_t mc = macro_begin; mc < macro_end && !stop; ++mc) {
+                uint4 nxt_m = make_uint4(0, 0, 0, 0), nxt_b = make_uint4(0, 0, 0, 0);
+                if (M.aligned && mc + 1 < macro_end) fetch_macro(mc + 1, nxt_m, nxt_b);
+                const uint32_t st_lo = mc * STEPS_PER_MACRO;
+#pragma unroll
+                for (uint32_t ks = 0; ks < STEPS_PER_MACRO; ++ks) {
+                    if (st_lo + ks >= step_end || stop) continue;           // the same in every thread
+                    // mask and sign word of this thread's 32 columns
+                    uint32_t mw, bw;
+                    if (M.aligned) {
+                        // words 2 ks and 2 ks + 1 of the macro: the lower four live in the half-0 thread,
+                        // the upper four in the half-1 thread; the neighbour hands over the one this thread lacks
+                        const uint32_t am[4] = {cur_m.x, cur_m.y, cur_m.z, cur_m.w};
+                        const uint32_t ab[4] = {cur_b.x, cur_b.y, cur_b.z, cur_b.w};
+                        const uint32_t m0 = am[(2 * ks) & 3u], m1 = am[(2 * ks + 1) & 3u];      // compile-time picks
+                        const uint32_t b0 = ab[(2 * ks) & 3u], b1 = ab[(2 * ks + 1) & 3u];
+                        const uint32_t gm = __shfl_xor_sync(0xffffffffu, half ? m0 : m1, 1);
+                        const uint32_t gb = __shfl_xor_sync(0xffffffffu, half ? b0 : b1, 1);
+                        const bool mine = half == (ks >> 1);                // the owner of words 2 ks, 2 ks + 1
+                        mw = mine ? (half ? m1 : m0) : gm;
+                        bw = mine ? (half ? b1 : b0) : gb;
+                    } else {
+                        const uint64_t c = (uint64_t)(st_lo + ks) * KC + 32 * half;
+                        mw = bw = 0;
+                        if (live && c < M.n) {
+                            mw = bits_at(M.mask32, M.mask_words32, r * M.n + c);
+                            bw = bits_at(src_b, M.plane_words32, r * M.n + c);
+                        }
+                    }
+                    // table indices (mask nibble << 4 | sign nibble) of the eight groups of four weights, one per
+                    // byte: byte j of `lo` for weights 8j .. 8j+3, byte j of `hi` for weights 8j+4 .. 8j+7
+                    const uint32_t lo = ((mw & 0x0f0f0f0fu) << 4) | (bw & 0x0f0f0f0fu);
+                    const uint32_t hi = (mw & 0xf0f0f0f0u) | ((bw >> 4) & 0x0f0f0f0fu);
+                    uint2 e[8];
+#pragma unroll
+                    for (uint32_t j = 0; j < 4; ++j) {
+                        const uint32_t a0 = lut_sa + ((lo >> (8 * j)) & 0xffu) * (LUT_COPIES * 8);
+                        const uint32_t a1 = lut_sa + ((hi >> (8 * j)) & 0xffu) * (LUT_COPIES * 8);
+                        asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(e[2 * j].x), "=r"(e[2 * j].y) : "r"(a0));
+                        asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(e[2 * j + 1].x), "=r"(e[2 * j + 1].y) : "r"(a1));
+                    }
                     // one lane per warp watches the barrier that frees the stage; the warp follows it
                     if (use > 0) {
                         uint32_t freed = 1;
-                        if (lane == 0) freed = mbar_wait(empty + stage, (use - 1) & 1u, abort_flag, A.status) ? 1u : 0u;
-                        if (!__shfl_sync(0xffffffffu, freed, 0)) break;
+                        if (lane == 0) freed = mbar_wait(empty + stage, (use - 1) & 1u, abort_flag, M.status, M.wait_limit) ? 1u : 0u;
+                        if (!__shfl_sync(0xffffffffu, freed, 0)) { stop = true; continue; }
                     }
-                    uint8_t *a_stage = a_stages + stage * a_stage_bytes;
-                    const uint32_t wi = ks * 2 + (quarter >> 1), sh16 = (quarter & 1) * 16;
-                    uint32_t mw = (rbb[(A.n_q * ROWS + row) * rbp + wi] >> sh16) & 0xffffu;
-                    if (M.per_plane) {
-                        // sign tiles, one per plane: -1 / 0 / +1 in bf16 (the scales are applied to
-                        // the accumulators afterwards), four weights per table read
-                        for (uint32_t i = 0; i < A.n_q; ++i) {
-                            const uint32_t bw = (rbb[(i * ROWS + row) * rbp + wi] >> sh16) & 0xffffu;
-                            uint2 e[4];
+                    const uint32_t brow = brow0 + stage * B_STAGE_BYTES;
 #pragma unroll
-                            for (uint32_t q = 0; q < 4; ++q)
-                                e[q] = lut_mine[((((mw >> (4 * q)) & 15u) << 4) | ((bw >> (4 * q)) & 15u)) * LUT_COPIES];
-                            uint8_t *arow = a_stage + i * A_STAGE_BYTES + row * 128;
-                            *reinterpret_cast<uint4 *>(arow + (((quarter * 2) ^ sw) << 4)) = make_uint4(e[0].x, e[0].y, e[1].x, e[1].y);
-                            *reinterpret_cast<uint4 *>(arow + (((quarter * 2 + 1) ^ sw) << 4)) = make_uint4(e[2].x, e[2].y, e[3].x, e[3].y);
-                        }
-                    } else {
-                        // one tile of rescaled weights: clear the thread's 32 bytes, then write only
-                        // the unpruned positions (most are zero)
-                        uint8_t *arow = a_stage + row * 128;
-#pragma unroll
-                        for (uint32_t q = 0; q < 2; ++q)
-                            *reinterpret_cast<uint4 *>(arow + (((quarter * 2 + q) ^ sw) << 4)) = make_uint4(0, 0, 0, 0);
-                        if (A.n_q <= 3) {
-                            uint32_t bw[3];
-#pragma unroll
-                            for (uint32_t i = 0; i < 3; ++i)
-                                bw[i] = i < A.n_q ? rbb[(i * ROWS + row) * rbp + wi] >> sh16 : 0u;
-                            const uint16_t *lr = reinterpret_cast<const uint16_t *>(lut) + row * 16;
-                            while (mw) {
-                                const uint32_t k = 31u - (uint32_t)__clz((int)mw);
-                                mw ^= 1u << k;
-                                const uint32_t e = 8u | ((bw[0] >> k) & 1u) | (((bw[1] >> k) & 1u) << 1) |
-                                                   (((bw[2] >> k) & 1u) << 2);
-                                *reinterpret_cast<uint16_t *>(arow + (((quarter * 2 + (k >> 3)) ^ sw) << 4) + (k & 7) * 2) = lr[e];
-                            }
-                        } else {
-                            while (mw) {
-                                const uint32_t k = 31u - (uint32_t)__clz((int)mw);
-                                mw ^= 1u << k;
-                                float sum = 0.0f;
-                                for (uint32_t i = 0; i < A.n_q; ++i) {
-                                    const float a = alpha_s[row * 8 + i];
-                                    sum = __fadd_rn(sum, ((rbb[(i * ROWS + row) * rbp + wi] >> (sh16 + k)) & 1u) ? a : -a);
-                                }
-                                *reinterpret_cast<uint16_t *>(arow + (((quarter * 2 + (k >> 3)) ^ sw) << 4) + (k & 7) * 2) =
-                                    __bfloat16_as_ushort(__float2bfloat16_rn(sum));
-                            }
-                        }
-                    }
+                    for (uint32_t j = 0; j < 4; ++j)                        // 8 weights = one 16-byte chunk
+                        asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};"
+                                     :: "r"(brow + chunk_off[j]), "r"(e[2 * j].x), "r"(e[2 * j].y), "r"(e[2 * j + 1].x), "r"(e[2 * j + 1].y) : "memory");
                     fence_async_smem();                 // generic-proxy writes -> visible to the tensor core
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(full_a + stage);     // the warp's 32 row segments are in place
+                    if (lane == 0) mbar_arrive(full_b + stage);     // the warp's 16 rows are in place
+                    if (++stage == M.stages) { stage = 0; ++use; }
                 }
-                __syncwarp();
-                if (M.tma_bits && lane == 0) mbar_arrive(bits_empty + buf);   // this warp is done with the buffer
-                if (decode_barrier_any(*abort_flag)) break;       // same decision in every decode thread
+                cur_m = nxt_m;
+                cur_b = nxt_b;
+                // a warp that gave up makes every decode thread leave at the same macro
+                if (decode_barrier_any(stop || *abort_flag)) stop = true;
             }
         } else if (warp == DEC_WARPS) {
             // ------------------------------ TMA producer ------------------------------
-            if (lane == 0) {
-                uint32_t it = step_count, mi = macro_count;
-                bool ok = true;
-                auto fetch_bits = [&](uint32_t mc, uint32_t mix) {
-                    const uint32_t buf = mix & 1u, useb = mix >> 1;
-                    if (useb > 0 && !mbar_wait(bits_empty + buf, (useb - 1) & 1u, abort_flag, A.status)) return false;
-                    uint8_t *dst = reinterpret_cast<uint8_t *>(rb + buf * rb_buf_words);
-                    mbar_expect_tx(bits_full + buf, n_items * ROWS * 64);
-                    for (uint32_t i = 0; i < A.n_q; ++i)
-                        tma_load_3d(dst + i * ROWS * 64, &pmap, bits_full + buf, (int32_t)(mc * (MACRO / 8)), (int32_t)r0, (int32_t)i);
-                    tma_load_2d(dst + A.n_q * ROWS * 64, &kmap, bits_full + buf, (int32_t)(mc * (MACRO / 8)), (int32_t)r0);
-                    return true;
-                };
-                if (M.tma_bits && nmacros) ok = fetch_bits(macro_begin, mi);
-                for (uint32_t mc = macro_begin; mc < macro_end && ok; ++mc, ++mi) {
-                    if (M.tma_bits && mc + 1 < macro_end) ok = fetch_bits(mc + 1, mi + 1);
-                    uint32_t st_lo = mc * STEPS_PER_MACRO, st_hi = st_lo + STEPS_PER_MACRO;
-                    if (st_hi > step_end) st_hi = step_end;
-                    for (uint32_t st = st_lo; st < st_hi && ok; ++st, ++it) {
-                        const uint32_t stage = it % M.stages, use = it / M.stages;
-                        if (use > 0 && !mbar_wait(empty + stage, (use - 1) & 1u, abort_flag, A.status)) { ok = false; break; }
-                        uint8_t *b_stage = b_stages + (size_t)stage * M.b_stage_bytes;
-                        mbar_expect_tx(full_b + stage, M.b_stage_bytes);
-                        for (uint32_t h = 0; h * 256 < M.nbt; ++h)
-                            tma_load_2d(b_stage + h * 256 * 128, &xmap, full_b + stage, (int32_t)(st * KC),
-                                        (int32_t)(bc + h * 256));
-                    }
+            if (lane == 0 && !M.skip_loads) {
+                uint32_t it = step_count;
+                for (uint32_t st = step_begin; st < step_end; ++st, ++it) {
+                    const uint32_t stage = it % M.stages, use = it / M.stages;
+                    if (use > 0 && !mbar_wait(empty + stage, (use - 1) & 1u, abort_flag, M.status, M.wait_limit)) break;
+                    uint8_t *a_stage = a_stages + (size_t)stage * a_stage_bytes;
+                    mbar_expect_tx(full_a + stage, a_stage_bytes);
+                    for (uint32_t c = 0; c < M.nchunks; ++c)
+                        tma_load_2d(a_stage + c * A_TILE_BYTES, &xmap, full_a + stage, (int32_t)(st * KC), (int32_t)(bc + c * MB));
                 }
             }
         } else {
             // ------------------------------ MMA issuer ------------------------------
             if (lane == 0) {
                 uint32_t it = step_count;
-                const uint32_t nmma = M.nbt > 256 ? 2 : 1;
-                const uint32_t ncols = M.nbt > 256 ? 256 : M.nbt;
-                const uint32_t idesc = instr_desc_bf16(ncols);
+                const uint32_t idesc = instr_desc_bf16(NROWS);
                 // descriptors differ only in the start-address field (units of 16 bytes): keep the
                 // constant part and add offsets, so that issuing an MMA costs a few instructions
                 const uint64_t a_desc0 = smem_desc_sw128(smem_addr(a_stages));
                 const uint64_t b_desc0 = smem_desc_sw128(smem_addr(b_stages));
-                const uint32_t a_stage16 = a_stage_bytes >> 4, b_stage16 = M.b_stage_bytes >> 4;
                 bool ok = true;
                 uint32_t acc = 0;                       // 0 for the very first MMA of every accumulator
                 for (uint32_t st = step_begin; st < step_end && ok; ++st, ++it) {
                     const uint32_t stage = it % M.stages, use = it / M.stages;
-                    ok = mbar_wait(full_a + stage, use & 1u, abort_flag, A.status) &&
-                         mbar_wait(full_b + stage, use & 1u, abort_flag, A.status);
+                    ok = mbar_wait(full_b + stage, use & 1u, abort_flag, M.status, M.wait_limit) &&
+                         mbar_wait(full_a + stage, use & 1u, abort_flag, M.status, M.wait_limit);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint64_t a_desc = a_desc0 + (uint64_t)(stage * a_stage16);
-                    const uint64_t b_desc = b_desc0 + (uint64_t)(stage * b_stage16);
-                    for (uint32_t t = 0; t < a_tiles; ++t) {
-                        for (uint32_t h = 0; h < nmma; ++h) {
-                            const uint32_t d = tmem_base + t * M.nbt + h * 256;
-                            const uint64_t ad = a_desc + (uint64_t)(t * (A_STAGE_BYTES >> 4));
-                            const uint64_t bd = b_desc + (uint64_t)(h * (256 * 128 >> 4));
-                            mma_bf16(d, ad, bd, idesc, acc);
+                    const uint64_t a_desc = a_desc0 + (uint64_t)(stage * (a_stage_bytes >> 4));
+                    const uint64_t b_desc = b_desc0 + (uint64_t)(stage * (B_STAGE_BYTES >> 4));
 #pragma unroll
-                            for (uint32_t k16 = 1; k16 < KC / 16; ++k16)
-                                mma_bf16(d, ad + 2 * k16, bd + 2 * k16, idesc, 1u);
-                        }
+                    for (uint32_t k16 = 0; k16 < KC / 16; ++k16) {
+                        for (uint32_t c = 0; c < M.nchunks; ++c)
+                            mma_bf16(tmem_base + c * NROWS, a_desc + (uint64_t)(c * (A_TILE_BYTES >> 4)) + 2 * k16,
+                                     b_desc + 2 * k16, idesc, (acc | k16) ? 1u : 0u);
                     }
                     acc = 1;
                     mma_commit(empty + stage);          // frees the stage when these MMAs are done
@@ -462,40 +414,39 @@ k_decode_mma(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ C
             }
         }
         step_count += nsteps;
-        macro_count += nmacros;
 
         // ------------------------------ epilogue ------------------------------
         if (warp < DEC_WARPS && nsteps) {
-            const bool ready = mbar_wait(accum, accum_parity, abort_flag, A.status);
+            const bool ready = mbar_wait(accum, accum_parity, abort_flag, M.status, M.wait_limit);
             if (__all_sync(0xffffffffu, ready)) {                  // tcgen05.ld needs the whole warp
                 tc_fence_after();
-                const uint32_t quad = warp & 3, part = warp >> 2;       // TMEM lane quarter, column class
-                const uint32_t rl = quad * 32 + lane;
-                const uint64_t r = r0 + rl;
-                for (uint32_t c = part * 8; c < M.nbt; c += 8 * (DEC_WARPS / 4)) {
-                    float out[8];
-                    if (M.per_plane) {
-                        // Y = sum over planes of alpha[r][i] * (sign tile i . X)
+                const uint32_t quad = warp & 3, part = warp >> 2;       // TMEM lane quarter (batch rows), column quarter
+                for (uint32_t c = 0; c < M.nchunks; ++c) {
+                    const uint32_t b = bc + c * MB + quad * 32 + lane;  // batch row of this thread
+                    if (bc + c * MB + quad * 32 >= M.batch) continue;   // the same in the whole warp
+#pragma unroll 1
+                    for (uint32_t q = 0; q < 2; ++q) {
+                        const uint32_t col = part * 64 + q * 32;        // first of 32 weight rows
+                        uint32_t v[32];
+                        tmem_ld32(tmem_base + ((quad * 32) << 16) + c * NROWS + col, v);
+                        if (b < M.batch) {
+                            float *dst = M.y + (int64_t)b * M.ldy + (int64_t)(r0 + col);
 #pragma unroll
-                        for (uint32_t e = 0; e < 8; ++e) out[e] = 0.0f;
-                        for (uint32_t i = 0; i < A.n_q; ++i) {
-                            uint32_t v[8];
-                            tmem_ld8(tmem_base + ((quad * 32) << 16) + i * M.nbt + c, v);
-                            const float a = alpha_s[rl * 8 + i];
-#pragma unroll
-                            for (uint32_t e = 0; e < 8; ++e) out[e] = fmaf(a, __uint_as_float(v[e]), out[e]);
+                            for (uint32_t e = 0; e < 32; e += 4) {
+                                const float o0 = alpha_s[col + e] * __uint_as_float(v[e]);
+                                const float o1 = alpha_s[col + e + 1] * __uint_as_float(v[e + 1]);
+                                const float o2 = alpha_s[col + e + 2] * __uint_as_float(v[e + 2]);
+                                const float o3 = alpha_s[col + e + 3] * __uint_as_float(v[e + 3]);
+                                if (M.vec_y && r0 + col + e + 4 <= M.m) {
+                                    red_add_v4(dst + e, o0, o1, o2, o3);
+                                } else {
+                                    if (r0 + col + e < M.m) atomicAdd(dst + e, o0);
+                                    if (r0 + col + e + 1 < M.m) atomicAdd(dst + e + 1, o1);
+                                    if (r0 + col + e + 2 < M.m) atomicAdd(dst + e + 2, o2);
+                                    if (r0 + col + e + 3 < M.m) atomicAdd(dst + e + 3, o3);
+                                }
+                            }
                         }
-                    } else {
-                        uint32_t v[8];
-                        tmem_ld8(tmem_base + ((quad * 32) << 16) + c, v);
-#pragma unroll
-                        for (uint32_t e = 0; e < 8; ++e) out[e] = __uint_as_float(v[e]);
-                    }
-                    if (r < M.m) {
-#pragma unroll
-                        for (uint32_t e = 0; e < 8; ++e)
-                            if (bc + c + e < M.batch)
-                                atomicAdd(M.y + (int64_t)(bc + c + e) * M.ldy + r, out[e]);
                     }
                 }
             }
@@ -505,7 +456,7 @@ k_decode_mma(const __grid_constant__ CUtensorMap xmap, const __grid_constant__ C
         __syncthreads();                       // accumulators are read before the next pass overwrites them
         tc_fence_after();
     }
-    if (warp == DEC_WARPS + 1) tmem_dealloc(tmem_base, M.tmem_cols);
+    if (warp == DEC_WARPS + 1) tmem_dealloc(tmem_base, tmem_cols);
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
@@ -544,84 +495,54 @@ int mma_dispatch(const sqnn_desc *desc, const DecodeArgs &A0, const uint64_t *d_
     if (!encode) return SQNN_E_CUDA;
 
     MmaArgs M;
-    M.A = A0;
+    M.bits32 = (const uint32_t *)d_workspace;
+    M.plane_words32 = A0.words64 * 2;
     M.mask32 = (const uint32_t *)d_mask;
-    M.mask_words32 = M.A.words64 * 2;
+    M.mask_words32 = A0.words64 * 2;
     M.alpha = d_alpha;
     M.y = d_y;
     M.ldy = ldy;
     M.m = desc->m;
     M.n = desc->n;
+    M.n_q = desc->n_q;
     M.batch = batch;
-    // One sign tile and one accumulator per plane, scales applied to the accumulators: the weights stay
-    // exact.  (One tile of rescaled weights rounded to bf16 is not an option: a row holds only 2^n_q
-    // distinct values, their rounding errors add up coherently, and the result misses the 1e-2 tolerance
-    // on wide layers.)  The n_q accumulators of a pass must fit the 512 columns of tensor memory, so the
-    // batch is taken in passes of at most 512 / n_q columns.
-    const uint32_t b16 = (batch + 15) / 16 * 16;
-    const uint32_t cap = (512u / M.A.n_q) / 16 * 16;
-    M.nbt = b16 < cap ? b16 : cap;
-    if (M.nbt > 256) M.nbt = 512;                       // one plane: two full 256-column MMAs per step
-    M.b_stage_bytes = M.nbt * 128;
-    M.bits32 = (const uint32_t *)d_workspace;
-    M.plane_words32 = M.A.words64 * 2;
-    M.per_plane = 1u;
-    // The bit buffer is filled by TMA when the rows of the packed planes start on 16-byte boundaries.
-    M.tma_bits = (desc->n % 128 == 0 && ((uintptr_t)d_mask & 15) == 0) ? 1u : 0u;
+    M.nchunks = batch > MB ? 2u : 1u;
+    M.status = A0.status;
+    // rows of the packed vectors start on 16-byte boundaries when n is a multiple of 128 (the workspace is
+    // 256-byte aligned and every plane in it starts on a multiple of 8 bytes: check that too)
+    M.aligned = (desc->n % 128 == 0 && ((uintptr_t)d_mask & 15) == 0 && (M.plane_words32 % 4 == 0 || desc->n_q == 1)) ? 1u : 0u;
+    M.vec_y = (((uintptr_t)d_y & 15) == 0 && ldy % 4 == 0) ? 1u : 0u;
+    const uint32_t dbg = g_debug_flags.load();
+    M.skip_loads = (dbg & 1u) ? 1u : 0u;
+    M.wait_limit = g_debug_wait_cycles.load() ? g_debug_wait_cycles.load() : WAIT_LIMIT_CYCLES;
+
     const size_t budget = 225 * 1024;        // + 1 KB of static shared memory stays within the 227 KB a block may have
-    size_t fixed = 0, per_stage = 0;
-    for (;;) {
-        M.rbp = M.tma_bits ? 16 : RB_WORDS;
-        M.rb_bufs = M.tma_bits ? 2 : 1;
-        const uint32_t a_tiles = M.per_plane ? M.A.n_q : 1;
-        M.tmem_cols = 32;
-        while (M.tmem_cols < a_tiles * M.nbt) M.tmem_cols *= 2;
-        fixed = (size_t)M.rb_bufs * (M.A.n_q + 1) * ROWS * M.rbp * 4 +
-                256 * 8 * LUT_COPIES + ROWS * 16 * 2 +
-                ROWS * 8 * 4 + (3 * MAX_STAGES + 5) * 8 + 16 + 1024;
-        per_stage = (size_t)a_tiles * A_STAGE_BYTES + M.b_stage_bytes;
-        if (fixed + 2 * per_stage <= budget) break;
-        if (M.tma_bits) { M.tma_bits = 0; continue; }          // single bit buffer
-        if (M.per_plane) { M.per_plane = 0; continue; }        // too many planes for two stages
-        break;
-    }
+    const size_t fixed = 256 * 8 * LUT_COPIES + NROWS * 4 + (3 * MAX_STAGES + 1) * 8 + 16 + 1024;
+    const size_t per_stage = B_STAGE_BYTES + (size_t)M.nchunks * A_TILE_BYTES;
     M.stages = MAX_STAGES;
     while (M.stages > 1 && fixed + (size_t)M.stages * per_stage > budget) --M.stages;
     const size_t smem = fixed + (size_t)M.stages * per_stage;
     if (smem > budget) return SQNN_E_UNSUPPORTED;
 
-    const uint32_t row_tiles = (uint32_t)((desc->m + ROWS - 1) / ROWS);
+    const uint64_t row_tiles = (desc->m + NROWS - 1) / NROWS;
     const uint32_t total_macros = (uint32_t)((desc->n + MACRO - 1) / MACRO);
-    uint32_t splits = (uint32_t)sm_count() / row_tiles;
+    const uint64_t items = row_tiles * desc->n_q;
+    uint32_t splits = items >= (uint64_t)sm_count() ? 1u : (uint32_t)((uint64_t)sm_count() / items);
     if (splits < 1) splits = 1;
     if (splits > total_macros) splits = total_macros;
     M.macros_per_split = (total_macros + splits - 1) / splits;
     M.splits = (total_macros + M.macros_per_split - 1) / M.macros_per_split;
+    if (items * M.splits > 0x7fffffffull) return SQNN_E_UNSUPPORTED;
 
-    CUtensorMap xmap, pmap, kmap;
+    CUtensorMap xmap;
     const cuuint64_t gdim[2] = {(cuuint64_t)desc->n, (cuuint64_t)batch};
     const cuuint64_t gstride[1] = {(cuuint64_t)ldx * 2};
-    const cuuint32_t box[2] = {KC, M.nbt > 256 ? 256u : M.nbt};
-    const cuuint32_t estride[3] = {1, 1, 1};
+    const cuuint32_t box[2] = {KC, MB};
+    const cuuint32_t estride[2] = {1, 1};
     if (encode(&xmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(d_x), gdim, gstride, box, estride,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return SQNN_E_CUDA;
-    pmap = xmap;
-    kmap = xmap;
-    if (M.tma_bits) {
-        // packed planes as bytes: [plane][row][n / 8], and the mask [row][n / 8]; boxes of 128 rows x 64 bytes
-        const cuuint64_t pdim[3] = {(cuuint64_t)(desc->n / 8), (cuuint64_t)desc->m, (cuuint64_t)M.A.n_q};
-        const cuuint64_t pstride[2] = {(cuuint64_t)(desc->n / 8), (cuuint64_t)(M.A.words64 * 8)};
-        const cuuint32_t pbox[3] = {MACRO / 8, ROWS, 1};
-        if (encode(&pmap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, d_workspace, pdim, pstride, pbox, estride,
-                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS ||
-            encode(&kmap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint64_t *>(d_mask), pdim, pstride, pbox, estride,
-                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-            return SQNN_E_CUDA;
-    }
 
     cudaError_t e = (ldy == (int64_t)desc->m)
         ? cudaMemsetAsync(d_y, 0, (size_t)batch * desc->m * sizeof(float), st)
@@ -631,11 +552,20 @@ int mma_dispatch(const sqnn_desc *desc, const DecodeArgs &A0, const uint64_t *d_
     // stage 1: the decode kernel writes the planes as packed bits into the workspace
     const int rc = decode_bits_dispatch(A0, d_workspace, st);
     if (rc != SQNN_OK) return rc;
-    k_decode_mma<<<row_tiles * M.splits, THREADS, smem, st>>>(xmap, pmap, kmap, M);
+    k_decode_mma<<<(uint32_t)(items * M.splits), THREADS, smem, st>>>(xmap, M);
     return cudaGetLastError() == cudaSuccess ? SQNN_OK : SQNN_E_CUDA;
 }
 
 }  // namespace sqnn
+
+// For the library's own tests: bit 0 of `flags` makes the tensor-core kernel's loader issue no loads, so that
+// the bounded waits of its consumers run out; wait_limit_cycles (0 = default, about 2 s) is the number of
+// clock cycles such a wait may take.  Affects calls made after it; not meant for applications.
+extern "C" void sqnn_set_debug_flags(uint32_t flags, uint64_t wait_limit_cycles)
+{
+    sqnn::g_debug_flags.store(flags);
+    sqnn::g_debug_wait_cycles.store(wait_limit_cycles);
+}
 
 // ---------------------------------------------------------------------------------------------
 // Tensor-core product for callers that must not allocate device memory.

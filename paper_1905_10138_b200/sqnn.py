@@ -123,6 +123,8 @@ def lib():
         L.sqnn_decode_matmul_static.restype = i32
         L.sqnn_store_probe.argtypes = [vp, sz, u32, vp]
         L.sqnn_store_probe.restype = i32
+        L.sqnn_set_debug_flags.argtypes = [u32, u64]
+        L.sqnn_set_debug_flags.restype = None
         L.sqnn_workspace_bytes.argtypes = [P(Desc), u32]
         L.sqnn_workspace_bytes.restype = sz
         L.sqnn_status_string.argtypes = [i32]
@@ -318,6 +320,11 @@ def sqnn_store_probe(d_out, chunk_bytes: int = 3200, stream=None):
     out of shared memory) and nothing else, to measure the write ceiling of that path."""
     _check(lib().sqnn_store_probe(_dev_ptr(d_out), d_out.numel() * d_out.element_size(), int(chunk_bytes),
                                   _stream_ptr(stream)), "sqnn_store_probe")
+
+
+def sqnn_set_debug_flags(flags: int, wait_limit_cycles: int = 0) -> None:
+    """Test knob: bit 0 = the tensor-core kernel's loader issues no loads; wait_limit_cycles bounds its waits."""
+    lib().sqnn_set_debug_flags(int(flags), int(wait_limit_cycles))
 
 
 def sqnn_workspace_bytes(desc: Desc, batch: int) -> int:
