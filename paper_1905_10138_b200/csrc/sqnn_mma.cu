@@ -10,7 +10,8 @@
 //   - the decode warps expand the plane's sign tile -1 / 0 / +1 (mask and sign only, four weights per table
 //     read) into the B stage (bf16, 128-byte rows, 128-byte swizzle) -- the expanded weights exist only in
 //     shared memory;
-//   - one thread issues tcgen05.mma (M = 128, N = 256, K = 16 each) that accumulate in tensor memory.
+//   - one thread issues tcgen05.mma (M = 128, N = 256, K = 16 each) that accumulate in tensor memory, never
+//     twice in a row into the same accumulator.
 // A tcgen05.mma of M = 128 takes about as long whatever its N, so the weight rows sit on the N side at the
 // full N = 256.  The scale alpha[r][i] is applied to the accumulator in the epilogue, so the weights stay
 // exact (one tile of rescaled weights rounded to bf16 would not meet the tolerance: a row has only 2^n_q
@@ -235,7 +236,11 @@ k_decode_mma(const __grid_constant__ CUtensorMap xmap, const MmaArgs M)
     const uint32_t step_begin = macro_begin * STEPS_PER_MACRO;
     const uint32_t step_end = macro_end * STEPS_PER_MACRO < total_steps ? macro_end * STEPS_PER_MACRO : total_steps;
     const uint32_t nsteps = step_end > step_begin ? step_end - step_begin : 0;
-    const uint32_t tmem_cols = M.nchunks * NROWS;                            // 256 or 512
+    // Two accumulators always: with two batch chunks one per chunk; with one chunk the K = 16 slices
+    // alternate between them and the epilogue adds them up.  (Measured: a tcgen05.mma that accumulates
+    // into the accumulator of the one before it is issued about 300 cycles after it at N = 256; when
+    // consecutive ones go to different accumulators the spacing is about 160 cycles.)
+    const uint32_t tmem_cols = 2 * NROWS;
 
     if (tid == 0) {
         for (uint32_t s = 0; s < MAX_STAGES; ++s) {
@@ -401,11 +406,18 @@ k_decode_mma(const __grid_constant__ CUtensorMap xmap, const MmaArgs M)
                     tc_fence_after();
                     const uint64_t a_desc = a_desc0 + (uint64_t)(stage * (a_stage_bytes >> 4));
                     const uint64_t b_desc = b_desc0 + (uint64_t)(stage * (B_STAGE_BYTES >> 4));
+                    if (M.nchunks == 2) {
 #pragma unroll
-                    for (uint32_t k16 = 0; k16 < KC / 16; ++k16) {
-                        for (uint32_t c = 0; c < M.nchunks; ++c)
-                            mma_bf16(tmem_base + c * NROWS, a_desc + (uint64_t)(c * (A_TILE_BYTES >> 4)) + 2 * k16,
-                                     b_desc + 2 * k16, idesc, (acc | k16) ? 1u : 0u);
+                        for (uint32_t k16 = 0; k16 < KC / 16; ++k16)
+#pragma unroll
+                            for (uint32_t c = 0; c < 2; ++c)
+                                mma_bf16(tmem_base + c * NROWS, a_desc + (uint64_t)(c * (A_TILE_BYTES >> 4)) + 2 * k16,
+                                         b_desc + 2 * k16, idesc, (acc | k16) ? 1u : 0u);
+                    } else {
+#pragma unroll
+                        for (uint32_t k16 = 0; k16 < KC / 16; ++k16)
+                            mma_bf16(tmem_base + (k16 & 1u) * NROWS, a_desc + 2 * k16, b_desc + 2 * k16, idesc,
+                                     (acc | (k16 >> 1)) ? 1u : 0u);
                     }
                     acc = 1;
                     mma_commit(empty + stage);          // frees the stage when these MMAs are done
@@ -429,6 +441,12 @@ k_decode_mma(const __grid_constant__ CUtensorMap xmap, const MmaArgs M)
                         const uint32_t col = part * 64 + q * 32;        // first of 32 weight rows
                         uint32_t v[32];
                         tmem_ld32(tmem_base + ((quad * 32) << 16) + c * NROWS + col, v);
+                        if (M.nchunks == 1) {                           // the second accumulator of the only chunk
+                            uint32_t u[32];
+                            tmem_ld32(tmem_base + ((quad * 32) << 16) + NROWS + col, u);
+#pragma unroll
+                            for (uint32_t e = 0; e < 32; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) + __uint_as_float(u[e]));
+                        }
                         if (b < M.batch) {
                             float *dst = M.y + (int64_t)b * M.ldy + (int64_t)(r0 + col);
 #pragma unroll

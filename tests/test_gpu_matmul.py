@@ -175,3 +175,32 @@ def test_convolution_tensor_goes_through_decode_and_product():
         ref = orc.matmul(ref_bits, layer.mask, layer.alpha, x.astype(np.float64))
         assert H.rel_err(y, ref) <= tol, (batch, H.rel_err(y, ref))
     assert dev.status_value() == 0
+
+
+def test_a_bounded_wait_that_runs_out_reports_a_timeout_and_the_kernel_returns():
+    """Every wait of the tensor-core kernel is bounded.  With the library's test knob its loader role issues no
+    loads and the limit is about a millisecond: the consumer's wait runs out, the kernel reports 6
+    (-SQNN_E_TIMEOUT) through the status word, frees its tensor memory and returns -- nothing traps, the
+    context stays usable, and the same call made normally right afterwards is correct."""
+    import torch
+    from paper_1905_10138_b200 import sqnn
+    layer = wl.make_layer(1)                                            # the smallest tensor-core case
+    layer.x_dtype = "bf16"
+    x = layer.activations(16)
+    ref = reference(layer, x)
+    dev = H.DeviceLayer(layer, H.blob_from_library(layer)[0])
+    d_x = torch.from_numpy(x).cuda().to(torch.bfloat16)
+    d_y = torch.zeros((16, layer.m), dtype=torch.float32, device="cuda")
+    ws = torch.empty(sqnn.sqnn_workspace_bytes(dev.desc, 16), dtype=torch.uint8, device="cuda")
+    try:
+        sqnn.sqnn_set_debug_flags(1, 2_000_000)                         # no loads; waits give up after ~1 ms
+        sqnn.sqnn_decode_matmul(dev.desc, dev.blob, dev.mask, dev.alpha, d_x, d_y, ws, dev.status)
+        torch.cuda.synchronize()                                        # returns: the kernel did not hang
+        assert dev.status_value() == -sqnn.E_TIMEOUT
+    finally:
+        sqnn.sqnn_set_debug_flags(0, 0)
+    dev.status.zero_()
+    sqnn.sqnn_decode_matmul(dev.desc, dev.blob, dev.mask, dev.alpha, d_x, d_y, ws, dev.status)
+    torch.cuda.synchronize()
+    assert dev.status_value() == 0
+    assert H.rel_err(d_y.cpu().numpy(), ref) <= 2e-4
