@@ -301,7 +301,9 @@ int sqnn_decode_matmul(const sqnn_desc *desc, const void *d_blob, const uint64_t
  *  - batch < 16 or F32 activations: SQNN_E_UNSUPPORTED (those paths need no scratch; use
  *    sqnn_decode_matmul).
  *  - The first call on each device looks up the array's device address (with that device
- *    current); make that first call before any stream capture begins.
+ *    current) and remembers it for the life of the process; make that first call before any
+ *    stream capture begins.  After a cudaDeviceReset the remembered address is stale: do not
+ *    reset a device this entry point has been used on.
  *  - All calls share the one array and it keeps whatever the last call left.  Nothing in it needs
  *    clearing (each call overwrites all it reads), but two calls whose kernels may run at the
  *    same time on one GPU -- different streams, or different threads -- race on it: serialise them.

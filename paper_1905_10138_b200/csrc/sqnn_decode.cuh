@@ -110,6 +110,16 @@ SQNN_DEV uint4 ldg_ahead(const uint4 *p)
     return v;
 }
 
+// Makes the warp wait here for a value loaded earlier (a volatile register move reads it).  Used before
+// new loads are issued: the few scoreboards a warp has are shared between loads, so a register whose
+// load finished long ago can otherwise end up waiting for loads issued just before its first use.
+SQNN_DEV uint32_t settle(uint32_t v)
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %1;" : "=r"(r) : "r"(v));
+    return r;
+}
+
 // Flips one bit of a shared-memory word (address given as a 32-bit shared address).
 SQNN_DEV void smem_flip(uint32_t region_sa, uint32_t bit)
 {
@@ -310,7 +320,8 @@ SQNN_DEV void tile_patch(const DecodeArgs &A, const PlanePtrs &P, const TileRun 
 #pragma unroll
             for (uint32_t k = 0; k < RB; ++k) {
                 const uint32_t aw = at + lane + 32 * k;
-                w[k] = aw < wend ? __ldg(pp32 + aw) : 0u;
+                w[k] = 0u;
+                if (aw < wend) w[k] = ldg_ahead(pp32 + aw);
             }
         };
         request(a0, cur);

@@ -119,9 +119,17 @@ k_decode_bits(DecodeArgs A, uint64_t *__restrict__ out)
         auto step = [&](TilePos &p0, TileSeeds<N_OUT, N_IN> &s0, TileRun &r0, uint32_t (&w0)[PATCH_AHEAD],
                         TilePos &p1, TileRun &r1, uint32_t (&w1)[PATCH_AHEAD],
                         TilePos &p2, TileSeeds<N_OUT, N_IN> &s2, TileRun &r2) {
+            // everything this step consumes was requested at least a step ago: take delivery of it now,
+            // before the loads of this step are issued
+#pragma unroll
+            for (uint32_t k = 0; k < S::NRAW; ++k) s0.raw[k] = settle(s0.raw[k]);
+#pragma unroll
+            for (uint32_t k = 0; k < PATCH_AHEAD; ++k) w0[k] = settle(w0[k]);
+            r0.base = settle(r0.base); r0.end = settle(r0.end);
+            r1.base = settle(r1.base); r1.end = settle(r1.end);
             p2 = advance(p1, stride, live, A.n_q);
-            if (p2.plane < A.n_q) { fetch_seeds<N_OUT, N_IN>(plane_of(p2), p2.tile, lane, s2); r2 = fetch_run(plane_of(p2), p2.tile); }
             if (p1.plane < A.n_q) fetch_patches(A, plane_of(p1), r1, lane, w1);
+            if (p2.plane < A.n_q) { fetch_seeds<N_OUT, N_IN>(plane_of(p2), p2.tile, lane, s2); r2 = fetch_run(plane_of(p2), p2.tile); }
             tile_expand<N_OUT, N_IN, !SINK, REP>(s0, region, smem, lane);
             __syncwarp();
             tile_patch(A, plane_of(p0), r0, w0, region, 0u, S::TILE_BITS, lane);
@@ -175,6 +183,13 @@ SQNN_DEV void stage_mask(uint32_t *mask_s, const uint32_t *__restrict__ mask32, 
 // of byte j of a 32-byte group of the tile's bit run, so a warp stores 512 contiguous bytes.
 // The tile's mask words arrive by cp.async while the tile is decoded; a lane keeps the scales
 // of the row it is in.  NQ = number of planes when it is 1, 2 or 3, 0 = any.
+// With one plane a weight is +-bf16(alpha) or 0, so four weights at a time come from a table indexed
+// by (mask nibble, bit nibble): a keep-mask and a sign-flip per weight, applied to the row's scale
+// with one logic operation per pair of weights (exact for any alpha; a pruned weight is +0).  The
+// table is kept in 8 copies, lane l reads copy l % 8, so that lookups of different entries do not
+// share banks.
+constexpr uint32_t BF16_LUT_COPIES = 8;
+constexpr uint32_t BF16_LUT_WORDS = 256 * BF16_LUT_COPIES * 4;
 template <int N_OUT, int N_IN, int NQ>
 __global__ void __launch_bounds__(256)
 k_decode_bf16(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__restrict__ alpha,
@@ -182,13 +197,29 @@ k_decode_bf16(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__
 {
     extern __shared__ __align__(16) uint32_t smem[];
     tables_request(A, smem);
+    uint4 *lut = reinterpret_cast<uint4 *>(smem + A.tab_words);          // [256][copies]: keep masks (x, y), sign flips (z, w)
+    if constexpr (NQ == 1) {
+        for (uint32_t e = threadIdx.x; e < 256; e += blockDim.x) {
+            uint32_t keep[4], flip[4];
+#pragma unroll
+            for (uint32_t k = 0; k < 4; ++k) {
+                const uint32_t m = (e >> (4 + k)) & 1u, b = (e >> k) & 1u;
+                keep[k] = m ? 0xffffu : 0u;
+                flip[k] = (m && !b) ? 0x8000u : 0u;
+            }
+            const uint4 v = make_uint4(keep[0] | (keep[1] << 16), keep[2] | (keep[3] << 16),
+                                       flip[0] | (flip[1] << 16), flip[2] | (flip[3] << 16));
+#pragma unroll
+            for (uint32_t c = 0; c < BF16_LUT_COPIES; ++c) lut[e * BF16_LUT_COPIES + c] = v;
+        }
+    }
     cp_async_wait_all();
     __syncthreads();
     const uint32_t W = words_per_lane<N_OUT>(A);
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     const uint32_t n_q = A.n_q;
     const uint32_t per_warp = (n_q + 1) * 32 * W;
-    uint32_t *region = smem + A.tab_words + warp * per_warp;
+    uint32_t *region = smem + A.tab_words + (NQ == 1 ? BF16_LUT_WORDS : 0u) + warp * per_warp;
     uint32_t *mask_s = region + n_q * 32 * W;
     const uint8_t *mask_s8 = reinterpret_cast<const uint8_t *>(mask_s);
     const uint32_t tile_bytes = 128 * W;                 // bytes of bits per tile and plane
@@ -212,7 +243,19 @@ k_decode_bf16(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__
             if (p >= A.mn) break;
             while (c >= n) { c -= n; ++r; }
             const uint32_t mk = mask_s8[t];
-            if (NQ > 0 && c + 8 <= n && p + 8 <= A.mn) {
+            if (NQ == 1 && c + 8 <= n && p + 8 <= A.mn) {
+                if (r != r_al) {
+                    al[0] = __ldg(alpha + r);
+                    r_al = r;
+                }
+                const uint32_t ab = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(al[0]));
+                const uint32_t ab2 = ab | (ab << 16);                    // the row's scale, twice
+                const uint32_t bt = reinterpret_cast<const uint8_t *>(region)[t];
+                const uint4 e0 = lut[((((mk & 15u) << 4) | (bt & 15u))) * BF16_LUT_COPIES + (lane & (BF16_LUT_COPIES - 1))];
+                const uint4 e1 = lut[((mk & 0xf0u) | (bt >> 4)) * BF16_LUT_COPIES + (lane & (BF16_LUT_COPIES - 1))];
+                *reinterpret_cast<uint4 *>(out + p) = make_uint4((ab2 & e0.x) ^ e0.z, (ab2 & e0.y) ^ e0.w,
+                                                                 (ab2 & e1.x) ^ e1.z, (ab2 & e1.y) ^ e1.w);
+            } else if (NQ > 0 && c + 8 <= n && p + 8 <= A.mn) {
                 if (r != r_al) {
 #pragma unroll
                     for (int i = 0; i < NR; ++i) al[i] = __ldg(alpha + r * n_q + i);
@@ -327,8 +370,10 @@ inline int launch_decode(const DecodeArgs &A, sqnn_out_mode mode, const uint64_t
 #undef SQNN_BITS_LAUNCH2
 #undef SQNN_BITS_LAUNCH
     } else {
-        const uint32_t warps = pick_warps(A, A.n_q + 1, &smem, 8, 200 * 1024);
+        const size_t lut_bytes = A.n_q == 1 ? (size_t)BF16_LUT_WORDS * 4 : 0;
+        const uint32_t warps = pick_warps(A, A.n_q + 1, &smem, 8, 200 * 1024 - lut_bytes);
         if (!warps) return SQNN_E_UNSUPPORTED;
+        smem += lut_bytes;
         const uint64_t live = (A.words64 * 2 + 32ull * A.W - 1) / (32ull * A.W);
         const uint32_t grid = grid_for(live, warps, 4);
 #define SQNN_BF16_LAUNCH(NQV)                                                                            \

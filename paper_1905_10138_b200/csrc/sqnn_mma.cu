@@ -313,6 +313,10 @@ k_decode_mma(const __grid_constant__ CUtensorMap xmap, const MmaArgs M)
             };
             if (M.aligned && macro_begin < macro_end) fetch_macro(macro_begin, cur_m, cur_b);
             for (uint32_t mc = macro_begin; mc < macro_end && !stop; ++mc) {
+                // take delivery of this macro's bits before the next macro's are requested (a warp's few
+                // scoreboards are shared between loads: a first use after the new request would wait for it)
+                cur_m.x = settle(cur_m.x); cur_m.y = settle(cur_m.y); cur_m.z = settle(cur_m.z); cur_m.w = settle(cur_m.w);
+                cur_b.x = settle(cur_b.x); cur_b.y = settle(cur_b.y); cur_b.z = settle(cur_b.z); cur_b.w = settle(cur_b.w);
                 uint4 nxt_m = make_uint4(0, 0, 0, 0), nxt_b = make_uint4(0, 0, 0, 0);
                 if (M.aligned && mc + 1 < macro_end) fetch_macro(mc + 1, nxt_m, nxt_b);
                 const uint32_t st_lo = mc * STEPS_PER_MACRO;
@@ -629,6 +633,7 @@ extern "C" int sqnn_decode_matmul_static(const sqnn_desc *desc, const void *d_bl
     if (!d_mask || !d_alpha || !d_x || !d_y || batch == 0) return SQNN_E_INVALID_ARG;
     if (ldx < (int64_t)desc->n || ldy < (int64_t)desc->m) return SQNN_E_INVALID_ARG;
     if (((uintptr_t)d_mask & 7) || ((uintptr_t)d_alpha & 3) || ((uintptr_t)d_y & 3)) return SQNN_E_INVALID_ARG;
+    if (x_dtype != SQNN_X_F32 && x_dtype != SQNN_X_BF16) return SQNN_E_INVALID_ARG;
     if (x_dtype != SQNN_X_BF16 || batch < 16 || batch > SQNN_MAX_BATCH || desc->n > (1ull << 30))
         return SQNN_E_UNSUPPORTED;
     if (sqnn::mma_workspace_bytes(desc, batch) > SQNN_STATIC_SCRATCH_BYTES) return SQNN_E_WORKSPACE;
