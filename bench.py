@@ -37,8 +37,10 @@ UNIT = "weights/s"
 WORKLOAD = "alexnet-fc6 4096x9216, n_q=1, M 100x10, S=0.91, bf16 activations, batch 1"
 # DRAM bytes (read + write) of one launch, from one ncu capture of each kernel as it stands now on exactly
 # these workloads (summaries under profiles/).  An entry is None while its kernel has changed since the
-# counters were taken.
-NCU_DRAM_BYTES_PER_LAUNCH = {"k_decode_gemv": None, "k_decode_bits": None}
+# counters were taken.  k_decode_gemv: 5.652 MB read, nothing written.  k_decode_bits at 2^30 weights,
+# 100x10, S = 0.90: 29.796 MB read + 74.684 MB written while the kernel ran; the other 59.5 MB of its
+# 134.2 MB of output were still in L2 when it ended and reach DRAM afterwards.
+NCU_DRAM_BYTES_PER_LAUNCH = {"k_decode_gemv": 5.652e6, "k_decode_bits": 104.48e6}
 LANES_PER_SM = 128
 SMS = 148
 
