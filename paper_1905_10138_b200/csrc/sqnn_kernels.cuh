@@ -190,8 +190,9 @@ SQNN_DEV void stage_mask(uint32_t *mask_s, const uint32_t *__restrict__ mask32, 
 // share banks.
 constexpr uint32_t BF16_LUT_COPIES = 8;
 constexpr uint32_t BF16_LUT_WORDS = 256 * BF16_LUT_COPIES * 4;
+constexpr uint32_t BF16_THREADS = 768;                   // one block per SM, as many warps as shared memory holds
 template <int N_OUT, int N_IN, int NQ>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(BF16_THREADS, 1)
 k_decode_bf16(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__restrict__ alpha,
               uint64_t n, __nv_bfloat16 *__restrict__ out)
 {
@@ -234,28 +235,36 @@ k_decode_bf16(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__
             decode_warp_tile<N_OUT, N_IN>(A, i, tile, region + i * 32 * W, smem, lane);
         cp_async_wait_all();
         __syncwarp();
-        uint64_t p = p_tile + 8ull * lane;               // first weight of this lane's group
-        uint64_t r = p / n;
-        uint64_t c = p - r * n;
+        // byte t of the tile's bit run holds the weights p_tile + 8 t ..; bytes below nfull lie wholly inside
+        // the plane, bytes below nbytes hold at least one of its weights
+        const uint64_t left = A.mn - p_tile;
+        const uint32_t nbytes = left >= 8ull * tile_bytes ? tile_bytes : (uint32_t)((left + 7) / 8);
+        const uint32_t nfull = left >= 8ull * tile_bytes ? tile_bytes : (uint32_t)(left / 8);
+        __nv_bfloat16 *out_t = out + p_tile;
+        const uint8_t *bits_s8 = reinterpret_cast<const uint8_t *>(region);
+        const uint32_t lut_lane = lane & (BF16_LUT_COPIES - 1);
+        uint64_t r = (p_tile + 8ull * lane) / n;         // row and column of the lane's first weight
+        uint64_t c = (p_tile + 8ull * lane) - r * n;
         float al[NR];
+        uint32_t ab2 = 0;                                // bf16(alpha) of the row, twice (one plane)
         uint64_t r_al = ~0ull;
-        for (uint32_t t = lane; t < tile_bytes; t += 32, p += 256, c += 256) {
-            if (p >= A.mn) break;
+        for (uint32_t t = lane; t < nbytes; t += 32, c += 256) {
             while (c >= n) { c -= n; ++r; }
             const uint32_t mk = mask_s8[t];
-            if (NQ == 1 && c + 8 <= n && p + 8 <= A.mn) {
+            const uint64_t p = p_tile + 8ull * t;        // (the slow path's)
+            if (NQ == 1 && c + 8 <= n && t < nfull) {
                 if (r != r_al) {
                     al[0] = __ldg(alpha + r);
                     r_al = r;
+                    const uint32_t ab = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(al[0]));
+                    ab2 = ab | (ab << 16);
                 }
-                const uint32_t ab = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(al[0]));
-                const uint32_t ab2 = ab | (ab << 16);                    // the row's scale, twice
-                const uint32_t bt = reinterpret_cast<const uint8_t *>(region)[t];
-                const uint4 e0 = lut[((((mk & 15u) << 4) | (bt & 15u))) * BF16_LUT_COPIES + (lane & (BF16_LUT_COPIES - 1))];
-                const uint4 e1 = lut[((mk & 0xf0u) | (bt >> 4)) * BF16_LUT_COPIES + (lane & (BF16_LUT_COPIES - 1))];
-                *reinterpret_cast<uint4 *>(out + p) = make_uint4((ab2 & e0.x) ^ e0.z, (ab2 & e0.y) ^ e0.w,
-                                                                 (ab2 & e1.x) ^ e1.z, (ab2 & e1.y) ^ e1.w);
-            } else if (NQ > 0 && c + 8 <= n && p + 8 <= A.mn) {
+                const uint32_t bt = bits_s8[t];
+                const uint4 e0 = lut[((((mk & 15u) << 4) | (bt & 15u))) * BF16_LUT_COPIES + lut_lane];
+                const uint4 e1 = lut[((mk & 0xf0u) | (bt >> 4)) * BF16_LUT_COPIES + lut_lane];
+                *reinterpret_cast<uint4 *>(out_t + 8 * t) = make_uint4((ab2 & e0.x) ^ e0.z, (ab2 & e0.y) ^ e0.w,
+                                                                       (ab2 & e1.x) ^ e1.z, (ab2 & e1.y) ^ e1.w);
+            } else if (NQ > 0 && c + 8 <= n && t < nfull) {
                 if (r != r_al) {
 #pragma unroll
                     for (int i = 0; i < NR; ++i) al[i] = __ldg(alpha + r * n_q + i);
@@ -282,7 +291,7 @@ k_decode_bf16(DecodeArgs A, const uint32_t *__restrict__ mask32, const float *__
                     const __nv_bfloat162 pk = __floats2bfloat162_rn(two[0], two[1]);
                     w[h] = *reinterpret_cast<const uint32_t *>(&pk);
                 }
-                *reinterpret_cast<uint4 *>(out + p) = make_uint4(w[0], w[1], w[2], w[3]);
+                *reinterpret_cast<uint4 *>(out_t + 8 * t) = make_uint4(w[0], w[1], w[2], w[3]);
             } else {
                 uint64_t rr = r, cc = c;
                 for (uint32_t k = 0; k < 8 && p + k < A.mn; ++k) {
@@ -371,11 +380,11 @@ inline int launch_decode(const DecodeArgs &A, sqnn_out_mode mode, const uint64_t
 #undef SQNN_BITS_LAUNCH
     } else {
         const size_t lut_bytes = A.n_q == 1 ? (size_t)BF16_LUT_WORDS * 4 : 0;
-        const uint32_t warps = pick_warps(A, A.n_q + 1, &smem, 8, 200 * 1024 - lut_bytes);
+        const uint32_t warps = pick_warps(A, A.n_q + 1, &smem, BF16_THREADS / 32, 224 * 1024 - lut_bytes);
         if (!warps) return SQNN_E_UNSUPPORTED;
         smem += lut_bytes;
         const uint64_t live = (A.words64 * 2 + 32ull * A.W - 1) / (32ull * A.W);
-        const uint32_t grid = grid_for(live, warps, 4);
+        const uint32_t grid = grid_for(live, warps, 1);
 #define SQNN_BF16_LAUNCH(NQV)                                                                            \
     do {                                                                                                 \
         auto k = k_decode_bf16<N_OUT, N_IN, NQV>;                                                        \
