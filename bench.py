@@ -82,7 +82,21 @@ class ClockSampler:
         self._thread = None
         self.error = None
 
+    def _sample(self):
+        self.sm.append(float(self._nvml.nvmlDeviceGetClockInfo(self._h, self._nvml.NVML_CLOCK_SM)))
+        self.bits |= int(self._nvml.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+
     def _run(self):
+        try:
+            while not self._stop.is_set():
+                self._sample()
+                time.sleep(self.period)
+        except Exception as e:                      # noqa: BLE001 - report, never fail the benchmark
+            self.error = repr(e)
+
+    def start(self):
+        """Opens NVML and takes the first sample before returning, so that even a timed region of a few
+        milliseconds has samples from inside it."""
         try:
             import pynvml
             pynvml.nvmlInit()
@@ -92,17 +106,12 @@ class ClockSampler:
                 ids = [v.strip() for v in visible.split(",") if v.strip()]
                 if self.index < len(ids) and ids[self.index].isdigit():
                     phys = int(ids[self.index])
-            h = pynvml.nvmlDeviceGetHandleByIndex(phys)
-            self.smax = float(pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM))
-            while not self._stop.is_set():
-                self.sm.append(float(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM)))
-                self.bits |= int(pynvml.nvmlDeviceGetCurrentClocksThrottleReasons(h))
-                time.sleep(self.period)
-            pynvml.nvmlShutdown()
-        except Exception as e:                      # noqa: BLE001 - report, never fail the benchmark
+            self._nvml = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(phys)
+            self.smax = float(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception as e:                      # noqa: BLE001
             self.error = repr(e)
-
-    def start(self):
+            return
         self._thread = threading.Thread(target=self._run, daemon=True)
         self._thread.start()
 
@@ -110,6 +119,11 @@ class ClockSampler:
         self._stop.set()
         if self._thread is not None:
             self._thread.join(timeout=2.0)
+            try:
+                self._sample()                      # one more, taken as the region ends
+                self._nvml.nvmlShutdown()
+            except Exception as e:                  # noqa: BLE001
+                self.error = self.error or repr(e)
         reasons = sorted(k for k, bit in self.REASONS.items() if self.bits & bit)
         if self.error:
             reasons.append("nvml: " + self.error)
@@ -529,7 +543,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--quick", action="store_true", help="headline line only (no extra reference points)")
