@@ -36,6 +36,13 @@
  *    kernel had to skip a malformed patch entry (1: position outside its tile, 2: a tile's
  *    offsets point past the end of the patch section) or gave up a bounded wait
  *    (6 = -SQNN_E_TIMEOUT); the caller zeroes it.  Kernels never trap.
+ *  - Checked mode: with the environment variable SQNN_DEBUG_CHECKS=1 (read once, at the first
+ *    device call) every device entry point, after queueing its work, waits for the stream,
+ *    and returns SQNN_E_CUDA if a CUDA error surfaced, SQNN_E_TIMEOUT if *d_status is 6 and
+ *    SQNN_E_BAD_BLOB if it is any other non-zero code, instead of SQNN_OK.  Meant for
+ *    debugging; it serialises the stream.
+ *  - Every device entry point is an NVTX range named after the function (domain "sqnn"), visible
+ *    in profiler timelines; without a profiler attached the ranges cost nothing measurable.
  */
 #ifndef SQNN_H_
 #define SQNN_H_

@@ -1,6 +1,8 @@
 // C entry points of the device side: argument checks and dispatch on the network shape.
 #include "sqnn.h"
 #include "sqnn_decode.cuh"
+#include <cstdlib>
+#include <nvtx3/nvToolsExt.h>
 #include "sqnn_launch.h"
 #include "sqnn_shapes.h"
 
@@ -116,14 +118,54 @@ int decode_bits_dispatch(const DecodeArgs &A, void *d_out, cudaStream_t st)
     return decode_shape<0, 0>(A, SQNN_OUT_BITS, nullptr, nullptr, 0, d_out, st);
 }
 
+namespace {
+bool checked_mode()
+{
+    static const bool on = [] {
+        const char *v = std::getenv("SQNN_DEBUG_CHECKS");
+        return v && v[0] == '1';
+    }();
+    return on;
+}
+nvtxDomainHandle_t nvtx_domain()
+{
+    static nvtxDomainHandle_t d = nvtxDomainCreateA("sqnn");
+    return d;
+}
+}  // namespace
+
+ApiScope::ApiScope(const char *name)
+{
+    nvtxEventAttributes_t a = {};
+    a.version = NVTX_VERSION;
+    a.size = NVTX_EVENT_ATTRIB_STRUCT_SIZE;
+    a.messageType = NVTX_MESSAGE_TYPE_ASCII;
+    a.message.ascii = name;
+    nvtxDomainRangePushEx(nvtx_domain(), &a);
+}
+ApiScope::~ApiScope() { nvtxDomainRangePop(nvtx_domain()); }
+
+int ApiScope::finish(int rc, const uint32_t *d_status, cudaStream_t st) const
+{
+    if (rc != SQNN_OK || !checked_mode()) return rc;
+    if (cudaStreamSynchronize(st) != cudaSuccess || cudaGetLastError() != cudaSuccess) return SQNN_E_CUDA;
+    if (d_status) {
+        uint32_t word = 0;
+        if (cudaMemcpy(&word, d_status, sizeof word, cudaMemcpyDeviceToHost) != cudaSuccess) return SQNN_E_CUDA;
+        if (word == (uint32_t)(-SQNN_E_TIMEOUT)) return SQNN_E_TIMEOUT;
+        if (word != 0) return SQNN_E_BAD_BLOB;
+    }
+    return SQNN_OK;
+}
+
 }  // namespace sqnn
 
 using namespace sqnn;
 
 
-extern "C" int sqnn_decode(const sqnn_desc *desc, const void *d_blob, const uint64_t *d_mask,
-                           const float *d_alpha, sqnn_out_mode mode, void *d_out, size_t out_bytes,
-                           uint32_t *d_status, void *cuda_stream)
+static int decode_queue(const sqnn_desc *desc, const void *d_blob, const uint64_t *d_mask,
+                        const float *d_alpha, sqnn_out_mode mode, void *d_out, size_t out_bytes,
+                        uint32_t *d_status, void *cuda_stream)
 {
     DecodeArgs A;
     int rc = fill_decode_args(desc, d_blob, d_status, &A);
@@ -144,6 +186,15 @@ extern "C" int sqnn_decode(const sqnn_desc *desc, const void *d_blob, const uint
     SQNN_FOR_SHAPES(SQNN_DECODE_CASE)
 #undef SQNN_DECODE_CASE
     return decode_shape<0, 0>(A, mode, d_mask, d_alpha, desc->n, d_out, st);
+}
+
+extern "C" int sqnn_decode(const sqnn_desc *desc, const void *d_blob, const uint64_t *d_mask,
+                           const float *d_alpha, sqnn_out_mode mode, void *d_out, size_t out_bytes,
+                           uint32_t *d_status, void *cuda_stream)
+{
+    ApiScope scope("sqnn_decode");
+    return scope.finish(decode_queue(desc, d_blob, d_mask, d_alpha, mode, d_out, out_bytes, d_status, cuda_stream),
+                        d_status, (cudaStream_t)cuda_stream);
 }
 
 namespace sqnn {
@@ -189,10 +240,10 @@ extern "C" size_t sqnn_workspace_bytes(const sqnn_desc *desc, uint32_t batch)
     return mma_workspace_bytes(desc, batch);
 }
 
-extern "C" int sqnn_decode_matmul(const sqnn_desc *desc, const void *d_blob, const uint64_t *d_mask,
-                                  const float *d_alpha, const void *d_x, int x_dtype, uint32_t batch,
-                                  int64_t ldx, float *d_y, int64_t ldy, void *d_workspace,
-                                  size_t workspace_bytes, uint32_t *d_status, void *cuda_stream)
+static int decode_matmul_queue(const sqnn_desc *desc, const void *d_blob, const uint64_t *d_mask,
+                               const float *d_alpha, const void *d_x, int x_dtype, uint32_t batch,
+                               int64_t ldx, float *d_y, int64_t ldy, void *d_workspace,
+                               size_t workspace_bytes, uint32_t *d_status, void *cuda_stream)
 {
     DecodeArgs A;
     int rc = fill_decode_args(desc, d_blob, d_status, &A);
@@ -211,4 +262,15 @@ extern "C" int sqnn_decode_matmul(const sqnn_desc *desc, const void *d_blob, con
     if (!d_workspace || workspace_bytes < mma_workspace_bytes(desc, batch) || ((uintptr_t)d_workspace & 255))
         return SQNN_E_WORKSPACE;
     return mma_dispatch(desc, A, d_mask, d_alpha, d_x, ldx, batch, d_y, ldy, d_workspace, st);
+}
+
+extern "C" int sqnn_decode_matmul(const sqnn_desc *desc, const void *d_blob, const uint64_t *d_mask,
+                                  const float *d_alpha, const void *d_x, int x_dtype, uint32_t batch,
+                                  int64_t ldx, float *d_y, int64_t ldy, void *d_workspace,
+                                  size_t workspace_bytes, uint32_t *d_status, void *cuda_stream)
+{
+    ApiScope scope("sqnn_decode_matmul");
+    return scope.finish(decode_matmul_queue(desc, d_blob, d_mask, d_alpha, d_x, x_dtype, batch, ldx, d_y, ldy,
+                                            d_workspace, workspace_bytes, d_status, cuda_stream),
+                        d_status, (cudaStream_t)cuda_stream);
 }

@@ -809,6 +809,8 @@ int sqnn_load_host(const void *stored, size_t stored_bytes, void **blob, size_t 
         std::vector<std::vector<uint16_t>> dp16(h.n_q);
         for (uint32_t i = 0; i < h.n_q; ++i) {
             if (h.n_dp[i] > 0xffffffffull) return SQNN_E_BAD_BLOB;
+            // nothing is allocated for more slices than the rest of the buffer could hold seeds for
+            if (l > (uint64_t)(end - p) * 8 / h.n_in) return SQNN_E_BAD_BLOB;
             BitReader br(p, end);
             pa[i].wc.resize(l);
             pa[i].np.resize(l);
@@ -830,6 +832,7 @@ int sqnn_load_host(const void *stored, size_t stored_bytes, void **blob, size_t 
             }
             if (!br.ok || sum != h.n_dp[i]) return SQNN_E_BAD_BLOB;
             br.align();
+            if (w_dp && sum > (uint64_t)(end - br.p) * 8 / w_dp) return SQNN_E_BAD_BLOB;
             dp16[i].resize(sum ? sum : 1);
             for (uint64_t k = 0; k < sum; ++k) dp16[i][k] = (uint16_t)br.get(w_dp);
             if (!br.ok) return SQNN_E_BAD_BLOB;

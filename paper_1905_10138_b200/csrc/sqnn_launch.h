@@ -15,4 +15,16 @@ size_t mma_workspace_bytes(const sqnn_desc *desc, uint32_t batch);
 int mma_dispatch(const sqnn_desc *desc, const DecodeArgs &A, const uint64_t *d_mask, const float *d_alpha,
                  const void *d_x, int64_t ldx, uint32_t batch, float *d_y, int64_t ldy, void *d_workspace,
                  cudaStream_t st);
+
+// A device entry point: an NVTX range for its duration on the host, and in checked mode
+// (SQNN_DEBUG_CHECKS=1) the wait for the stream and the translation of what it left behind.
+class ApiScope {
+  public:
+    explicit ApiScope(const char *name);
+    ~ApiScope();
+    ApiScope(const ApiScope &) = delete;
+    ApiScope &operator=(const ApiScope &) = delete;
+    // rc of the queueing code -> what the entry point returns
+    int finish(int rc, const uint32_t *d_status, cudaStream_t st) const;
+};
 }  // namespace sqnn

@@ -622,10 +622,10 @@ int static_scratch_address(void **out)
 
 }  // namespace
 
-extern "C" int sqnn_decode_matmul_static(const sqnn_desc *desc, const void *d_blob, const uint64_t *d_mask,
-                                         const float *d_alpha, const void *d_x, int x_dtype, uint32_t batch,
-                                         int64_t ldx, float *d_y, int64_t ldy, uint32_t *d_status,
-                                         void *cuda_stream)
+static int decode_matmul_static_queue(const sqnn_desc *desc, const void *d_blob, const uint64_t *d_mask,
+                                      const float *d_alpha, const void *d_x, int x_dtype, uint32_t batch,
+                                      int64_t ldx, float *d_y, int64_t ldy, uint32_t *d_status,
+                                      void *cuda_stream)
 {
     sqnn::DecodeArgs A;
     int rc = sqnn::fill_decode_args(desc, d_blob, d_status, &A);
@@ -644,4 +644,15 @@ extern "C" int sqnn_decode_matmul_static(const sqnn_desc *desc, const void *d_bl
     // product stage reads.  Y is cleared by the product path itself.
     return sqnn::mma_dispatch(desc, A, d_mask, d_alpha, d_x, ldx, batch, d_y, ldy, scratch,
                               (cudaStream_t)cuda_stream);
+}
+
+extern "C" int sqnn_decode_matmul_static(const sqnn_desc *desc, const void *d_blob, const uint64_t *d_mask,
+                                         const float *d_alpha, const void *d_x, int x_dtype, uint32_t batch,
+                                         int64_t ldx, float *d_y, int64_t ldy, uint32_t *d_status,
+                                         void *cuda_stream)
+{
+    sqnn::ApiScope scope("sqnn_decode_matmul_static");
+    return scope.finish(decode_matmul_static_queue(desc, d_blob, d_mask, d_alpha, d_x, x_dtype, batch, ldx, d_y, ldy,
+                                                   d_status, cuda_stream),
+                        d_status, (cudaStream_t)cuda_stream);
 }

@@ -112,9 +112,9 @@ k_search_seeds(const __grid_constant__ SearchArgs S)
 
 }  // namespace sqnn
 
-extern "C" int sqnn_search_seeds(const sqnn_xornet *net, uint64_t m, uint64_t n, uint32_t n_q,
-                                 const uint64_t *d_planes, const uint64_t *d_mask, uint32_t *d_wc,
-                                 uint16_t *d_np, void *cuda_stream)
+static int search_seeds_queue(const sqnn_xornet *net, uint64_t m, uint64_t n, uint32_t n_q,
+                              const uint64_t *d_planes, const uint64_t *d_mask, uint32_t *d_wc,
+                              uint16_t *d_np, void *cuda_stream)
 {
     using namespace sqnn;
     if (!net || !net->rows || !d_planes || !d_mask || !d_wc || !d_np) return SQNN_E_INVALID_ARG;
@@ -140,4 +140,13 @@ extern "C" int sqnn_search_seeds(const sqnn_xornet *net, uint64_t m, uint64_t n,
     else if (nw <= 4) k_search_seeds<4><<<(uint32_t)blocks, 256, 0, st>>>(S);
     else k_search_seeds<8><<<(uint32_t)blocks, 256, 0, st>>>(S);
     return cudaGetLastError() == cudaSuccess ? SQNN_OK : SQNN_E_CUDA;
+}
+
+extern "C" int sqnn_search_seeds(const sqnn_xornet *net, uint64_t m, uint64_t n, uint32_t n_q,
+                                 const uint64_t *d_planes, const uint64_t *d_mask, uint32_t *d_wc,
+                                 uint16_t *d_np, void *cuda_stream)
+{
+    sqnn::ApiScope scope("sqnn_search_seeds");
+    return scope.finish(search_seeds_queue(net, m, n, n_q, d_planes, d_mask, d_wc, d_np, cuda_stream), nullptr,
+                        (cudaStream_t)cuda_stream);
 }

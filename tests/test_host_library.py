@@ -325,3 +325,11 @@ def test_storage_form_dense_region_case_and_rejection_of_damaged_buffers():
     widths_at = 128 + 4 * n_out + (l * n_in + 7) // 8           # header, rows of M, seed stream
     b = blocked.copy(); b[widths_at + 4] = 0; bad(b)            # the busy block's width set to 0: counts no longer add up
     b = blocked.copy(); b[widths_at + 4] = 12; bad(b)           # a width no count needs
+    # a header that claims far more rows than the buffer could hold seeds for is refused before anything of
+    # that size is allocated (m is the first 64-bit field after the magic)
+    import time
+    b = blocked.copy()
+    b[8 + 3] |= 0x40                                            # m += 2^30: 10^9 slices claimed
+    t0 = time.perf_counter()
+    bad(b)
+    assert time.perf_counter() - t0 < 1.0
