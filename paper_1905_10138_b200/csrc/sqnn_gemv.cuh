@@ -12,6 +12,10 @@
 // clearing of Y.  Everything the walk reads is on chip: tables, decoded bits, mask words, the
 // scales of the block's rows and (XS = true) the activations of the current batch chunk as
 // xs[c][BT].  Rows that do not fit shared memory at once are taken in chunks.
+// With one activation vector and 16-byte aligned operands the tables, the activations and the mask
+// range of a block's first chunk are fetched by three bulk copies (cp.async.bulk, completion on an
+// mbarrier, bounded wait) that thread 0 issues at kernel entry; otherwise by cp.async from every
+// thread.
 #pragma once
 #include "sqnn_kernels.cuh"
 
@@ -31,7 +35,38 @@ struct GemvArgs {
     uint32_t rows_per_block, rows_per_chunk, parts;
     uint32_t region_words;        // words of one bit vector of a chunk in shared memory (whole kernel tiles)
     uint32_t alpha_words, part_words, xs_words;
+    uint32_t bulk_stage;          // tables, activations and mask may be staged by bulk copies (sizes and alignment allow it)
 };
+
+// One-dimensional bulk copy global -> shared by the copy engine, completion counted in bytes on an
+// mbarrier; both addresses 16-byte aligned, size a multiple of 16.
+SQNN_DEV void stage_bar_init(uint64_t *bar)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;\n" :: "r"(smem_addr(bar)) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+}
+SQNN_DEV void stage_bar_expect(uint64_t *bar, uint32_t bytes)
+{
+    asm volatile("{\n .reg .b64 st;\n mbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1;\n}\n"
+                 :: "r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+SQNN_DEV void bulk_load(void *sdst, const void *gsrc, uint32_t bytes, uint64_t *bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n"
+                 :: "r"(smem_addr(sdst)), "l"(gsrc), "r"(bytes), "r"(smem_addr(bar)) : "memory");
+}
+// Waits for phase 0 of the barrier, for about a second at most; false if it gave up.
+SQNN_DEV bool stage_bar_wait(uint64_t *bar)
+{
+    const long long t0 = clock64();
+    for (;;) {
+        uint32_t ok;
+        asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], 0, %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+                     : "=r"(ok) : "r"(smem_addr(bar)), "r"(1000000u) : "memory");
+        if (ok) return true;
+        if (clock64() - t0 > 2000000000ll) return false;
+    }
+}
 
 SQNN_DEV float to_float(float v) { return v; }
 SQNN_DEV float to_float(__nv_bfloat16 v) { return __bfloat162float(v); }
@@ -122,8 +157,29 @@ k_decode_gemv(const GemvArgs g)
         cp_async_commit();
     };
 
-    tables_request(A, tab_s);                                    // commit group: tables
-    stage_x(0);                                                  // commit group: activations
+    // With one activation vector and everything 16-byte aligned, thread 0 hands the three big transfers of the
+    // block's first chunk -- tables, activations, mask -- to the copy engine at once, before anything else
+    // runs; otherwise every thread requests its share by cp.async (three commit groups, as below).
+    __shared__ uint64_t stage_bar;
+    bool bulk = false;
+    if constexpr (XS && BT == 1) {
+        const uint64_t tile_bits = 32ull * TW;
+        const uint64_t rb0 = row0 + g.rows_per_chunk < row_end ? row0 + g.rows_per_chunk : row_end;
+        const uint64_t k0 = (row0 * n) / tile_bits, k1 = (rb0 * n + tile_bits - 1) / tile_bits;
+        bulk = g.bulk_stage && row0 < row_end && k1 * TW <= g.mask_words;      // the mask range lies inside the array
+        if (bulk && threadIdx.x == 0) {
+            const uint32_t tab_bytes = A.tab_words * 4, x_bytes = n * (uint32_t)sizeof(XT), mask_bytes = (uint32_t)(k1 - k0) * TW * 4;
+            stage_bar_init(&stage_bar);
+            stage_bar_expect(&stage_bar, tab_bytes + x_bytes + mask_bytes);
+            bulk_load(tab_s, A.tab, tab_bytes, &stage_bar);
+            bulk_load(xs, x, x_bytes, &stage_bar);
+            bulk_load(mask_s, g.mask32 + k0 * TW, mask_bytes, &stage_bar);
+        }
+    }
+    if (!bulk) {
+        tables_request(A, tab_s);                                // commit group: tables
+        stage_x(0);                                              // commit group: activations
+    }
     uint32_t xs_holds = 0;                                       // batch chunk in xs
 
     for (uint64_t ra = row0; ra < row_end; ra += g.rows_per_chunk) {
@@ -135,7 +191,8 @@ k_decode_gemv(const GemvArgs g)
         const uint32_t nt = (uint32_t)(kt1 - kt0);
         const uint64_t gw0 = kt0 * TW;                           // first word of the chunk's regions
         if (ra != row0) __syncthreads();                         // the walk of the previous chunk is over
-        stage_mask(mask_s, g.mask32, gw0, g.mask_words, nt * TW, threadIdx.x, blockDim.x, mask_vec);
+        if (!(bulk && ra == row0))
+            stage_mask(mask_s, g.mask32, gw0, g.mask_words, nt * TW, threadIdx.x, blockDim.x, mask_vec);
         for (uint32_t i = threadIdx.x; i < nrows * n_q; i += blockDim.x) cp_async4(alpha_s + i, g.alpha + ra * n_q + i);
         cp_async_commit();                                       // commit group: mask and scales
 
@@ -156,8 +213,13 @@ k_decode_gemv(const GemvArgs g)
             };
             if (item < items) fetch(item);
             if (ra == row0) {
-                cp_async_wait_group<2>();                        // tables (the two younger groups may be pending)
-                __syncthreads();
+                if (bulk) {
+                    __syncthreads();                             // the barrier's initialisation is visible to all
+                    if (!stage_bar_wait(&stage_bar)) flag(A.status, (uint32_t)(-SQNN_E_TIMEOUT));
+                } else {
+                    cp_async_wait_group<2>();                    // tables (the two younger groups may be pending)
+                    __syncthreads();
+                }
             }
             while (item < items) {
                 const uint32_t t = item / n_q, pl = item - t * n_q;
@@ -170,8 +232,13 @@ k_decode_gemv(const GemvArgs g)
             }
         } else {
             if (ra == row0) {
-                cp_async_wait_group<2>();
-                __syncthreads();
+                if (bulk) {
+                    __syncthreads();
+                    if (!stage_bar_wait(&stage_bar)) flag(A.status, (uint32_t)(-SQNN_E_TIMEOUT));
+                } else {
+                    cp_async_wait_group<2>();
+                    __syncthreads();
+                }
             }
             for (; item < items; item += nwarps) {
                 const uint32_t t = item / n_q, pl = item - t * n_q;
@@ -338,6 +405,10 @@ inline int launch_gemv_bt(const DecodeArgs &A, const uint64_t *d_mask, const flo
         if (xs) { xs = false; RC = R; continue; }               // leave the activations in global memory
         return SQNN_E_UNSUPPORTED;                               // one row of bits does not fit
     }
+    // bulk staging of the first chunk: one activation vector in shared memory, 16-byte aligned sources and sizes
+    g.bulk_stage = (BT == 1 && xs && ((uintptr_t)d_x & 15) == 0 && (n * sizeof(XT)) % 16 == 0 &&
+                    ((uintptr_t)d_mask & 15) == 0 && ((uintptr_t)A.tab & 15) == 0 && (tab + 0) % 16 == 0 &&
+                    (size_t)g.region_words * 4 < (1u << 20)) ? 1u : 0u;
 #define SQNN_GEMV_LAUNCH(XSV, NQV)                                                                       \
     do {                                                                                                 \
         auto k = k_decode_gemv<N_OUT, N_IN, BT, XT, XSV, NQV>;                                           \
