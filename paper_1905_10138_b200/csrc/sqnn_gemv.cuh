@@ -352,7 +352,7 @@ template <int N_OUT, int N_IN, int BT, typename XT>
 inline int launch_gemv_bt(const DecodeArgs &A, const uint64_t *d_mask, const float *d_alpha, const void *d_x,
                           int64_t ldx, uint32_t batch, float *d_y, int64_t ldy, uint64_t m, uint64_t n, cudaStream_t st)
 {
-    constexpr uint32_t nwarps = 32;
+    uint32_t nwarps = 32;
     const size_t limit = 220 * 1024;
     const uint32_t sms = (uint32_t)sm_count();
     GemvArgs g;
@@ -366,6 +366,16 @@ inline int launch_gemv_bt(const DecodeArgs &A, const uint64_t *d_mask, const flo
     const uint64_t grid = (m + R - 1) / R;
     if (R > 0xffffffffull) return SQNN_E_UNSUPPORTED;
     g.rows_per_block = (uint32_t)R;
+    {
+        // a block with a few rows and a few tiles to decode gets a few warps: a thread block is cheaper to start
+        // and to synchronise the smaller it is (tiny layers are all launch and latency)
+        const uint64_t tb = 32ull * 32ull * A.W;
+        const uint64_t items = ((R * n + tb - 1) / tb + 1) * A.n_q;
+        const uint64_t want = R > items ? R : items;
+        if (want <= 4) nwarps = 4;
+        else if (want <= 8) nwarps = 8;
+        else if (want <= 16) nwarps = 16;
+    }
     const uint64_t TW = 32ull * A.W, tile_bits = 32 * TW;
     const size_t tab = (size_t)A.tab_words * 4;
     const size_t xbytes = ((size_t)n * BT * sizeof(XT) + 15) & ~(size_t)15;
